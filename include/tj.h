@@ -1,0 +1,216 @@
+/*
+ * tj.h -- C ABI of the B200 (sm_100a) sample production/consumption library.
+ *
+ * The library runs, on ONE GPU and ONE CUDA stream, the data-parallel hot path of
+ * a TianJi-style actor/buffer/learner pipeline (arXiv 2502.20190):
+ *
+ *   actor   (Sec. 3.1, actor loop; Algorithm 1 tasks 1-2):
+ *           observation -> policy MLP -> epsilon-greedy / categorical action ->
+ *           vectorised environment step -> version-tagged trajectory record
+ *   buffer  (Sec. 3.1, buffer loop; dependency III relaxed into an asynchronous
+ *           hand-over): a replay ring of (s, a, r, s', done, version) records, or
+ *           rollout segments for the on-policy case
+ *   learner (Sec. 3.1, learner loop; Sec. 3.3 and Eq. 2-3 for staleness control):
+ *           staleness-bounded minibatch sampling, gather, online/target forward,
+ *           TD target and Huber error (Algorithm 1, TD-error line); GAE for the
+ *           on-policy case (Table 2: gae 0.95, gamma 0.99)
+ *   weights (dependency I relaxed): the learner publishes a new parameter version,
+ *           the actor picks up the newest one at its next call.
+ *
+ * Conventions
+ *   - Every function returns a tj_status (0 = OK, negative = error).  Nothing
+ *     throws, aborts or prints.  tj_last_error() gives a readable message.
+ *   - All device work is enqueued on the stream given to tj_create; calls are
+ *     asynchronous with respect to the host unless stated otherwise, and take
+ *     effect in host call order.
+ *   - OWNERSHIP: the caller owns every byte of device memory.  tj_query_workspace
+ *     reports how much the context needs, tj_create carves the caller's buffer.
+ *     The library never calls cudaMalloc/cudaFree.  tj_ctx is a small host object.
+ *   - Pointers are DEVICE pointers unless the parameter name starts with host_ or
+ *     the comment says "host".  Arrays are dense and row-major.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ *   - Host-detectable errors are returned before anything is enqueued.
+ */
+#ifndef TJ_H
+#define TJ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tj_ctx tj_ctx;
+
+typedef enum {
+  TJ_OK = 0,
+  TJ_ERR_INVALID_ARG = -1,   /* null pointer, negative size, wrong blob length ... */
+  TJ_ERR_CONFIG = -2,        /* inconsistent tj_config */
+  TJ_ERR_WORKSPACE = -3,     /* workspace too small or misaligned */
+  TJ_ERR_CUDA = -4,          /* a CUDA runtime call failed; see tj_last_error */
+  TJ_ERR_NO_WEIGHTS = -5,    /* actor or learner called before the first publish */
+  TJ_ERR_WARMUP = -6,        /* fewer resident records than cfg.warmup (Table 2: buffer warmup size) */
+  TJ_ERR_STARVED = -7,       /* nothing eligible: the consumer is ahead of the producer (Eq. 3: TR_L ~ TR_A) */
+  TJ_ERR_STALE_SEGMENT = -8, /* reserved */
+  TJ_ERR_TIMEOUT = -9,       /* reserved */
+  TJ_ERR_UNSUPPORTED = -10   /* valid request this build does not implement */
+} tj_status;
+
+enum { TJ_ENV_CARTPOLE = 0, TJ_ENV_ACROBOT = 1, TJ_ENV_LINGAUSS = 2 };
+enum { TJ_POLICY_EPS_GREEDY = 0, TJ_POLICY_CATEGORICAL = 1 };
+enum { TJ_W_FP32 = 0, TJ_W_BF16 = 1 };
+
+/* Configuration (App. B: one configuration with distribution / training / model / environment groups). */
+typedef struct {
+  uint32_t struct_size;          /* = sizeof(tj_config); lets the struct grow */
+  int32_t device;                /* CUDA device ordinal the workspace lives on */
+  /* environment group */
+  int32_t env_kind;              /* TJ_ENV_* */
+  int32_t n_envs;                /* N, environments stepped together */
+  int32_t obs_dim;               /* D: 4 CartPole, 6 Acrobot, multiple of 4 (<= 128) LinGauss */
+  int32_t n_actions;             /* A: 2 CartPole, 3 Acrobot, <= 64 LinGauss */
+  int32_t max_episode_steps;     /* 0 = env default (500 / 500 / 200) */
+  float lg_done_norm;            /* LinGauss: terminate when ||s'|| exceeds this (4) */
+  float lg_noise_std;            /* LinGauss: noise scale (0.01) */
+  const float *host_lg_A;        /* LinGauss: A [D][D], HOST pointer, copied at create */
+  const float *host_lg_B;        /* LinGauss: B [A][D], HOST pointer, copied at create */
+  /* model group */
+  int32_t hidden;                /* H, width of both hidden ReLU layers */
+  int32_t policy_kind;           /* TJ_POLICY_*: Q head, or softmax head + value head */
+  int32_t weight_dtype;          /* TJ_W_FP32: FP32 FMA in a fixed rounding order; TJ_W_BF16: tensor cores */
+  float epsilon;                 /* exploration rate (eps-greedy) */
+  uint64_t seed;                 /* Philox key */
+  /* training / distribution group */
+  int64_t replay_capacity;       /* C, multiple of n_envs; 0 => on-policy segment mode */
+  int32_t minibatch;             /* B */
+  int32_t staleness_bound;       /* S: a record is eligible iff learner_version - record_version <= S */
+  int32_t warmup;                /* minimum resident records before sampling */
+  int32_t rollout_len;           /* T (segment mode) */
+  int32_t n_segments;            /* segment slots (segment mode) */
+  int32_t target_sync_interval;  /* learner steps between target-network refreshes (Table 2) */
+  float gamma, huber_delta, gae_lambda;
+} tj_config;
+
+/* A gathered minibatch: caller-owned device arrays, n rows each. */
+typedef struct {
+  int32_t n;
+  float *obs;        /* [n][D] */
+  int32_t *act;      /* [n] */
+  float *rew;        /* [n] */
+  float *next_obs;   /* [n][D] */
+  int32_t *done;     /* [n] */
+  int32_t *ver;      /* [n] policy version that produced the record */
+} tj_batch;
+
+/* A rollout segment: a view into the context's workspace, valid until the producer reuses the slot. */
+typedef struct {
+  int32_t T, N;
+  int64_t version;   /* policy version in force when the segment's first step ran */
+  const float *obs;      /* [T][N][D] */
+  const int32_t *act;    /* [T][N] */
+  const float *rew;      /* [T][N] */
+  const uint8_t *done;   /* [T][N] */
+  const float *logp;     /* [T][N] */
+  const float *val;      /* [T+1][N]; row T is the bootstrap value of the state after the last step */
+} tj_segment;
+
+/* Environment state and counters (views into the workspace / values to restore). */
+typedef struct {
+  float *state;          /* [N][S_d], S_d = 4 (CartPole, Acrobot) or D (LinGauss) */
+  int32_t *ep_step;      /* [N] steps taken in the running episode */
+  uint64_t cursor;       /* transitions ever written to the ring */
+  int64_t t;             /* actor steps taken so far (per env) */
+  int64_t k;             /* learner steps taken so far */
+  int64_t actor_version, learner_version;
+} tj_state_view;
+
+/* Production/consumption and staleness statistics (Eq. 2-3; Table 1 columns). */
+typedef struct {
+  int64_t produced;             /* transitions written */
+  int64_t consumed;             /* transitions handed to the learner */
+  int64_t dropped_stale;        /* resident records (or segment transitions) refused for staleness */
+  int64_t dropped_overwritten;  /* segment transitions overwritten before they were consumed */
+  int64_t starved_calls;
+  int64_t actor_version, learner_version, actor_steps, learner_steps;
+  int64_t max_sampled_staleness;
+  int64_t episodes_finished;
+  double return_sum;            /* sum of the returns of finished episodes */
+  int64_t staleness_hist[33];   /* sampled staleness 0..31, last bin = 32 and more */
+  int64_t device_error;         /* 0, or a code latched by a kernel's own bounds check */
+} tj_stats_t;
+
+/* Bytes (and alignment) of device memory a context with this configuration needs. */
+int tj_query_workspace(const tj_config *cfg, size_t *bytes, size_t *align);
+
+/* Build a context inside `workspace` (device memory, >= bytes, aligned as reported) on `cuda_stream`
+ * (a cudaStream_t; NULL = the legacy default stream).  Seeds every environment from the reset stream.
+ * Errors: INVALID_ARG, CONFIG, WORKSPACE, CUDA. */
+int tj_create(const tj_config *cfg, void *workspace, size_t bytes, void *cuda_stream, tj_ctx **out);
+
+/* Free the host object.  Does not touch the workspace.  Synchronises the stream. */
+int tj_destroy(tj_ctx *ctx);
+
+/* Learner -> actor hand-over of parameters (Sec. 3.1: the learner stores the model and a trigger decides
+ * when to send it; dependency I as an asynchronous exchange).  `blob` holds FP32
+ *   [W1 HxD, b1 H, W2 HxH, b2 H, W3 AxH, b3 A (, Wv 1xH, bv 1 when policy_kind = categorical)]
+ * row-major (out x in); nbytes must match exactly.  on_device = 0: host pointer (copied before return);
+ * 1: device pointer (read on the stream).  The new parameters become version+1 (returned in version_out)
+ * and are what the actor uses from its next call and what the learner's online forward uses.  The target
+ * network takes the same parameters on the first publish and then on the first publish after
+ * target_sync_interval further learner steps.  With TJ_W_BF16 the weight matrices are rounded to bfloat16
+ * (nearest even); biases stay FP32. */
+int tj_publish_weights(tj_ctx *ctx, const void *blob, size_t nbytes, int32_t on_device, int64_t *version_out);
+
+/* Actor: n_steps environment steps for all N environments (Algorithm 1: policy inference, then
+ * simulation, then the trajectory tuple; Sec. 3.1 actor loop).  Per env e and global step t:
+ *   logits = MLP(obs);  action from the ACTION Philox words of (e, t);  env step;  done = terminated or
+ *   step limit;  record (obs, a, r, next_obs before reset, done, version) at ring slot (cursor + e) mod C
+ *   (or into the running segment);  done envs are re-seeded from the RESET words of (e, t).
+ * After each step cursor += N.  dbg_logits (nullable) receives [n_steps][N][A] network outputs.
+ * Errors: INVALID_ARG, NO_WEIGHTS, CUDA. */
+int tj_actor_step(tj_ctx *ctx, int32_t n_steps, float *dbg_logits);
+
+/* Learner, step 1 (Sec. 3.1: loading trajectories; Sec. 3.3 / Eq. 2-3 / App. D.1: controlling sample
+ * staleness).  E = valid slots with learner_version - version <= S in ascending slot order; draw j of
+ * learner step k takes E[mulhi(x0, |E|)], x0 from the SAMPLE Philox words of (j, k); with replacement.
+ * staleness_bound = -1 uses the configured S.  idx_out (nullable) receives the B slots; `out` arrays
+ * receive the gathered rows bit for bit.  Errors: NO_WEIGHTS, WARMUP, STARVED (nothing enqueued, k unchanged). */
+int tj_replay_sample(tj_ctx *ctx, int32_t staleness_bound, int32_t *idx_out, const tj_batch *out);
+
+/* Learner, step 2, forward half (Algorithm 1: delta = r + gamma V(s') - V(s), here with a target network
+ * and a done mask): q = Q_online(obs)[act]; q' = max_a Q_target(next_obs); y = r + gamma (1-done) q';
+ * delta = y - q; Huber(delta; huber_delta).  td_out, huber_out: [n] (nullable); loss_mean_out: 1 float
+ * (nullable), the mean Huber loss summed in a fixed order. */
+int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
+
+/* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
+ *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0;
+ *   R_t = A_t + V_t.   rew [T][N], val [T+1][N], done [T][N] -> adv [T][N], ret [T][N].
+ * ctx supplies only the stream. */
+int tj_gae(tj_ctx *ctx, const float *rew, const float *val, const uint8_t *done, int32_t T, int32_t N, float gamma,
+           float lambda, float *adv_out, float *ret_out);
+
+/* On-policy consumption (App. D.1: buffer = batch, staleness controlled by how far the learner has moved
+ * on): the oldest complete, unconsumed segment whose version is at most S behind the learner; staler ones
+ * are dropped and counted.  Errors: STARVED. */
+int tj_segment_acquire(tj_ctx *ctx, tj_segment *out);
+
+/* Views of the env state and the counters; no copy, no synchronisation. */
+int tj_get_state(tj_ctx *ctx, tj_state_view *out);
+/* Restore env state (device pointers, nullable = keep) and the cursor / t / k counters; versions are ignored. */
+int tj_set_state(tj_ctx *ctx, const tj_state_view *in);
+
+/* Counters (Eq. 2-3: produced vs consumed, sampled staleness).  Synchronises the stream. */
+int tj_stats(tj_ctx *ctx, tj_stats_t *host_out);
+
+/* Views into the ring for inspection: records [C][2D+4] (obs, next_obs, act, rew, done, ver as 32-bit words)
+ * and the per-block version summary [C/N]. */
+int tj_ring_view(tj_ctx *ctx, const float **records, const int32_t **block_version, int32_t *record_words);
+
+const char *tj_last_error(const tj_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TJ_H */

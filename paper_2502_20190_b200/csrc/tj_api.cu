@@ -1,0 +1,454 @@
+// C ABI shell: configuration checks, workspace carving, host-side bookkeeping (versions, cursor, segment
+// slots, counters) and the kernel launches behind each entry point.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "tj_internal.h"
+
+using namespace tj;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxTdRows = 1 << 20;
+
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+  template <typename T>
+  T* take(size_t count) {
+    off = (off + kAlign - 1) & ~(kAlign - 1);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+int env_state_dim(const tj_config& c) { return c.env_kind == TJ_ENV_LINGAUSS ? c.obs_dim : 4; }
+
+const char* validate(const tj_config* c) {
+  if (!c) return "null config";
+  if (c->struct_size != sizeof(tj_config)) return "struct_size does not match this library's tj_config";
+  if (c->n_envs < 1) return "n_envs must be positive";
+  if (c->hidden < 1 || c->hidden > 4096) return "hidden out of range";
+  if (c->n_actions < 1 || c->n_actions > 64) return "n_actions out of range";
+  switch (c->env_kind) {
+    case TJ_ENV_CARTPOLE:
+      if (c->obs_dim != 4 || c->n_actions != 2) return "CartPole needs obs_dim 4 and 2 actions";
+      break;
+    case TJ_ENV_ACROBOT:
+      if (c->obs_dim != 6 || c->n_actions != 3) return "Acrobot needs obs_dim 6 and 3 actions";
+      break;
+    case TJ_ENV_LINGAUSS:
+      if (c->obs_dim < 4 || c->obs_dim > 128 || c->obs_dim % 4) return "LinGauss needs obs_dim a multiple of 4, at most 128";
+      if (!c->host_lg_A || !c->host_lg_B) return "LinGauss needs host_lg_A and host_lg_B";
+      break;
+    default:
+      return "unknown env_kind";
+  }
+  if (c->policy_kind != TJ_POLICY_EPS_GREEDY && c->policy_kind != TJ_POLICY_CATEGORICAL) return "unknown policy_kind";
+  if (c->weight_dtype != TJ_W_FP32 && c->weight_dtype != TJ_W_BF16) return "unknown weight_dtype";
+  if (!(c->epsilon >= 0.f && c->epsilon <= 1.f)) return "epsilon must lie in [0,1]";
+  if (c->max_episode_steps < 0) return "max_episode_steps must not be negative";
+  if (c->replay_capacity < 0) return "replay_capacity must not be negative";
+  if (c->replay_capacity > 0) {
+    if (c->replay_capacity % c->n_envs) return "replay_capacity must be a multiple of n_envs";
+    if (c->replay_capacity > (int64_t)1 << 31) return "replay_capacity too large";
+    if (c->minibatch < 1 || c->minibatch > kMaxTdRows) return "minibatch out of range";
+    if (c->staleness_bound < 0 || c->warmup < 0) return "staleness_bound and warmup must not be negative";
+    if (c->policy_kind != TJ_POLICY_EPS_GREEDY) return "the replay ring is used with the eps-greedy Q head";
+  } else {
+    if (c->rollout_len < 1 || c->n_segments < 1) return "segment mode needs rollout_len and n_segments";
+    if (c->env_kind == TJ_ENV_LINGAUSS) return "segment mode is implemented for CartPole and Acrobot";
+    if (c->policy_kind != TJ_POLICY_CATEGORICAL) return "segment mode is used with the categorical policy";
+    if (c->staleness_bound < 0) return "staleness_bound must not be negative";
+  }
+  if (c->target_sync_interval < 0) return "target_sync_interval must not be negative";
+  return nullptr;
+}
+
+size_t blob_floats(int D, int H, int A, int vh) {
+  return (size_t)H * D + H + (size_t)H * H + H + (size_t)A * H + A + (vh ? (size_t)H + 1 : 0);
+}
+
+// one pass decides every address; base == nullptr only measures
+size_t carve(tj_ctx* x, void* base) {
+  const tj_config& c = x->cfg;
+  Carver cv(base);
+  const int N = c.n_envs, D = c.obs_dim, S_d = env_state_dim(c);
+  const int vh = c.policy_kind == TJ_POLICY_CATEGORICAL;
+  const WeightLayout wl = make_weight_layout(D, c.hidden, c.n_actions, vh);
+  x->state = cv.take<float>((size_t)N * S_d);
+  x->ep_step = cv.take<int>(N);
+  x->ep_return = cv.take<float>(N);
+  x->wbuf[0] = cv.take<float>(wl.total);
+  x->wbuf[1] = cv.take<float>(wl.total);
+  x->wtarget = cv.take<float>(wl.total);
+  x->blob_stage = cv.take<float>(blob_floats(D, c.hidden, c.n_actions, vh));
+  x->dstats = cv.take<DevStats>(1);
+  x->td_partial = cv.take<float>((size_t)td_grid(kMaxTdRows));
+  if (c.replay_capacity > 0) {
+    const size_t nb = (size_t)(c.replay_capacity / N);
+    x->ring = cv.take<float>((size_t)c.replay_capacity * (2 * D + 4));
+    x->block_ver = cv.take<int>(nb);
+    x->elig_list = cv.take<int>(nb);
+    x->elig_count = cv.take<int>(1);
+  } else {
+    const size_t TN = (size_t)c.rollout_len * N, G = c.n_segments;
+    x->seg_obs = cv.take<float>(G * TN * D);
+    x->seg_act = cv.take<int>(G * TN);
+    x->seg_rew = cv.take<float>(G * TN);
+    x->seg_logp = cv.take<float>(G * TN);
+    x->seg_val = cv.take<float>(G * ((size_t)c.rollout_len + 1) * N);
+    x->seg_done = cv.take<uint8_t>(G * TN);
+  }
+  if (c.env_kind == TJ_ENV_LINGAUSS) {
+    x->lgAt = cv.take<float>((size_t)D * round_up4(D));
+    x->lgB = cv.take<float>((size_t)c.n_actions * round_up4(D));
+    x->lg_stage = cv.take<float>((size_t)D * D + (size_t)c.n_actions * D);
+  }
+  return (cv.off + kAlign - 1) & ~(kAlign - 1);
+}
+
+int fail(tj_ctx* x, int code, const char* msg) {
+  if (x) x->err = msg;
+  return code;
+}
+int cuda_fail(tj_ctx* x, cudaError_t e, const char* where) {
+  if (x) x->err = std::string(where) + ": " + cudaGetErrorString(e);
+  return TJ_ERR_CUDA;
+}
+
+thread_local std::string g_err;  // for failures before a context exists
+
+uint64_t explore_threshold(float eps) {
+  const double e = (double)eps;
+  if (!(e > 0.0)) return 0;
+  if (e >= 1.0) return 4294967296ull;
+  return (uint64_t)std::floor(e * 4294967296.0);
+}
+
+}  // namespace
+
+extern "C" {
+
+int tj_query_workspace(const tj_config* cfg, size_t* bytes, size_t* align) {
+  const char* why = validate(cfg);
+  if (why) { g_err = why; return TJ_ERR_CONFIG; }
+  if (!bytes) { g_err = "bytes is null"; return TJ_ERR_INVALID_ARG; }
+  tj_ctx tmp{};
+  tmp.cfg = *cfg;
+  *bytes = carve(&tmp, nullptr);
+  if (align) *align = kAlign;
+  return TJ_OK;
+}
+
+int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_stream, tj_ctx** out) {
+  if (!out) { g_err = "out is null"; return TJ_ERR_INVALID_ARG; }
+  *out = nullptr;
+  const char* why = validate(cfg);
+  if (why) { g_err = why; return TJ_ERR_CONFIG; }
+  if (!workspace) { g_err = "workspace is null"; return TJ_ERR_INVALID_ARG; }
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) { g_err = "workspace is not 256-byte aligned"; return TJ_ERR_WORKSPACE; }
+  tj_ctx* x = new (std::nothrow) tj_ctx{};
+  if (!x) { g_err = "out of host memory"; return TJ_ERR_INVALID_ARG; }
+  x->cfg = *cfg;
+  x->cfg.host_lg_A = x->cfg.host_lg_B = nullptr;
+  const size_t need = carve(x, workspace);
+  if (bytes < need) { delete x; g_err = "workspace smaller than tj_query_workspace reports"; return TJ_ERR_WORKSPACE; }
+  x->stream = static_cast<cudaStream_t>(cuda_stream);
+  x->N = cfg->n_envs; x->D = cfg->obs_dim; x->H = cfg->hidden; x->A = cfg->n_actions;
+  x->S_d = env_state_dim(*cfg);
+  x->value_head = cfg->policy_kind == TJ_POLICY_CATEGORICAL;
+  x->rec_words = 2 * x->D + 4;
+  x->max_ep = cfg->max_episode_steps > 0 ? cfg->max_episode_steps : (cfg->env_kind == TJ_ENV_LINGAUSS ? 200 : 500);
+  x->n_blob = blob_floats(x->D, x->H, x->A, x->value_head);
+  x->wl = make_weight_layout(x->D, x->H, x->A, x->value_head);
+  x->active = 0; x->version = 0; x->k_last_sync = 0; x->has_target = false;
+  x->t = 0; x->k = 0; x->cursor = 0; x->next_consume = 0;
+  std::memset(&x->hs, 0, sizeof(x->hs));
+  if (cfg->replay_capacity > 0) x->h_block_ver.assign((size_t)(cfg->replay_capacity / cfg->n_envs), 0);
+  else x->seg.assign((size_t)cfg->n_segments, SegSlot{});
+
+  cudaError_t e = cudaSetDevice(cfg->device);
+  if (e != cudaSuccess) { g_err = std::string("cudaSetDevice: ") + cudaGetErrorString(e); delete x; return TJ_ERR_CUDA; }
+  auto bail = [&](cudaError_t err, const char* where) {
+    g_err = std::string(where) + ": " + cudaGetErrorString(err);
+    delete x;
+    return (int)TJ_ERR_CUDA;
+  };
+  if ((e = cudaMemsetAsync(x->dstats, 0, sizeof(DevStats), x->stream)) != cudaSuccess) return bail(e, "memset stats");
+  if (cfg->replay_capacity > 0) {
+    if ((e = cudaMemsetAsync(x->block_ver, 0, sizeof(int) * x->h_block_ver.size(), x->stream)) != cudaSuccess)
+      return bail(e, "memset block versions");
+    if ((e = cudaMemsetAsync(x->elig_count, 0, sizeof(int), x->stream)) != cudaSuccess) return bail(e, "memset count");
+  }
+  if (cfg->env_kind == TJ_ENV_LINGAUSS) {
+    // stage A and B as given, then transpose/pad A on the device
+    const int D = x->D, Dp = round_up4(D), A = x->A;
+    float* stage = x->lg_stage;
+    if ((e = cudaMemcpyAsync(stage, cfg->host_lg_A, sizeof(float) * D * D, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess)
+      return bail(e, "copy A");
+    if ((e = cudaMemcpyAsync(stage + (size_t)D * D, cfg->host_lg_B, sizeof(float) * A * D, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess)
+      return bail(e, "copy B");
+    if ((e = launch_transpose_pad(stage, x->lgAt, D, D, Dp, x->stream)) != cudaSuccess) return bail(e, "transpose A");
+    // B [A][D] is used as it is: D is a multiple of 4, so rows are already 16-byte aligned
+    if ((e = cudaMemcpyAsync(x->lgB, stage + (size_t)D * D, sizeof(float) * A * D, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+      return bail(e, "copy B to its place");
+    if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e, "sync after LinGauss set-up");
+  }
+  const uint2 seed = make_uint2((uint32_t)cfg->seed, (uint32_t)(cfg->seed >> 32));
+  if ((e = launch_init_env(cfg->env_kind, x->N, x->S_d, seed, x->state, x->ep_step, x->ep_return, x->stream)) != cudaSuccess)
+    return bail(e, "init envs");
+  *out = x;
+  return TJ_OK;
+}
+
+int tj_destroy(tj_ctx* ctx) {
+  if (!ctx) return TJ_ERR_INVALID_ARG;
+  cudaStreamSynchronize(ctx->stream);
+  delete ctx;
+  return TJ_OK;
+}
+
+int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_device, int64_t* version_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!blob) return fail(x, TJ_ERR_INVALID_ARG, "blob is null");
+  if (nbytes != x->n_blob * sizeof(float)) return fail(x, TJ_ERR_INVALID_ARG, "blob size does not match the configured network");
+  cudaError_t e;
+  const float* src = static_cast<const float*>(blob);
+  if (!on_device) {
+    if ((e = cudaMemcpyAsync(x->blob_stage, blob, nbytes, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: host to device copy");
+    src = x->blob_stage;
+  }
+  const int next = x->active ^ 1;
+  float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
+  if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->stream)) != cudaSuccess)
+    return cuda_fail(x, e, "publish: repack");
+  if (x->version != 0) x->active = next;
+  x->version += 1;
+  if (!x->has_target || (x->cfg.target_sync_interval > 0 && x->k - x->k_last_sync >= x->cfg.target_sync_interval)) {
+    if ((e = cudaMemcpyAsync(x->wtarget, dst, x->wl.total * sizeof(float), cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: target refresh");
+    x->has_target = true;
+    x->k_last_sync = x->k;
+  }
+  if (!on_device) {
+    // the staging buffer is reused by the next host publish; the copy above already left host memory
+  }
+  if (version_out) *version_out = x->version;
+  return TJ_OK;
+}
+
+int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (n_steps < 0) return fail(x, TJ_ERR_INVALID_ARG, "n_steps is negative");
+  if (x->version == 0) return fail(x, TJ_ERR_NO_WEIGHTS, "actor called before the first publish");
+  if (n_steps == 0) return TJ_OK;
+  const tj_config& c = x->cfg;
+  const bool on_policy = c.replay_capacity == 0;
+  ActorParams p{};
+  p.N = x->N; p.D = x->D; p.H = x->H; p.A = x->A; p.Aout = x->wl.Aout; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
+  p.S_d = x->S_d; p.rec_words = x->rec_words; p.max_ep = x->max_ep; p.policy_kind = c.policy_kind;
+  p.W = x->wbuf[x->active];
+  p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.state = x->state; p.ep_step = x->ep_step; p.ep_return = x->ep_return;
+  p.seed = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
+  p.explore_thr = explore_threshold(c.epsilon);
+  p.t0 = x->t; p.n_steps = n_steps;
+  p.ring = x->ring; p.C = c.replay_capacity; p.cursor0 = x->cursor; p.block_ver = x->block_ver;
+  p.version = (int)x->version;
+  p.T = c.rollout_len; p.G = c.n_segments;
+  p.seg_obs = x->seg_obs; p.seg_act = x->seg_act; p.seg_rew = x->seg_rew; p.seg_done = x->seg_done;
+  p.seg_logp = x->seg_logp; p.seg_val = x->seg_val;
+  p.lgAt = x->lgAt; p.lgB = x->lgB; p.lg_noise_std = c.lg_noise_std; p.lg_done_norm = c.lg_done_norm;
+  p.dbg_logits = dbg_logits; p.stats = x->dstats;
+  cudaError_t e = launch_actor(c.env_kind, p, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "actor step");
+  // host mirror of what the kernel does to versions, cursor and segment slots
+  for (int i = 0; i < n_steps; ++i) {
+    if (on_policy) {
+      const int64_t g = x->t / c.rollout_len;
+      const int pos = (int)(x->t % c.rollout_len);
+      SegSlot& sl = x->seg[(size_t)(g % c.n_segments)];
+      if (pos == 0) {
+        if (sl.state == 2) x->hs.dropped_overwritten += (int64_t)c.rollout_len * x->N;
+        sl.state = 1; sl.index = g; sl.version = x->version;
+      }
+      if (pos == c.rollout_len - 1) sl.state = 2;
+    } else {
+      x->h_block_ver[(size_t)((x->cursor % (uint64_t)c.replay_capacity) / (uint64_t)x->N)] = (int32_t)x->version;
+      x->cursor += (uint64_t)x->N;
+    }
+    x->t += 1;
+  }
+  x->hs.produced += (int64_t)n_steps * x->N;
+  x->hs.actor_steps += n_steps;
+  return TJ_OK;
+}
+
+int tj_replay_sample(tj_ctx* x, int32_t staleness_bound, int32_t* idx_out, const tj_batch* out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  const tj_config& c = x->cfg;
+  if (c.replay_capacity == 0) return fail(x, TJ_ERR_INVALID_ARG, "no replay ring in segment mode");
+  if (!out || !out->obs || !out->act || !out->rew || !out->next_obs || !out->done || !out->ver)
+    return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
+  if (out->n != c.minibatch) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must equal the configured minibatch");
+  if (x->version == 0) return fail(x, TJ_ERR_NO_WEIGHTS, "sample called before the first publish");
+  const int64_t S = staleness_bound >= 0 ? staleness_bound : c.staleness_bound;
+  const int64_t valid = (int64_t)std::min<uint64_t>(x->cursor, (uint64_t)c.replay_capacity);
+  if (valid < c.warmup) return fail(x, TJ_ERR_WARMUP, "fewer resident records than warmup");
+  const int n_blocks = (int)(valid / x->N);
+  int64_t n_elig = 0;
+  for (int b = 0; b < n_blocks; ++b)
+    if (x->version - (int64_t)x->h_block_ver[(size_t)b] <= S) ++n_elig;
+  if (n_elig == 0) {
+    x->hs.starved_calls += 1;
+    return fail(x, TJ_ERR_STARVED, "no resident record within the staleness bound");
+  }
+  if ((uint64_t)n_elig * (uint64_t)x->N > 0xFFFFFFFFull) return fail(x, TJ_ERR_UNSUPPORTED, "eligible set too large");
+  cudaError_t e = launch_eligible(x->block_ver, n_blocks, x->version, S, x->elig_list, x->elig_count, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "eligible list");
+  SampleParams p{};
+  p.B = c.minibatch; p.D = x->D; p.N = x->N; p.rec_words = x->rec_words;
+  p.seed = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
+  p.k = x->k; p.v_learner = x->version;
+  p.ring = x->ring; p.elig_list = x->elig_list; p.elig_count = x->elig_count;
+  p.idx_out = idx_out;
+  p.obs = out->obs; p.act = out->act; p.rew = out->rew; p.next_obs = out->next_obs; p.done = out->done; p.ver = out->ver;
+  p.stats = x->dstats;
+  if ((e = launch_sample_gather(p, x->stream)) != cudaSuccess) return cuda_fail(x, e, "sample and gather");
+  x->k += 1;
+  x->hs.learner_steps += 1;
+  x->hs.consumed += c.minibatch;
+  x->hs.dropped_stale += valid - n_elig * x->N;
+  return TJ_OK;
+}
+
+int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
+  if (b->n < 1 || b->n > kMaxTdRows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n out of range");
+  if (x->cfg.policy_kind != TJ_POLICY_EPS_GREEDY) return fail(x, TJ_ERR_UNSUPPORTED, "TD error needs the Q head");
+  if (x->version == 0 || !x->has_target) return fail(x, TJ_ERR_NO_WEIGHTS, "TD error called before the first publish");
+  TdParams p{};
+  p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
+  p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
+  p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
+  p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
+  p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = x->td_partial;
+  cudaError_t e = launch_td(p, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "TD error");
+  return TJ_OK;
+}
+
+int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, int32_t T, int32_t N, float gamma,
+           float lambda, float* adv_out, float* ret_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!rew || !val || !done || !adv_out || !ret_out) return fail(x, TJ_ERR_INVALID_ARG, "GAE arrays must not be null");
+  if (T < 0 || N < 0) return fail(x, TJ_ERR_INVALID_ARG, "T and N must not be negative");
+  if (T == 0 || N == 0) return TJ_OK;
+  cudaError_t e = launch_gae(rew, val, done, T, N, gamma, lambda, adv_out, ret_out, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "GAE");
+  return TJ_OK;
+}
+
+int tj_segment_acquire(tj_ctx* x, tj_segment* out) {
+  if (!x || !out) return TJ_ERR_INVALID_ARG;
+  const tj_config& c = x->cfg;
+  if (c.replay_capacity != 0) return fail(x, TJ_ERR_INVALID_ARG, "segments exist only in segment mode");
+  const int T = c.rollout_len, N = x->N, G = c.n_segments;
+  const int64_t begun = (x->t + T - 1) / T;
+  if (x->next_consume < begun - G) x->next_consume = begun - G;
+  for (; x->next_consume < begun; ++x->next_consume) {
+    SegSlot& sl = x->seg[(size_t)(x->next_consume % G)];
+    if (sl.index != x->next_consume) continue;  // overwritten by a later segment
+    if (sl.state == 1) break;                   // still being produced
+    if (sl.state != 2) continue;
+    if (x->version - sl.version > c.staleness_bound) {
+      sl.state = 3;
+      x->hs.dropped_stale += (int64_t)T * N;
+      continue;
+    }
+    const size_t slot = (size_t)(x->next_consume % G), TN = (size_t)T * N;
+    out->T = T; out->N = N; out->version = sl.version;
+    out->obs = x->seg_obs + slot * TN * x->D;
+    out->act = x->seg_act + slot * TN;
+    out->rew = x->seg_rew + slot * TN;
+    out->done = x->seg_done + slot * TN;
+    out->logp = x->seg_logp + slot * TN;
+    out->val = x->seg_val + slot * ((size_t)T + 1) * N;
+    sl.state = 3;
+    x->next_consume += 1;
+    x->k += 1;
+    x->hs.learner_steps += 1;
+    x->hs.consumed += (int64_t)T * N;
+    const int64_t stale = x->version - sl.version;
+    x->hs.max_sampled_staleness = std::max(x->hs.max_sampled_staleness, stale);
+    x->hs.staleness_hist[stale > 32 ? 32 : stale] += (int64_t)T * N;
+    return TJ_OK;
+  }
+  x->hs.starved_calls += 1;
+  return fail(x, TJ_ERR_STARVED, "no complete segment within the staleness bound");
+}
+
+int tj_get_state(tj_ctx* x, tj_state_view* out) {
+  if (!x || !out) return TJ_ERR_INVALID_ARG;
+  out->state = x->state; out->ep_step = x->ep_step;
+  out->cursor = x->cursor; out->t = x->t; out->k = x->k;
+  out->actor_version = out->learner_version = x->version;
+  return TJ_OK;
+}
+
+int tj_set_state(tj_ctx* x, const tj_state_view* in) {
+  if (!x || !in) return TJ_ERR_INVALID_ARG;
+  if (in->t < 0 || in->k < 0) return fail(x, TJ_ERR_INVALID_ARG, "counters must not be negative");
+  if (x->cfg.replay_capacity > 0 && in->cursor % (uint64_t)x->N) return fail(x, TJ_ERR_INVALID_ARG, "cursor must be a multiple of n_envs");
+  cudaError_t e;
+  if (in->state && in->state != x->state &&
+      (e = cudaMemcpyAsync(x->state, in->state, sizeof(float) * (size_t)x->N * x->S_d, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+    return cuda_fail(x, e, "set state");
+  if (in->ep_step && in->ep_step != x->ep_step &&
+      (e = cudaMemcpyAsync(x->ep_step, in->ep_step, sizeof(int) * (size_t)x->N, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+    return cuda_fail(x, e, "set episode steps");
+  x->cursor = in->cursor; x->t = in->t; x->k = in->k;
+  return TJ_OK;
+}
+
+int tj_stats(tj_ctx* x, tj_stats_t* o) {
+  if (!x || !o) return TJ_ERR_INVALID_ARG;
+  DevStats d;
+  cudaError_t e = cudaMemcpyAsync(&d, x->dstats, sizeof(d), cudaMemcpyDeviceToHost, x->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "read counters");
+  *o = x->hs;
+  o->actor_version = o->learner_version = x->version;
+  o->episodes_finished = (int64_t)d.episodes;
+  o->return_sum = d.return_sum;
+  o->device_error = (int64_t)d.error;
+  if (x->cfg.replay_capacity > 0) {
+    o->max_sampled_staleness = (int64_t)d.max_stale;
+    for (int i = 0; i < 33; ++i) o->staleness_hist[i] = (int64_t)d.hist[i];
+  }
+  return TJ_OK;
+}
+
+int tj_ring_view(tj_ctx* x, const float** records, const int32_t** block_version, int32_t* record_words) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (records) *records = x->ring;
+  if (block_version) *block_version = x->block_ver;
+  if (record_words) *record_words = x->rec_words;
+  return TJ_OK;
+}
+
+const char* tj_last_error(const tj_ctx* x) { return x ? x->err.c_str() : g_err.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,173 @@
+// Host-side context and the launch interface between the C ABI shell and the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/tj.h"
+
+namespace tj {
+
+// Policy parameters as the kernels read them: every matrix transposed to [in][out_padded] so that a thread
+// fetches four consecutive output neurons with one 128-bit load; the value head (if any) is column A of the
+// last matrix.  All sizes in floats.
+struct WeightLayout {
+  int D, H, A, Aout, Hp, Ap;
+  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3, total;
+};
+
+inline int round_up4(int x) { return (x + 3) & ~3; }
+
+inline WeightLayout make_weight_layout(int D, int H, int A, int value_head) {
+  WeightLayout L;
+  L.D = D; L.H = H; L.A = A; L.Aout = A + (value_head ? 1 : 0);
+  L.Hp = round_up4(H);
+  L.Ap = round_up4(L.Aout);
+  size_t o = 0;
+  auto take = [&](size_t n) { size_t r = o; o += (n + 63) & ~(size_t)63; return r; };  // 256-byte aligned parts
+  L.off_W1t = take((size_t)D * L.Hp);
+  L.off_b1 = take(L.Hp);
+  L.off_W2t = take((size_t)H * L.Hp);
+  L.off_b2 = take(L.Hp);
+  L.off_W3t = take((size_t)H * L.Ap);
+  L.off_b3 = take(L.Ap);
+  L.total = o;
+  return L;
+}
+
+struct DevStats {
+  unsigned long long episodes;
+  double return_sum;
+  unsigned long long hist[33];
+  unsigned long long max_stale;
+  unsigned long long error;
+};
+
+struct ActorParams {
+  int N, D, H, A, Aout, Hp, Ap, S_d, rec_words, max_ep, policy_kind;
+  const float* W;  // packed weights, WeightLayout offsets below
+  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3;
+  float* state;
+  int* ep_step;
+  float* ep_return;
+  uint2 seed;
+  unsigned long long explore_thr;
+  long long t0;
+  int n_steps;
+  float* ring;
+  long long C;
+  unsigned long long cursor0;
+  int* block_ver;
+  int version;
+  int T, G;
+  float* seg_obs;
+  int* seg_act;
+  float* seg_rew;
+  uint8_t* seg_done;
+  float* seg_logp;
+  float* seg_val;
+  const float* lgAt;  // [D][Dp], transposed
+  const float* lgB;   // [A][Dp]
+  float lg_noise_std, lg_done_norm;
+  float* dbg_logits;
+  DevStats* stats;
+};
+
+struct TdParams {
+  int n, D, H, A, Hp, Ap;
+  const float* Wonline;
+  const float* Wtarget;
+  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3;
+  const float* obs;
+  const int* act;
+  const float* rew;
+  const float* next_obs;
+  const int* done;
+  float gamma, kappa;
+  float* td_out;
+  float* huber_out;
+  float* loss_out;
+  float* partial;  // scratch: one float per thread block
+};
+
+struct SampleParams {
+  int B, D, N, rec_words;
+  uint2 seed;
+  long long k;
+  long long v_learner;
+  const float* ring;
+  const int* elig_list;
+  const int* elig_count;
+  int* idx_out;
+  float* obs;
+  int* act;
+  float* rew;
+  float* next_obs;
+  int* done;
+  int* ver;
+  DevStats* stats;
+};
+
+// launchers (each returns the cudaGetLastError() of its launches)
+cudaError_t launch_init_env(int env_kind, int N, int S_d, uint2 seed, float* state, int* ep_step, float* ep_return,
+                            cudaStream_t s);
+cudaError_t launch_pack_weights(const float* blob, float* dst, const WeightLayout& L, int value_head, int bf16,
+                                cudaStream_t s);
+cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s);
+size_t actor_td_scratch_floats(int n);
+cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_learner, long long bound, int* elig_list,
+                            int* elig_count, cudaStream_t s);
+cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
+cudaError_t launch_td(const TdParams& p, cudaStream_t s);
+int td_grid(int n);
+cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
+                       float* adv, float* ret, cudaStream_t s);
+cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);
+
+}  // namespace tj
+
+struct SegSlot {
+  int64_t index = -1;   // which segment number sits in the slot
+  int64_t version = 0;
+  int state = 0;        // 0 empty, 1 filling, 2 complete, 3 consumed or dropped
+};
+
+struct tj_ctx {
+  tj_config cfg;
+  cudaStream_t stream;
+  int N, D, H, A, S_d, value_head, rec_words, max_ep;
+  size_t n_blob;
+  tj::WeightLayout wl;
+  // device memory (all inside the caller's workspace)
+  float* state;
+  int* ep_step;
+  float* ep_return;
+  float* wbuf[2];       // online parameters, double buffered
+  float* wtarget;
+  float* blob_stage;    // staging for host blobs
+  float* ring;
+  int* block_ver;
+  int* elig_list;
+  int* elig_count;
+  float* td_partial;
+  tj::DevStats* dstats;
+  float* lgAt;
+  float* lgB;
+  float* lg_stage;
+  float *seg_obs, *seg_rew, *seg_logp, *seg_val;
+  int* seg_act;
+  uint8_t* seg_done;
+  // host bookkeeping
+  int active;           // which wbuf is the newest published
+  int64_t version, k_last_sync;
+  bool has_target;
+  int64_t t, k;
+  uint64_t cursor;
+  std::vector<int32_t> h_block_ver;
+  std::vector<SegSlot> seg;
+  int64_t next_consume;
+  tj_stats_t hs;        // host-side counters
+  std::string err;
+};

@@ -1,0 +1,274 @@
+// Learner-side kernels: parameter publish (repack), eligible-block list, staleness-bounded sampling with
+// gather, TD error / Huber loss, and the GAE reverse scan.
+#include "tj_device.cuh"
+#include "tj_internal.h"
+#include "tj_mlp.cuh"
+
+namespace tj {
+
+namespace {
+
+__device__ __forceinline__ float bf16_round_rne(float x) {
+  uint32_t u = __float_as_uint(x);
+  if ((u & 0x7F800000u) == 0x7F800000u) return x;
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return __uint_as_float(u & 0xFFFF0000u);
+}
+
+// blob [W1 HxD, b1 H, W2 HxH, b2 H, W3 AxH, b3 A (, Wv H, bv 1)] -> transposed, padded kernel layout
+__global__ void pack_weights_kernel(const float* __restrict__ blob, float* __restrict__ dst, WeightLayout L,
+                                    int value_head, int bf16) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= L.total) return;
+  const int D = L.D, H = L.H, A = L.A;
+  const float* W1 = blob;
+  const float* b1 = W1 + (size_t)H * D;
+  const float* W2 = b1 + H;
+  const float* b2 = W2 + (size_t)H * H;
+  const float* W3 = b2 + H;
+  const float* b3 = W3 + (size_t)A * H;
+  const float* Wv = b3 + A;
+  const float* bv = Wv + H;
+  float v = 0.f;
+  bool is_weight = false;
+  if (i >= L.off_W1t && i < L.off_W1t + (size_t)D * L.Hp) {
+    const size_t j = i - L.off_W1t;
+    const int k = (int)(j / L.Hp), n = (int)(j % L.Hp);
+    if (n < H) { v = W1[(size_t)n * D + k]; is_weight = true; }
+  } else if (i >= L.off_b1 && i < L.off_b1 + L.Hp) {
+    const int n = (int)(i - L.off_b1);
+    if (n < H) v = b1[n];
+  } else if (i >= L.off_W2t && i < L.off_W2t + (size_t)H * L.Hp) {
+    const size_t j = i - L.off_W2t;
+    const int k = (int)(j / L.Hp), n = (int)(j % L.Hp);
+    if (n < H) { v = W2[(size_t)n * H + k]; is_weight = true; }
+  } else if (i >= L.off_b2 && i < L.off_b2 + L.Hp) {
+    const int n = (int)(i - L.off_b2);
+    if (n < H) v = b2[n];
+  } else if (i >= L.off_W3t && i < L.off_W3t + (size_t)H * L.Ap) {
+    const size_t j = i - L.off_W3t;
+    const int k = (int)(j / L.Ap), n = (int)(j % L.Ap);
+    if (n < A) { v = W3[(size_t)n * H + k]; is_weight = true; }
+    else if (value_head && n == A) { v = Wv[k]; is_weight = true; }
+  } else if (i >= L.off_b3 && i < L.off_b3 + L.Ap) {
+    const int n = (int)(i - L.off_b3);
+    if (n < A) v = b3[n];
+    else if (value_head && n == A) v = bv[0];
+  }
+  if (bf16 && is_weight) v = bf16_round_rne(v);
+  dst[i] = v;
+}
+
+__global__ void transpose_pad_kernel(const float* __restrict__ src, float* __restrict__ dst, int rows, int cols,
+                                     int ld_dst) {
+  // dst[c][r] = src[r][c], dst rows padded to ld_dst with zeros
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)cols * ld_dst) return;
+  const int c = (int)(i / ld_dst), r = (int)(i % ld_dst);
+  dst[i] = r < rows ? src[(size_t)r * cols + c] : 0.f;
+}
+
+// Ascending list of ring blocks (one block = the N records of one actor step, all with one version) whose
+// version is at most `bound` behind the learner.  One thread block, stable compaction by chunks.
+__global__ void eligible_kernel(const int* __restrict__ block_ver, int n_blocks, long long v_learner, long long bound,
+                                int* __restrict__ elig_list, int* __restrict__ elig_count) {
+  __shared__ int warp_tot[32];
+  __shared__ int base;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) base = 0;
+  __syncthreads();
+  for (int c0 = 0; c0 < n_blocks; c0 += blockDim.x) {
+    const int b = c0 + tid;
+    const int flag = (b < n_blocks && v_learner - (long long)block_ver[b] <= bound) ? 1 : 0;
+    const unsigned m = __ballot_sync(0xffffffffu, flag);
+    const int before = __popc(m & ((1u << lane) - 1u));
+    if (lane == 0) warp_tot[warp] = __popc(m);
+    __syncthreads();
+    int woff = 0, tot = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+      if (w < warp) woff += warp_tot[w];
+      tot += warp_tot[w];
+    }
+    if (flag) elig_list[base + woff + before] = b;
+    __syncthreads();
+    if (tid == 0) base += tot;
+    __syncthreads();
+  }
+  if (tid == 0) *elig_count = base;
+}
+
+// One warp per draw: slot = E[mulhi(x0, |E|)] with E enumerated block by block, then the record is copied
+// word for word into the dense minibatch arrays.
+__global__ void sample_gather_kernel(const SampleParams p) {
+  const int warp = (int)(((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+  if (warp >= p.B) return;
+  const int j = warp;
+  const unsigned long long nE = (unsigned long long)(*p.elig_count) * (unsigned long long)p.N;
+  const uint4 w = stream_words(p.seed, STREAM_SAMPLE, 0, (uint32_t)j, (unsigned long long)p.k);
+  const uint32_t r = __umulhi(w.x, (uint32_t)nE);
+  const int slot = p.elig_list[r / (uint32_t)p.N] * p.N + (int)(r % (uint32_t)p.N);
+  const float* rec = p.ring + (size_t)slot * p.rec_words;
+  const int D = p.D;
+  for (int i = lane; i < p.rec_words; i += 32) {
+    const float v = rec[i];
+    if (i < D) p.obs[(size_t)j * D + i] = v;
+    else if (i < 2 * D) p.next_obs[(size_t)j * D + (i - D)] = v;
+    else if (i == 2 * D) p.act[j] = __float_as_int(v);
+    else if (i == 2 * D + 1) p.rew[j] = v;
+    else if (i == 2 * D + 2) p.done[j] = __float_as_int(v);
+    else {
+      const int ver = __float_as_int(v);
+      p.ver[j] = ver;
+      long long stale = p.v_learner - (long long)ver;
+      if (stale < 0) stale = 0;
+      atomicAdd(&p.stats->hist[stale > 32 ? 32 : stale], 1ull);
+      atomicMax(&p.stats->max_stale, (unsigned long long)stale);
+    }
+  }
+  if (lane == 0 && p.idx_out) p.idx_out[j] = slot;
+}
+
+// TD error on a tile of TE samples: online forward on obs, target forward on next_obs.
+template <int TE>
+__global__ void __launch_bounds__(kThreads) td_kernel(const TdParams p) {
+  extern __shared__ __align__(16) float smem[];
+  const int Dx = (p.D + 3) & ~3;
+  float* xs = smem;
+  float* h1 = xs + (size_t)Dx * TE;
+  float* h2 = h1 + (size_t)p.Hp * TE;
+  float* out = h2 + (size_t)p.Hp * TE;
+  float* qsel = out + (size_t)p.Ap * TE;
+  float* hub = qsel + TE;
+  const int tid = threadIdx.x, j0 = blockIdx.x * TE, n_here = min(TE, p.n - j0), D = p.D;
+
+  for (int i = tid; i < TE * D; i += kThreads) {
+    const int el = i / D, k = i % D;
+    xs[k * TE + el] = el < n_here ? p.obs[(size_t)(j0 + el) * D + k] : 0.f;
+  }
+  __syncthreads();
+  mlp_forward_tile<TE>(p.Wonline, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, D, p.H, p.Hp, p.A,
+                       p.Ap, xs, h1, h2, out);
+  if (tid < n_here) {
+    int a = p.act[j0 + tid];
+    a = a < 0 ? 0 : (a >= p.A ? p.A - 1 : a);
+    qsel[tid] = out[a * TE + tid];
+  }
+  __syncthreads();
+  for (int i = tid; i < TE * D; i += kThreads) {
+    const int el = i / D, k = i % D;
+    xs[k * TE + el] = el < n_here ? p.next_obs[(size_t)(j0 + el) * D + k] : 0.f;
+  }
+  __syncthreads();
+  mlp_forward_tile<TE>(p.Wtarget, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, D, p.H, p.Hp, p.A,
+                       p.Ap, xs, h1, h2, out);
+  if (tid < TE) {
+    float h = 0.f;
+    if (tid < n_here) {
+      const int j = j0 + tid;
+      float qmax = out[tid];
+      for (int i = 1; i < p.A; ++i) qmax = fmaxf(qmax, out[i * TE + tid]);
+      const float y = p.rew[j] + p.gamma * (p.done[j] ? 0.f : 1.f) * qmax;
+      const float delta = y - qsel[tid];
+      const float ad = fabsf(delta);
+      h = ad <= p.kappa ? 0.5f * delta * delta : p.kappa * (ad - 0.5f * p.kappa);
+      if (p.td_out) p.td_out[j] = delta;
+      if (p.huber_out) p.huber_out[j] = h;
+    }
+    hub[tid] = h;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float sum = 0.f;
+    for (int i = 0; i < n_here; ++i) sum += hub[i];
+    p.partial[blockIdx.x] = sum;
+  }
+}
+
+// fixed-order sum of the per-block partial losses
+__global__ void td_finish_kernel(const float* __restrict__ partial, int n_partial, int n, float* __restrict__ loss_out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    float sum = 0.f;
+    for (int i = 0; i < n_partial; ++i) sum += partial[i];
+    *loss_out = sum / (float)n;
+  }
+}
+
+// GAE: one thread per environment walks its column backwards; a warp reads 32 consecutive environments.
+__global__ void gae_kernel(const float* __restrict__ rew, const float* __restrict__ val,
+                           const uint8_t* __restrict__ done, int T, int N, float gamma, float lambda,
+                           float* __restrict__ adv, float* __restrict__ ret) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= N) return;
+  float next_adv = 0.f;
+  float v_next = val[(size_t)T * N + e];
+  const float gl = gamma * lambda;
+  for (int t = T - 1; t >= 0; --t) {
+    const size_t i = (size_t)t * N + e;
+    const float nd = done[i] ? 0.f : 1.f;
+    const float v = val[i];
+    const float delta = rew[i] + gamma * nd * v_next - v;
+    const float a = delta + gl * nd * next_adv;
+    adv[i] = a;
+    ret[i] = a + v;
+    next_adv = a;
+    v_next = v;
+  }
+}
+
+constexpr int kTdTile = 32;
+
+}  // namespace
+
+cudaError_t launch_pack_weights(const float* blob, float* dst, const WeightLayout& L, int value_head, int bf16,
+                                cudaStream_t s) {
+  pack_weights_kernel<<<(unsigned)((L.total + 255) / 256), 256, 0, s>>>(blob, dst, L, value_head, bf16);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s) {
+  const size_t n = (size_t)cols * ld_dst;
+  transpose_pad_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(src, dst, rows, cols, ld_dst);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_learner, long long bound, int* elig_list,
+                            int* elig_count, cudaStream_t s) {
+  eligible_kernel<<<1, 1024, 0, s>>>(block_ver, n_blocks, v_learner, bound, elig_list, elig_count);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s) {
+  const int warps_per_block = 8;
+  sample_gather_kernel<<<(p.B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+int td_grid(int n) { return (n + kTdTile - 1) / kTdTile; }
+
+cudaError_t launch_td(const TdParams& p, cudaStream_t s) {
+  constexpr int TE = kTdTile;
+  const int Dx = (p.D + 3) & ~3;
+  const size_t smem = ((size_t)Dx * TE + 2 * (size_t)p.Hp * TE + (size_t)p.Ap * TE + 2 * TE) * sizeof(float);
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  if (smem > 48 * 1024) {
+    cudaError_t err = cudaFuncSetAttribute(td_kernel<TE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+  }
+  const int grid = td_grid(p.n);
+  td_kernel<TE><<<grid, kThreads, smem, s>>>(p);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  if (p.loss_out) {
+    td_finish_kernel<<<1, 32, 0, s>>>(p.partial, grid, p.n, p.loss_out);
+    err = cudaGetLastError();
+  }
+  return err;
+}
+
+cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
+                       float* adv, float* ret, cudaStream_t s) {
+  gae_kernel<<<(N + 127) / 128, 128, 0, s>>>(rew, val, done, T, N, gamma, lambda, adv, ret);
+  return cudaGetLastError();
+}
+
+}  // namespace tj
