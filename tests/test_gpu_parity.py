@@ -115,8 +115,10 @@ def test_small_env_lockstep_ragged_shapes(env, kind, D, A, H, N, steps):
             ctx.publish_weights(blob)
             o.publish(blob)
         r = lockstep_step(ctx, o, torch, rtol=RTOL_FP32, env_kind=kind, tally=tally)
-        compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=kind, tally=tally)
-    assert tally.ambiguous_done <= 0.002 * tally.total + 2
+        scale = float(np.sqrt(np.mean(r["o_logits"].astype(np.float64) ** 2)))
+        compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=kind, tally=tally, act_exact=(kind != 1),
+                          act_margin_scale=8 * RTOL_FP32 * scale)
+    assert tally.ambiguous_done <= 0.002 * tally.total + 2 and tally.ambiguous_act <= 0.002 * tally.total + 2
     assert ctx.stats()["episodes_finished"] > 0
 
 
@@ -339,7 +341,8 @@ def test_segment_mode_lockstep(env):
                 close(gseg["logp"].cpu().numpy()[same], oseg["logp"][same], RTOL_FP32, "logp")
                 assert np.array_equal(gseg["done"].cpu().numpy()[same], oseg["done"][same])
                 assert np.array_equal(gseg["rew"].cpu().numpy(), oseg["rew"])
-                assert np.array_equal(gseg["val"].cpu().numpy()[-1], oseg["val"][-1])
+                # the bootstrap row is evaluated on the stepped state, which the two sides hold to FP32 rounding
+                close(gseg["val"].cpu().numpy()[-1], oseg["val"][-1], 4 * RTOL_FP32, "bootstrap value")
                 adv, ret = ctx.gae(gseg["rew"], gseg["val"], gseg["done"], 0.99, 0.95)
                 o_adv, o_ret = orc.gae(oseg["rew"], oseg["val"], oseg["done"], 0.99, 0.95)
                 close(adv.cpu().numpy(), o_adv, RTOL_FP32, "segment adv")
