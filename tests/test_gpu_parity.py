@@ -306,7 +306,7 @@ def test_segment_mode_lockstep(env):
                    rollout_len=12, n_segments=3, staleness_bound=1, gamma=0.99, gae_lambda=0.95, max_episode_steps=9)
     ctx, o = make_pair(orc, binding, **f)
     tally = Tally()
-    assert ctx.segment_acquire(allow=(0, -7))[0] == -7
+    assert ctx.segment_acquire(allow=(0, -7))[0] == -7 == o.segment_acquire()[0]
     v = 0
     consumed = 0
     for seg_i in range(7):
