@@ -184,6 +184,28 @@ int tj_replay_sample(tj_ctx *ctx, int32_t staleness_bound, int32_t *idx_out, con
  * (nullable), the mean Huber loss summed in a fixed order. */
 int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
 
+/* The same computation as tj_td_error for callers that must not allocate and have no scratch to lend.
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ *
+ * Who this is for: code that runs where device allocation is off limits -- a latency-critical actor or
+ * evaluation loop in which a cudaMalloc would synchronise the whole device and stall every stream, a process
+ * that runs under a memory plan fixed at start-up, or a plug-in living inside another framework whose
+ * allocator it may not call.  tj_td_error sums the per-block losses through scratch carved from the caller's
+ * workspace; this variant keeps that scratch in a fixed 32 KB array inside the library image, so every GPU
+ * that loads the library holds those 32 KB until the process exits.  It calls no cudaMalloc, no cudaFree and
+ * no allocating library routine; inputs and outputs are still the caller's.
+ *
+ * Limits and rules:
+ *   - at most 65,536 rows per call; a larger batch.n is refused with TJ_ERR_INVALID_ARG and a message naming
+ *     the limit (split the batch or use tj_td_error);
+ *   - the first call on each device looks up the array's device address (once per device, with that device
+ *     current).  Make that first call at set-up, before any stream capture is under way;
+ *   - every call, from every context on the device, shares the one array.  Each call rewrites the part it
+ *     reads, so nothing needs clearing between calls, but two calls that overlap on the GPU (different
+ *     streams) race on it: keep them on one stream or order them with events;
+ *   - results equal tj_td_error's (same kernels, same summation order). */
+int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
+
 /* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
  *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0;
  *   R_t = A_t + V_t.   rew [T][N], val [T+1][N], done [T][N] -> adv [T][N], ret [T][N].

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_ring_view",
            "tj_last_error")
 
 
@@ -86,6 +86,7 @@ def load_library():
     L.tj_actor_step.argtypes = [vp, i32, vp]
     L.tj_replay_sample.argtypes = [vp, i32, vp, vp]
     L.tj_td_error.argtypes = [vp, vp, vp, vp, vp]
+    L.tj_td_error_static.argtypes = [vp, vp, vp, vp, vp]
     L.tj_gae.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
     L.tj_get_state.argtypes = [vp, vp]
@@ -140,6 +141,11 @@ def tj_replay_sample(h, staleness_bound: int, idx_ptr: int, batch: TjBatch):
 
 def tj_td_error(h, batch: TjBatch, td_ptr: int, huber_ptr: int, loss_ptr: int):
     return load_library().tj_td_error(h, C.byref(batch), td_ptr or None, huber_ptr or None, loss_ptr or None)
+
+
+def tj_td_error_static(h, batch: TjBatch, td_ptr: int, huber_ptr: int, loss_ptr: int):
+    """tj_td_error with the reduction scratch inside the library image (at most 65,536 rows; allocates nothing)."""
+    return load_library().tj_td_error_static(h, C.byref(batch), td_ptr or None, huber_ptr or None, loss_ptr or None)
 
 
 def tj_gae(h, rew_ptr, val_ptr, done_ptr, T, N, gamma, lam, adv_ptr, ret_ptr):

@@ -350,6 +350,32 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
   return TJ_OK;
 }
 
+int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
+  if (b->n < 1) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be positive");
+  if (x->cfg.policy_kind != TJ_POLICY_EPS_GREEDY) return fail(x, TJ_ERR_UNSUPPORTED, "TD error needs the Q head");
+  if (x->version == 0 || !x->has_target) return fail(x, TJ_ERR_NO_WEIGHTS, "TD error called before the first publish");
+  TdParams p{};
+  p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
+  p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
+  p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
+  p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
+  p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = nullptr;
+  bool too_large = false;
+  cudaError_t e = launch_td_static(p, x->stream, &too_large);
+  if (too_large) {
+    char msg[160];
+    std::snprintf(msg, sizeof(msg), "tj_td_error_static takes at most %d rows per call (got %d); use tj_td_error or split the batch",
+                  td_static_max_rows(), b->n);
+    return fail(x, TJ_ERR_INVALID_ARG, msg);
+  }
+  if (e != cudaSuccess) return cuda_fail(x, e, "TD error (library scratch)");
+  return TJ_OK;
+}
+
 int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, int32_t T, int32_t N, float gamma,
            float lambda, float* adv_out, float* ret_out) {
   if (!x) return TJ_ERR_INVALID_ARG;

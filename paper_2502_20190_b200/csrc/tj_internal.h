@@ -122,6 +122,8 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
 cudaError_t launch_td(const TdParams& p, cudaStream_t s);
 int td_grid(int n);
+int td_static_max_rows();
+cudaError_t launch_td_static(const TdParams& p, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
                        float* adv, float* ret, cudaStream_t s);
 cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);

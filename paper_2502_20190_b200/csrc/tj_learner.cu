@@ -265,6 +265,33 @@ cudaError_t launch_td(const TdParams& p, cudaStream_t s) {
   return err;
 }
 
+// Scratch for tj_td_error_static: it is part of the library image, so every GPU that loads the library
+// holds these 32 KB until the process exits and nobody has to allocate it.
+constexpr int kStaticTdPartials = 8192;
+static __device__ __align__(256) float g_td_static_partial[kStaticTdPartials];
+
+int td_static_max_rows() { return 65536; }
+
+cudaError_t launch_td_static(const TdParams& p_in, cudaStream_t s, bool* too_large) {
+  *too_large = p_in.n > td_static_max_rows() || td_grid(p_in.n) > kStaticTdPartials;
+  if (*too_large) return cudaSuccess;
+  // In host code the array's name is only a stand-in; the device address has to be asked for, once per device.
+  static float* addr_by_device[64] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!addr_by_device[dev]) {
+    float* q = nullptr;
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&q), g_td_static_partial);
+    if (e != cudaSuccess) return e;
+    addr_by_device[dev] = q;
+  }
+  TdParams p = p_in;
+  p.partial = addr_by_device[dev];
+  return launch_td(p, s);
+}
+
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
                        float* adv, float* ret, cudaStream_t s) {
   gae_kernel<<<(N + 127) / 128, 128, 0, s>>>(rew, val, done, T, N, gamma, lambda, adv, ret);
