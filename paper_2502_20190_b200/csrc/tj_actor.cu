@@ -4,6 +4,7 @@
 // Environments are independent, so a thread block keeps its TE environments for the whole call: state lives
 // in registers (CartPole, Acrobot) or shared memory (linear-Gaussian) between steps, and no block ever waits
 // on another.  The ring cursor advances by N per step, which every block can compute on its own.
+#include "tj_async.cuh"
 #include "tj_device.cuh"
 #include "tj_internal.h"
 #include "tj_mlp.cuh"
@@ -13,23 +14,30 @@ namespace tj {
 namespace {
 
 struct ActorSmem {
-  float *xs, *h1, *h2, *out, *nxt, *rew;
+  float *w, *xs, *h1, *h2, *out, *nxt, *rew;
   int *act, *done;
 };
 
-template <int TE>
-__host__ __device__ inline size_t actor_smem_floats(int D, int Hp, int Ap, bool lingauss) {
+// STAGE: 0 = parameters read from global memory, 1 = everything but the HxH matrix staged in shared memory,
+//        2 = all parameters staged.
+__host__ __device__ inline size_t staged_floats(int stage, size_t w_total, size_t off_W2t, size_t off_b2) {
+  if (stage == 2) return w_total;
+  if (stage == 1) return w_total - (off_b2 - off_W2t);
+  return 0;
+}
+
+__host__ __device__ inline size_t actor_smem_floats(int TE, int D, int Hp, int Ap, bool lingauss, size_t staged) {
   const int Dx = (D + 3) & ~3;
-  size_t n = (size_t)Dx * TE + 2 * (size_t)Hp * TE + (size_t)Ap * TE;
+  size_t n = staged + (size_t)Dx * TE + 2 * (size_t)Hp * TE + (size_t)Ap * TE;
   if (lingauss) n += (size_t)Dx * TE;
   n += 3 * TE;  // rew, act, done
   return n;
 }
 
-template <int TE>
-__device__ inline ActorSmem carve(float* base, int D, int Hp, int Ap, bool lingauss) {
+__device__ inline ActorSmem carve(float* base, int TE, int D, int Hp, int Ap, bool lingauss, size_t staged) {
   const int Dx = (D + 3) & ~3;
   ActorSmem s;
+  s.w = base; base += staged;
   s.xs = base; base += (size_t)Dx * TE;
   s.h1 = base; base += (size_t)Hp * TE;
   s.h2 = base; base += (size_t)Hp * TE;
@@ -42,6 +50,33 @@ __device__ inline ActorSmem carve(float* base, int D, int Hp, int Ap, bool linga
   return s;
 }
 
+// Queue the bulk copies of the staged parameter ranges (one thread) and name where each part is read from.
+template <int STAGE>
+__device__ __forceinline__ MlpWeights stage_weights(const ActorParams& p, float* wsm, uint64_t* bar, bool issue) {
+  MlpWeights w;
+  if (STAGE == 0) {
+    w.W1t = p.W + p.off_W1t; w.b1 = p.W + p.off_b1; w.W2t = p.W + p.off_W2t; w.b2 = p.W + p.off_b2;
+    w.W3t = p.W + p.off_W3t; w.b3 = p.W + p.off_b3;
+    return w;
+  }
+  const size_t gap = STAGE == 1 ? p.off_b2 - p.off_W2t : 0;
+  if (issue) {
+    if (STAGE == 2) {
+      mbar_expect_tx(bar, (uint32_t)(p.w_total * sizeof(float)));
+      bulk_copy_chunks(wsm, p.W, p.w_total * sizeof(float), bar);
+    } else {
+      const size_t head = p.off_W2t, tail = p.w_total - p.off_b2;
+      mbar_expect_tx(bar, (uint32_t)((head + tail) * sizeof(float)));
+      bulk_copy_chunks(wsm, p.W, head * sizeof(float), bar);
+      bulk_copy_chunks(wsm + head, p.W + p.off_b2, tail * sizeof(float), bar);
+    }
+  }
+  w.W1t = wsm + p.off_W1t; w.b1 = wsm + p.off_b1;
+  w.W2t = STAGE == 2 ? wsm + p.off_W2t : p.W + p.off_W2t;
+  w.b2 = wsm + p.off_b2 - gap; w.W3t = wsm + p.off_W3t - gap; w.b3 = wsm + p.off_b3 - gap;
+  return w;
+}
+
 __device__ __forceinline__ float4 reset4(uint2 seed, uint32_t block, uint32_t e, unsigned long long step, float lo,
                                          float width) {
   const uint4 w = stream_words(seed, STREAM_RESET, block, e, step);
@@ -52,14 +87,20 @@ __device__ __forceinline__ float4 reset4(uint2 seed, uint32_t block, uint32_t e,
 // ------------------------------------------------------------------------------------------------
 // CartPole / Acrobot: one thread owns one environment (state in registers).
 // ------------------------------------------------------------------------------------------------
-template <int TE, int ENV>
-__global__ void __launch_bounds__(kThreads) actor_small_env_kernel(const ActorParams p) {
-  extern __shared__ __align__(16) float smem[];
-  const ActorSmem sm = carve<TE>(smem, p.D, p.Hp, p.Ap, false);
+template <int TE, int NT, int ENV, int STAGE>
+__global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p) {
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) uint64_t wbar;
+  const ActorSmem sm = carve(smem, TE, p.D, p.Hp, p.Ap, false, staged_floats(STAGE, p.w_total, p.off_W2t, p.off_b2));
   const int tid = threadIdx.x;
   const int e = blockIdx.x * TE + tid;
   const bool owner = tid < TE && e < p.N;
   const bool on_policy = p.C == 0;
+  if (STAGE > 0) {
+    if (tid == 0) mbar_init(&wbar, 1);
+    __syncthreads();
+  }
+  const MlpWeights mw = stage_weights<STAGE>(p, sm.w, &wbar, tid == 0);
 
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   int ep = 0;
@@ -71,6 +112,10 @@ __global__ void __launch_bounds__(kThreads) actor_small_env_kernel(const ActorPa
   }
   unsigned long long n_episodes = 0;
   double ret_sum = 0.0;
+  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) {  // parameters never arrived: flag it and leave
+    if (tid == 0) atomicExch(&p.stats->error, 1ull);
+    return;
+  }
 
   for (int step = 0; step < p.n_steps; ++step) {
     const unsigned long long t = (unsigned long long)p.t0 + step;
@@ -90,8 +135,7 @@ __global__ void __launch_bounds__(kThreads) actor_small_env_kernel(const ActorPa
         if (k < p.D) sm.xs[k * TE + tid] = owner ? obs[k] : 0.f;
     }
     __syncthreads();
-    mlp_forward_tile<TE>(p.W, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, p.D, p.H, p.Hp, p.Aout,
-                         p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+    mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (owner) {
       auto logit = [&](int i) { return sm.out[i * TE + tid]; };
       if (p.dbg_logits) {
@@ -171,8 +215,7 @@ __global__ void __launch_bounds__(kThreads) actor_small_env_kernel(const ActorPa
           if (k < p.D) sm.xs[k * TE + tid] = owner ? o2[k] : 0.f;
       }
       __syncthreads();
-      mlp_forward_tile<TE>(p.W, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, p.D, p.H, p.Hp,
-                           p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+      mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
       if (owner) {
         const int slot = (int)((long long)(t / (unsigned long long)p.T) % p.G);
         p.seg_val[((size_t)slot * (p.T + 1) + p.T) * p.N + e] = sm.out[p.A * TE + tid];
@@ -194,17 +237,19 @@ __global__ void __launch_bounds__(kThreads) actor_small_env_kernel(const ActorPa
 // ------------------------------------------------------------------------------------------------
 // Linear-Gaussian env: the state (= observation) of the tile lives in shared memory, k-major.
 // ------------------------------------------------------------------------------------------------
-template <int TE>
-__global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorParams p) {
-  extern __shared__ __align__(16) float smem[];
-  const ActorSmem sm = carve<TE>(smem, p.D, p.Hp, p.Ap, true);
+template <int TE, int NT>
+__global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p) {
+  extern __shared__ __align__(128) float smem[];
+  const ActorSmem sm = carve(smem, TE, p.D, p.Hp, p.Ap, true, 0);
+  __shared__ uint64_t unused_bar;
+  const MlpWeights mw = stage_weights<0>(p, nullptr, &unused_bar, false);
   const int tid = threadIdx.x;
   const int e0 = blockIdx.x * TE;
   const int D = p.D, Dp = (p.D + 3) & ~3;
   const int n_here = min(TE, p.N - e0);
 
   // state -> xs[k][e]
-  for (int i = tid; i < TE * D; i += kThreads) {
+  for (int i = tid; i < TE * D; i += NT) {
     const int el = i / D, k = i % D;
     sm.xs[k * TE + el] = el < n_here ? p.state[(size_t)(e0 + el) * D + k] : 0.f;
   }
@@ -220,8 +265,7 @@ __global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorPar
 
   for (int step = 0; step < p.n_steps; ++step) {
     const unsigned long long t = (unsigned long long)p.t0 + step;
-    mlp_forward_tile<TE>(p.W, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, D, p.H, p.Hp, p.Aout, p.Ap,
-                         sm.xs, sm.h1, sm.h2, sm.out);
+    mlp_forward_tile<TE, NT, false, false>(mw, D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (tid < TE) {
       int a = 0;
       if (tid < n_here) {
@@ -238,10 +282,10 @@ __global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorPar
     }
     __syncthreads();
     // s' = tanh(A s + B[a]) ...
-    dense_layer<TE, ACT_TANH, true>(p.lgAt, p.lgB, Dp, D, D, sm.xs, sm.nxt, sm.act);
+    dense_layer<TE, NT, ACT_TANH, true, false>(p.lgAt, p.lgB, Dp, D, D, sm.xs, sm.nxt, sm.act);
     __syncthreads();
     // ... + noise_std * n, four normals per Philox call
-    for (int i = tid; i < TE * (D / 4); i += kThreads) {
+    for (int i = tid; i < TE * (D / 4); i += NT) {
       const int el = i % TE, b = i / TE;
       if (el < n_here) {
         const uint4 w = stream_words(p.seed, STREAM_NOISE, (uint32_t)b, (uint32_t)(e0 + el), t);
@@ -280,7 +324,7 @@ __global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorPar
     // record rows: [obs D][next_obs D][act, rew, done, ver]
     {
       const int rw = p.rec_words;
-      for (int i = tid; i < n_here * rw; i += kThreads) {
+      for (int i = tid; i < n_here * rw; i += NT) {
         const int el = i / rw, w = i % rw;
         const unsigned long long slot = (p.cursor0 + (unsigned long long)step * p.N + (e0 + el)) % (unsigned long long)p.C;
         float v;
@@ -297,7 +341,7 @@ __global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorPar
       p.block_ver[((p.cursor0 + (unsigned long long)step * p.N) % (unsigned long long)p.C) / p.N] = p.version;
     __syncthreads();
     // next state: the stepped state, or a fresh draw for finished episodes
-    for (int i = tid; i < TE * (D / 4); i += kThreads) {
+    for (int i = tid; i < TE * (D / 4); i += NT) {
       const int el = i % TE, b = i / TE;
       float4 v;
       if (el < n_here && sm.done[el]) {
@@ -313,7 +357,7 @@ __global__ void __launch_bounds__(kThreads) actor_lingauss_kernel(const ActorPar
     }
     __syncthreads();
   }
-  for (int i = tid; i < n_here * D; i += kThreads) {
+  for (int i = tid; i < n_here * D; i += NT) {
     const int el = i / D, k = i % D;
     p.state[(size_t)(e0 + el) * D + k] = sm.xs[k * TE + el];
   }
@@ -341,13 +385,24 @@ __global__ void init_env_kernel(int env_kind, int N, int S_d, uint2 seed, float*
 }
 
 template <typename K>
-cudaError_t launch_with_smem(K kernel, int grid, size_t smem_bytes, const ActorParams& p, cudaStream_t s) {
+cudaError_t launch_with_smem(K kernel, int grid, int threads, size_t smem_bytes, const ActorParams& p, cudaStream_t s) {
   if (smem_bytes > 48 * 1024) {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
     if (err != cudaSuccess) return err;
   }
-  kernel<<<grid, kThreads, smem_bytes, s>>>(p);
+  kernel<<<grid, threads, smem_bytes, s>>>(p);
   return cudaGetLastError();
+}
+
+constexpr size_t kSmemMax = 227 * 1024 - 1024;   // per block, leaving room for static shared memory
+constexpr size_t kSmemTwoPerSm = 112 * 1024;     // two resident blocks per SM
+
+template <int TE, int NT, int ENV>
+cudaError_t launch_small(int stage, size_t smem, const ActorParams& p, cudaStream_t s) {
+  const int grid = (p.N + TE - 1) / TE;
+  if (stage == 2) return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 2>, grid, NT, smem, p, s);
+  if (stage == 1) return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 1>, grid, NT, smem, p, s);
+  return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 0>, grid, NT, smem, p, s);
 }
 
 }  // namespace
@@ -360,14 +415,28 @@ cudaError_t launch_init_env(int env_kind, int N, int S_d, uint2 seed, float* sta
 }
 
 cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s) {
-  constexpr int TE = 32;
-  const int grid = (p.N + TE - 1) / TE;
-  const bool lg = env_kind == TJ_ENV_LINGAUSS;
-  const size_t smem = actor_smem_floats<TE>(p.D, p.Hp, p.Ap, lg) * sizeof(float);
-  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  if (env_kind == TJ_ENV_CARTPOLE) return launch_with_smem(actor_small_env_kernel<TE, TJ_ENV_CARTPOLE>, grid, smem, p, s);
-  if (env_kind == TJ_ENV_ACROBOT) return launch_with_smem(actor_small_env_kernel<TE, TJ_ENV_ACROBOT>, grid, smem, p, s);
-  return launch_with_smem(actor_lingauss_kernel<TE>, grid, smem, p, s);
+  if (env_kind == TJ_ENV_LINGAUSS) {
+    constexpr int TE = 32, NT = 256;
+    const size_t smem = actor_smem_floats(TE, p.D, p.Hp, p.Ap, true, 0) * sizeof(float);
+    if (smem > kSmemMax) return cudaErrorInvalidConfiguration;
+    return launch_with_smem(actor_lingauss_kernel<TE, NT>, (p.N + TE - 1) / TE, NT, smem, p, s);
+  }
+  // Tile: 16 envs x 128 threads while that still leaves SMs short of two blocks each, else 32 x 256.
+  const bool small_tile = p.N < 148 * 2 * 32;
+  const int TE = small_tile ? 16 : 32;
+  // Staging: everything if it fits (preferring a size that lets two blocks share an SM), else all but W2.
+  int stage = 0;
+  size_t smem = 0;
+  for (int st = 2; st >= 0; --st) {
+    smem = actor_smem_floats(TE, p.D, p.Hp, p.Ap, false, staged_floats(st, p.w_total, p.off_W2t, p.off_b2)) * sizeof(float);
+    if (smem <= (st == 0 ? kSmemMax : kSmemTwoPerSm) || (st == 2 && smem <= kSmemMax && p.H <= 160)) { stage = st; break; }
+    if (st == 0) return cudaErrorInvalidConfiguration;
+  }
+  if (env_kind == TJ_ENV_CARTPOLE)
+    return small_tile ? launch_small<16, 128, TJ_ENV_CARTPOLE>(stage, smem, p, s)
+                      : launch_small<32, 256, TJ_ENV_CARTPOLE>(stage, smem, p, s);
+  return small_tile ? launch_small<16, 128, TJ_ENV_ACROBOT>(stage, smem, p, s)
+                    : launch_small<32, 256, TJ_ENV_ACROBOT>(stage, smem, p, s);
 }
 
 }  // namespace tj

@@ -257,7 +257,7 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
   p.S_d = x->S_d; p.rec_words = x->rec_words; p.max_ep = x->max_ep; p.policy_kind = c.policy_kind;
   p.W = x->wbuf[x->active];
   p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
-  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3; p.w_total = x->wl.total;
   p.state = x->state; p.ep_step = x->ep_step; p.ep_return = x->ep_return;
   p.seed = make_uint2((uint32_t)c.seed, (uint32_t)(c.seed >> 32));
   p.explore_thr = explore_threshold(c.epsilon);
@@ -341,7 +341,7 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
   p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
   p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
   p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
-  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3; p.w_total = x->wl.total;
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = x->td_partial;
@@ -360,7 +360,7 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
   p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
   p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
   p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
-  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3;
+  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3; p.w_total = x->wl.total;
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = nullptr;

@@ -48,7 +48,7 @@ struct DevStats {
 struct ActorParams {
   int N, D, H, A, Aout, Hp, Ap, S_d, rec_words, max_ep, policy_kind;
   const float* W;  // packed weights, WeightLayout offsets below
-  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3;
+  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3, w_total;
   float* state;
   int* ep_step;
   float* ep_return;
@@ -79,7 +79,7 @@ struct TdParams {
   int n, D, H, A, Hp, Ap;
   const float* Wonline;
   const float* Wtarget;
-  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3;
+  size_t off_W1t, off_b1, off_W2t, off_b2, off_W3t, off_b3, w_total;
   const float* obs;
   const int* act;
   const float* rew;

@@ -1,5 +1,6 @@
 // Learner-side kernels: parameter publish (repack), eligible-block list, staleness-bounded sampling with
 // gather, TD error / Huber loss, and the GAE reverse scan.
+#include "tj_async.cuh"
 #include "tj_device.cuh"
 #include "tj_internal.h"
 #include "tj_mlp.cuh"
@@ -129,38 +130,75 @@ __global__ void sample_gather_kernel(const SampleParams p) {
 }
 
 // TD error on a tile of TE samples: online forward on obs, target forward on next_obs.
-template <int TE>
-__global__ void __launch_bounds__(kThreads) td_kernel(const TdParams p) {
-  extern __shared__ __align__(16) float smem[];
+// STAGE as in the actor kernel: 0 = parameters from global memory, 1 = all but the HxH matrix staged in shared
+// memory, 2 = all staged.  The staging buffer is filled twice (online, then target parameters).
+template <int STAGE>
+__device__ __forceinline__ MlpWeights td_stage(const TdParams& p, const float* W, float* wsm, uint64_t* bar, bool issue) {
+  MlpWeights w;
+  if (STAGE == 0) {
+    w.W1t = W + p.off_W1t; w.b1 = W + p.off_b1; w.W2t = W + p.off_W2t; w.b2 = W + p.off_b2;
+    w.W3t = W + p.off_W3t; w.b3 = W + p.off_b3;
+    return w;
+  }
+  const size_t gap = STAGE == 1 ? p.off_b2 - p.off_W2t : 0;
+  if (issue) {
+    if (STAGE == 2) {
+      mbar_expect_tx(bar, (uint32_t)(p.w_total * sizeof(float)));
+      bulk_copy_chunks(wsm, W, p.w_total * sizeof(float), bar);
+    } else {
+      const size_t head = p.off_W2t, tail = p.w_total - p.off_b2;
+      mbar_expect_tx(bar, (uint32_t)((head + tail) * sizeof(float)));
+      bulk_copy_chunks(wsm, W, head * sizeof(float), bar);
+      bulk_copy_chunks(wsm + head, W + p.off_b2, tail * sizeof(float), bar);
+    }
+  }
+  w.W1t = wsm + p.off_W1t; w.b1 = wsm + p.off_b1;
+  w.W2t = STAGE == 2 ? wsm + p.off_W2t : W + p.off_W2t;
+  w.b2 = wsm + p.off_b2 - gap; w.W3t = wsm + p.off_W3t - gap; w.b3 = wsm + p.off_b3 - gap;
+  return w;
+}
+
+template <int TE, int NT, int STAGE>
+__global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
+  extern __shared__ __align__(128) float smem[];
+  __shared__ __align__(8) uint64_t wbar;
+  const size_t staged = STAGE == 2 ? p.w_total : (STAGE == 1 ? p.w_total - (p.off_b2 - p.off_W2t) : 0);
   const int Dx = (p.D + 3) & ~3;
-  float* xs = smem;
+  float* wsm = smem;
+  float* xs = wsm + staged;
   float* h1 = xs + (size_t)Dx * TE;
   float* h2 = h1 + (size_t)p.Hp * TE;
   float* out = h2 + (size_t)p.Hp * TE;
   float* qsel = out + (size_t)p.Ap * TE;
   float* hub = qsel + TE;
   const int tid = threadIdx.x, j0 = blockIdx.x * TE, n_here = min(TE, p.n - j0), D = p.D;
+  if (STAGE > 0) {
+    if (tid == 0) mbar_init(&wbar, 1);
+    __syncthreads();
+  }
+  MlpWeights mw = td_stage<STAGE>(p, p.Wonline, wsm, &wbar, tid == 0);
 
-  for (int i = tid; i < TE * D; i += kThreads) {
+  for (int i = tid; i < TE * D; i += NT) {
     const int el = i / D, k = i % D;
     xs[k * TE + el] = el < n_here ? p.obs[(size_t)(j0 + el) * D + k] : 0.f;
   }
+  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) return;
   __syncthreads();
-  mlp_forward_tile<TE>(p.Wonline, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, D, p.H, p.Hp, p.A,
-                       p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < n_here) {
     int a = p.act[j0 + tid];
     a = a < 0 ? 0 : (a >= p.A ? p.A - 1 : a);
     qsel[tid] = out[a * TE + tid];
   }
-  __syncthreads();
-  for (int i = tid; i < TE * D; i += kThreads) {
+  __syncthreads();  // every thread is done with the online parameters: the buffer may be refilled
+  mw = td_stage<STAGE>(p, p.Wtarget, wsm, &wbar, tid == 0);
+  for (int i = tid; i < TE * D; i += NT) {
     const int el = i / D, k = i % D;
     xs[k * TE + el] = el < n_here ? p.next_obs[(size_t)(j0 + el) * D + k] : 0.f;
   }
+  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 1)) return;
   __syncthreads();
-  mlp_forward_tile<TE>(p.Wtarget, p.off_W1t, p.off_b1, p.off_W2t, p.off_b2, p.off_W3t, p.off_b3, D, p.H, p.Hp, p.A,
-                       p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < TE) {
     float h = 0.f;
     if (tid < n_here) {
@@ -215,7 +253,8 @@ __global__ void gae_kernel(const float* __restrict__ rew, const float* __restric
   }
 }
 
-constexpr int kTdTile = 32;
+constexpr int kTdTile = 16;
+constexpr int kTdThreads = 128;
 
 }  // namespace
 
@@ -245,18 +284,31 @@ cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s) {
 
 int td_grid(int n) { return (n + kTdTile - 1) / kTdTile; }
 
+template <int STAGE>
+cudaError_t launch_td_stage(const TdParams& p, size_t smem, int grid, cudaStream_t s) {
+  auto kernel = td_kernel<kTdTile, kTdThreads, STAGE>;
+  if (smem > 48 * 1024) {
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+  }
+  kernel<<<grid, kTdThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_td(const TdParams& p, cudaStream_t s) {
   constexpr int TE = kTdTile;
   const int Dx = (p.D + 3) & ~3;
-  const size_t smem = ((size_t)Dx * TE + 2 * (size_t)p.Hp * TE + (size_t)p.Ap * TE + 2 * TE) * sizeof(float);
-  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  if (smem > 48 * 1024) {
-    cudaError_t err = cudaFuncSetAttribute(td_kernel<TE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
-  }
+  const size_t acts = (size_t)Dx * TE + 2 * (size_t)p.Hp * TE + (size_t)p.Ap * TE + 2 * TE;
+  const size_t limit = 226 * 1024;
+  const size_t smem2 = (acts + p.w_total) * sizeof(float);
+  const size_t smem1 = (acts + p.w_total - (p.off_b2 - p.off_W2t)) * sizeof(float);
+  const size_t smem0 = acts * sizeof(float);
   const int grid = td_grid(p.n);
-  td_kernel<TE><<<grid, kThreads, smem, s>>>(p);
-  cudaError_t err = cudaGetLastError();
+  cudaError_t err;
+  if (smem2 <= 112 * 1024) err = launch_td_stage<2>(p, smem2, grid, s);
+  else if (smem1 <= limit) err = launch_td_stage<1>(p, smem1, grid, s);
+  else if (smem0 <= limit) err = launch_td_stage<0>(p, smem0, grid, s);
+  else return cudaErrorInvalidConfiguration;
   if (err != cudaSuccess) return err;
   if (p.loss_out) {
     td_finish_kernel<<<1, 32, 0, s>>>(p.partial, grid, p.n, p.loss_out);

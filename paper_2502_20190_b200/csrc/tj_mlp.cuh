@@ -1,4 +1,4 @@
-// FP32 dense layer for a tile of TE environments (or samples) held in shared memory.
+// FP32 dense layers for a tile of TE environments (or samples) held in shared memory.
 //
 // Activations are stored k-major, x[k][e], so that the four environments a thread owns are one 128-bit
 // shared-memory load and the four output neurons it owns are one 128-bit load from the transposed weight
@@ -9,8 +9,6 @@
 
 namespace tj {
 
-constexpr int kThreads = 256;
-
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_TANH = 2 };
 
 template <int ACT>
@@ -20,14 +18,27 @@ __device__ __forceinline__ float activate(float v) {
   return v;
 }
 
+// weights either sit in shared memory (plain load) or in global memory (read-only path)
+template <bool W_SMEM>
+__device__ __forceinline__ float4 load_w4(const float* p) {
+  if (W_SMEM) return *reinterpret_cast<const float4*>(p);
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+template <bool W_SMEM>
+__device__ __forceinline__ float load_w1(const float* p) {
+  if (W_SMEM) return *p;
+  return __ldg(p);
+}
+
 // y[i][e] = act(bias + sum_k Wt[k][i] x[k][e]) for i < round_up4(n_out), e < TE.
-//   Wt: [K][ldw] (global, zero padded to ldw = round_up4(n_out)),  x: [K][TE] shared,  y: [round_up4(n_out)][TE] shared
-//   ENV_BIAS = false: bias = b[i];  true: bias = b[bias_row[e] * ldw + i] (a per-environment row of b)
-template <int TE, int ACT, bool ENV_BIAS>
+//   Wt: [K][ldw] (zero padded to ldw = round_up4(n_out)),  x: [K][TE] shared,  y: [round_up4(n_out)][TE] shared
+//   ENV_BIAS = false: bias = b[i];  true: bias = b[bias_row[e] * ldw + i] (a per-environment row of b, global)
+//   W_SMEM / B_SMEM: whether Wt / b sit in shared memory (else global, read-only path)
+template <int TE, int NT, int ACT, bool ENV_BIAS, bool W_SMEM, bool B_SMEM = W_SMEM>
 __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const float* __restrict__ b, int ldw, int K,
                                             int n_out, const float* __restrict__ x, float* __restrict__ y,
                                             const int* __restrict__ bias_row) {
-  constexpr int EG = TE / 4, NG = kThreads / EG;
+  constexpr int EG = TE / 4, NG = NT / EG;
   const int eg = threadIdx.x % EG, ng = threadIdx.x / EG;
   for (int i0 = ng * 4; i0 < n_out; i0 += NG * 4) {
     float acc[4][4];  // [neuron][env]
@@ -38,16 +49,16 @@ __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const 
         acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w;
       }
     } else {
-      const float4 bb = __ldg(reinterpret_cast<const float4*>(b + i0));
+      const float4 bb = load_w4<B_SMEM>(b + i0);
 #pragma unroll
       for (int e = 0; e < 4; ++e) { acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w; }
     }
     const float* xp = x + eg * 4;
     const float* wp = Wt + i0;
-#pragma unroll 4
+#pragma unroll 8
     for (int k = 0; k < K; ++k) {
       const float4 xv = *reinterpret_cast<const float4*>(xp + k * TE);
-      const float4 wv = __ldg(reinterpret_cast<const float4*>(wp + (size_t)k * ldw));
+      const float4 wv = load_w4<W_SMEM>(wp + (size_t)k * ldw);
       const float xe[4] = {xv.x, xv.y, xv.z, xv.w};
       const float wn[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
@@ -65,17 +76,37 @@ __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const 
   }
 }
 
+// Narrow output layer (a few actions): one thread per (environment, output), same FMA chain.
+template <int TE, int NT, bool W_SMEM>
+__device__ __forceinline__ void head_layer(const float* __restrict__ Wt, const float* __restrict__ b, int ldw, int K,
+                                           int n_out, const float* __restrict__ x, float* __restrict__ y) {
+  for (int idx = threadIdx.x; idx < TE * n_out; idx += NT) {
+    const int e = idx % TE, a = idx / TE;
+    float acc = load_w1<W_SMEM>(b + a);
+    const float* xp = x + e;
+    const float* wp = Wt + a;
+#pragma unroll 8
+    for (int k = 0; k < K; ++k) acc = fmaf(load_w1<W_SMEM>(wp + (size_t)k * ldw), xp[k * TE], acc);
+    y[a * TE + e] = acc;
+  }
+}
+
+// Where each part of the packed parameters is read from (shared or global memory).
+struct MlpWeights {
+  const float *W1t, *b1, *W2t, *b2, *W3t, *b3;
+};
+
 // Policy forward for the tile: x [D][TE] -> h1 -> h2 -> out [Ap][TE]; ends with a barrier.
-template <int TE>
-__device__ __forceinline__ void mlp_forward_tile(const float* __restrict__ W, size_t off_W1t, size_t off_b1,
-                                                 size_t off_W2t, size_t off_b2, size_t off_W3t, size_t off_b3, int D,
-                                                 int H, int Hp, int Aout, int Ap, const float* x, float* h1, float* h2,
-                                                 float* out) {
-  dense_layer<TE, ACT_RELU, false>(W + off_W1t, W + off_b1, Hp, D, H, x, h1, nullptr);
+// SMALL_SMEM: W1t, the biases and W3t are in shared memory;  W2_SMEM: W2t is too.
+template <int TE, int NT, bool SMALL_SMEM, bool W2_SMEM>
+__device__ __forceinline__ void mlp_forward_tile(const MlpWeights& w, int D, int H, int Hp, int Aout, int Ap,
+                                                 const float* x, float* h1, float* h2, float* out) {
+  dense_layer<TE, NT, ACT_RELU, false, SMALL_SMEM>(w.W1t, w.b1, Hp, D, H, x, h1, nullptr);
   __syncthreads();
-  dense_layer<TE, ACT_RELU, false>(W + off_W2t, W + off_b2, Hp, H, H, h1, h2, nullptr);
+  dense_layer<TE, NT, ACT_RELU, false, W2_SMEM, SMALL_SMEM>(w.W2t, w.b2, Hp, H, H, h1, h2, nullptr);
   __syncthreads();
-  dense_layer<TE, ACT_NONE, false>(W + off_W3t, W + off_b3, Ap, H, Aout, h2, out, nullptr);
+  if (Aout <= 8) head_layer<TE, NT, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out);
+  else dense_layer<TE, NT, ACT_NONE, false, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out, nullptr);
   __syncthreads();
 }
 

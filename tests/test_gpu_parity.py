@@ -352,7 +352,17 @@ def test_segment_mode_lockstep(env):
     for key in ("produced", "consumed", "dropped_stale", "dropped_overwritten", "starved_calls",
                 "max_sampled_staleness", "staleness_hist", "learner_steps"):
         assert gs[key] == os_[key], key
-    assert gs["dropped_stale"] > 0 and gs["dropped_overwritten"] > 0
+    assert gs["dropped_stale"] > 0
+    # the producer laps the consumer: five more segments into three slots overwrite unconsumed ones
+    ctx.actor_step(12 * 5)
+    o.actor_step(12 * 5)
+    while ctx.segment_acquire(allow=(0, -7))[0] == 0:
+        assert o.segment_acquire()[0] == 0
+    assert o.segment_acquire()[0] == -7
+    gs, os_ = ctx.stats(), o.stats()
+    for key in ("produced", "consumed", "dropped_stale", "dropped_overwritten", "starved_calls", "learner_steps"):
+        assert gs[key] == os_[key], key
+    assert gs["dropped_overwritten"] > 0
 
 
 def test_categorical_actions_follow_the_margin_rule(env):
