@@ -231,16 +231,43 @@ __global__ void td_finish_kernel(const float* __restrict__ partial, int n_partia
   }
 }
 
-// GAE: one thread per environment walks its column backwards; a warp reads 32 consecutive environments.
-__global__ void gae_kernel(const float* __restrict__ rew, const float* __restrict__ val,
-                           const uint8_t* __restrict__ done, int T, int N, float gamma, float lambda,
-                           float* __restrict__ adv, float* __restrict__ ret) {
+// GAE: one thread per environment walks its column backwards; a warp reads 32 consecutive environments, so
+// every access is a full 128-byte line.  The recurrence is serial in t, but its inputs are not: each thread
+// fetches the next GAE_U time steps' rewards, values and done flags before it needs them, which keeps enough
+// loads in flight to stream at HBM speed.
+constexpr int GAE_U = 8;
+__global__ void __launch_bounds__(128) gae_kernel(const float* __restrict__ rew, const float* __restrict__ val,
+                                                  const uint8_t* __restrict__ done, int T, int N, float gamma,
+                                                  float lambda, float* __restrict__ adv, float* __restrict__ ret) {
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= N) return;
   float next_adv = 0.f;
-  float v_next = val[(size_t)T * N + e];
+  float v_next = __ldcs(val + (size_t)T * N + e);
   const float gl = gamma * lambda;
-  for (int t = T - 1; t >= 0; --t) {
+  int t = T - 1;
+  for (; t >= GAE_U - 1; t -= GAE_U) {
+    float r[GAE_U], v[GAE_U];
+    uint8_t d[GAE_U];
+#pragma unroll
+    for (int u = 0; u < GAE_U; ++u) {
+      const size_t i = (size_t)(t - u) * N + e;
+      r[u] = __ldcs(rew + i);
+      v[u] = __ldcs(val + i);
+      d[u] = __ldcs(done + i);
+    }
+#pragma unroll
+    for (int u = 0; u < GAE_U; ++u) {
+      const size_t i = (size_t)(t - u) * N + e;
+      const float nd = d[u] ? 0.f : 1.f;
+      const float delta = r[u] + gamma * nd * v_next - v[u];
+      const float a = delta + gl * nd * next_adv;
+      __stcs(adv + i, a);
+      __stcs(ret + i, a + v[u]);
+      next_adv = a;
+      v_next = v[u];
+    }
+  }
+  for (; t >= 0; --t) {
     const size_t i = (size_t)t * N + e;
     const float nd = done[i] ? 0.f : 1.f;
     const float v = val[i];
