@@ -87,7 +87,7 @@ __device__ __forceinline__ float4 reset4(uint2 seed, uint32_t block, uint32_t e,
 // ------------------------------------------------------------------------------------------------
 // CartPole / Acrobot: one thread owns one environment (state in registers).
 // ------------------------------------------------------------------------------------------------
-template <int TE, int NT, int ENV, int STAGE>
+template <int TE, int NT, int EPT, int ENV, int STAGE>
 __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p) {
   extern __shared__ __align__(128) float smem[];
   __shared__ __align__(8) uint64_t wbar;
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
         if (k < p.D) sm.xs[k * TE + tid] = owner ? obs[k] : 0.f;
     }
     __syncthreads();
-    mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+    mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (owner) {
       auto logit = [&](int i) { return sm.out[i * TE + tid]; };
       if (p.dbg_logits) {
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
           if (k < p.D) sm.xs[k * TE + tid] = owner ? o2[k] : 0.f;
       }
       __syncthreads();
-      mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+      mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
       if (owner) {
         const int slot = (int)((long long)(t / (unsigned long long)p.T) % p.G);
         p.seg_val[((size_t)slot * (p.T + 1) + p.T) * p.N + e] = sm.out[p.A * TE + tid];
@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p)
 
   for (int step = 0; step < p.n_steps; ++step) {
     const unsigned long long t = (unsigned long long)p.t0 + step;
-    mlp_forward_tile<TE, NT, false, false>(mw, D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+    mlp_forward_tile<TE, NT, 4, false, false>(mw, D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (tid < TE) {
       int a = 0;
       if (tid < n_here) {
@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p)
     }
     __syncthreads();
     // s' = tanh(A s + B[a]) ...
-    dense_layer<TE, NT, ACT_TANH, true, false>(p.lgAt, p.lgB, Dp, D, D, sm.xs, sm.nxt, sm.act);
+    dense_layer<TE, NT, 4, ACT_TANH, true, false>(p.lgAt, p.lgB, Dp, D, D, sm.xs, sm.nxt, sm.act);
     __syncthreads();
     // ... + noise_std * n, four normals per Philox call
     for (int i = tid; i < TE * (D / 4); i += NT) {
@@ -397,12 +397,12 @@ cudaError_t launch_with_smem(K kernel, int grid, int threads, size_t smem_bytes,
 constexpr size_t kSmemMax = 227 * 1024 - 1024;   // per block, leaving room for static shared memory
 constexpr size_t kSmemTwoPerSm = 112 * 1024;     // two resident blocks per SM
 
-template <int TE, int NT, int ENV>
+template <int TE, int NT, int EPT, int ENV>
 cudaError_t launch_small(int stage, size_t smem, const ActorParams& p, cudaStream_t s) {
   const int grid = (p.N + TE - 1) / TE;
-  if (stage == 2) return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 2>, grid, NT, smem, p, s);
-  if (stage == 1) return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 1>, grid, NT, smem, p, s);
-  return launch_with_smem(actor_small_env_kernel<TE, NT, ENV, 0>, grid, NT, smem, p, s);
+  if (stage == 2) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 2>, grid, NT, smem, p, s);
+  if (stage == 1) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 1>, grid, NT, smem, p, s);
+  return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 0>, grid, NT, smem, p, s);
 }
 
 }  // namespace
@@ -432,11 +432,13 @@ cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s) {
     if (smem <= (st == 0 ? kSmemMax : kSmemTwoPerSm) || (st == 2 && smem <= kSmemMax && p.H <= 160)) { stage = st; break; }
     if (st == 0) return cudaErrorInvalidConfiguration;
   }
+  // Small N: 16 envs x 128 threads, 4 envs per thread (more warps; the problem is latency-bound).
+  // Large N: 32 envs x 256 threads, 8 envs per thread (each weight fetched feeds twice the FMAs).
   if (env_kind == TJ_ENV_CARTPOLE)
-    return small_tile ? launch_small<16, 128, TJ_ENV_CARTPOLE>(stage, smem, p, s)
-                      : launch_small<32, 256, TJ_ENV_CARTPOLE>(stage, smem, p, s);
-  return small_tile ? launch_small<16, 128, TJ_ENV_ACROBOT>(stage, smem, p, s)
-                    : launch_small<32, 256, TJ_ENV_ACROBOT>(stage, smem, p, s);
+    return small_tile ? launch_small<16, 128, 4, TJ_ENV_CARTPOLE>(stage, smem, p, s)
+                      : launch_small<32, 256, 8, TJ_ENV_CARTPOLE>(stage, smem, p, s);
+  return small_tile ? launch_small<16, 128, 4, TJ_ENV_ACROBOT>(stage, smem, p, s)
+                    : launch_small<32, 256, 8, TJ_ENV_ACROBOT>(stage, smem, p, s);
 }
 
 }  // namespace tj

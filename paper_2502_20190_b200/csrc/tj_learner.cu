@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   }
   if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) return;
   __syncthreads();
-  mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, 4, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < n_here) {
     int a = p.act[j0 + tid];
     a = a < 0 ? 0 : (a >= p.A ? p.A - 1 : a);
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   }
   if (STAGE > 0 && !mbar_wait_bounded(&wbar, 1)) return;
   __syncthreads();
-  mlp_forward_tile<TE, NT, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, 4, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < TE) {
     float h = 0.f;
     if (tid < n_here) {

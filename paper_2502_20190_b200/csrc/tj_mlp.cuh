@@ -34,45 +34,53 @@ __device__ __forceinline__ float load_w1(const float* p) {
 //   Wt: [K][ldw] (zero padded to ldw = round_up4(n_out)),  x: [K][TE] shared,  y: [round_up4(n_out)][TE] shared
 //   ENV_BIAS = false: bias = b[i];  true: bias = b[bias_row[e] * ldw + i] (a per-environment row of b, global)
 //   W_SMEM / B_SMEM: whether Wt / b sit in shared memory (else global, read-only path)
-template <int TE, int NT, int ACT, bool ENV_BIAS, bool W_SMEM, bool B_SMEM = W_SMEM>
+//   EPT: environments per thread (4 or 8).  A thread owns EPT environments x 4 neurons; with 8 environments each
+//   weight fetched feeds twice as many FMAs, which is what shared-memory (or L2) bandwidth asks for.
+template <int TE, int NT, int EPT, int ACT, bool ENV_BIAS, bool W_SMEM, bool B_SMEM = W_SMEM>
 __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const float* __restrict__ b, int ldw, int K,
                                             int n_out, const float* __restrict__ x, float* __restrict__ y,
                                             const int* __restrict__ bias_row) {
-  constexpr int EG = TE / 4, NG = NT / EG;
+  constexpr int EG = TE / EPT, NG = NT / EG, XV = EPT / 4;
   const int eg = threadIdx.x % EG, ng = threadIdx.x / EG;
   for (int i0 = ng * 4; i0 < n_out; i0 += NG * 4) {
-    float acc[4][4];  // [neuron][env]
+    float acc[4][EPT];  // [neuron][env]
     if (ENV_BIAS) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float4 bb = __ldg(reinterpret_cast<const float4*>(b + (size_t)bias_row[eg * 4 + e] * ldw + i0));
+      for (int e = 0; e < EPT; ++e) {
+        const float4 bb = __ldg(reinterpret_cast<const float4*>(b + (size_t)bias_row[eg * EPT + e] * ldw + i0));
         acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w;
       }
     } else {
       const float4 bb = load_w4<B_SMEM>(b + i0);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) { acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w; }
+      for (int e = 0; e < EPT; ++e) { acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w; }
     }
-    const float* xp = x + eg * 4;
+    const float* xp = x + eg * EPT;
     const float* wp = Wt + i0;
 #pragma unroll 8
     for (int k = 0; k < K; ++k) {
-      const float4 xv = *reinterpret_cast<const float4*>(xp + k * TE);
+      float xe[EPT];
+#pragma unroll
+      for (int v = 0; v < XV; ++v) {
+        const float4 xv = *reinterpret_cast<const float4*>(xp + k * TE + 4 * v);
+        xe[4 * v] = xv.x; xe[4 * v + 1] = xv.y; xe[4 * v + 2] = xv.z; xe[4 * v + 3] = xv.w;
+      }
       const float4 wv = load_w4<W_SMEM>(wp + (size_t)k * ldw);
-      const float xe[4] = {xv.x, xv.y, xv.z, xv.w};
       const float wn[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
       for (int n = 0; n < 4; ++n)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) acc[n][e] = fmaf(wn[n], xe[e], acc[n][e]);
+        for (int e = 0; e < EPT; ++e) acc[n][e] = fmaf(wn[n], xe[e], acc[n][e]);
     }
 #pragma unroll
-    for (int n = 0; n < 4; ++n) {
-      float4 o;
-      o.x = activate<ACT>(acc[n][0]); o.y = activate<ACT>(acc[n][1]);
-      o.z = activate<ACT>(acc[n][2]); o.w = activate<ACT>(acc[n][3]);
-      *reinterpret_cast<float4*>(y + (size_t)(i0 + n) * TE + eg * 4) = o;
-    }
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+      for (int v = 0; v < XV; ++v) {
+        float4 o;
+        o.x = activate<ACT>(acc[n][4 * v]); o.y = activate<ACT>(acc[n][4 * v + 1]);
+        o.z = activate<ACT>(acc[n][4 * v + 2]); o.w = activate<ACT>(acc[n][4 * v + 3]);
+        *reinterpret_cast<float4*>(y + (size_t)(i0 + n) * TE + eg * EPT + 4 * v) = o;
+      }
   }
 }
 
@@ -98,15 +106,15 @@ struct MlpWeights {
 
 // Policy forward for the tile: x [D][TE] -> h1 -> h2 -> out [Ap][TE]; ends with a barrier.
 // SMALL_SMEM: W1t, the biases and W3t are in shared memory;  W2_SMEM: W2t is too.
-template <int TE, int NT, bool SMALL_SMEM, bool W2_SMEM>
+template <int TE, int NT, int EPT, bool SMALL_SMEM, bool W2_SMEM>
 __device__ __forceinline__ void mlp_forward_tile(const MlpWeights& w, int D, int H, int Hp, int Aout, int Ap,
                                                  const float* x, float* h1, float* h2, float* out) {
-  dense_layer<TE, NT, ACT_RELU, false, SMALL_SMEM>(w.W1t, w.b1, Hp, D, H, x, h1, nullptr);
+  dense_layer<TE, NT, EPT, ACT_RELU, false, SMALL_SMEM>(w.W1t, w.b1, Hp, D, H, x, h1, nullptr);
   __syncthreads();
-  dense_layer<TE, NT, ACT_RELU, false, W2_SMEM, SMALL_SMEM>(w.W2t, w.b2, Hp, H, H, h1, h2, nullptr);
+  dense_layer<TE, NT, EPT, ACT_RELU, false, W2_SMEM, SMALL_SMEM>(w.W2t, w.b2, Hp, H, H, h1, h2, nullptr);
   __syncthreads();
   if (Aout <= 8) head_layer<TE, NT, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out);
-  else dense_layer<TE, NT, ACT_NONE, false, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out, nullptr);
+  else dense_layer<TE, NT, EPT, ACT_NONE, false, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out, nullptr);
   __syncthreads();
 }
 
