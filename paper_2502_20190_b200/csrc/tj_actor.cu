@@ -240,7 +240,8 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
 template <int TE, int NT>
 __global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p) {
   extern __shared__ __align__(128) float smem[];
-  const ActorSmem sm = carve(smem, TE, p.D, p.Hp, p.Ap, true, 0);
+  const bool ext = p.logits_in != nullptr;   // network outputs come from the tensor-core kernel
+  const ActorSmem sm = carve(smem, TE, p.D, ext ? 0 : p.Hp, ext ? 0 : p.Ap, true, 0);
   __shared__ uint64_t unused_bar;
   const MlpWeights mw = stage_weights<0>(p, nullptr, &unused_bar, false);
   const int tid = threadIdx.x;
@@ -265,12 +266,12 @@ __global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p)
 
   for (int step = 0; step < p.n_steps; ++step) {
     const unsigned long long t = (unsigned long long)p.t0 + step;
-    mlp_forward_tile<TE, NT, 4, false, false>(mw, D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+    if (!ext) mlp_forward_tile<TE, NT, 4, false, false>(mw, D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (tid < TE) {
       int a = 0;
       if (tid < n_here) {
         const int e = e0 + tid;
-        auto logit = [&](int i) { return sm.out[i * TE + tid]; };
+        auto logit = [&](int i) { return ext ? p.logits_in[(size_t)e * p.A + i] : sm.out[i * TE + tid]; };
         if (p.dbg_logits) {
           float* dl = p.dbg_logits + ((size_t)step * p.N + e) * p.A;
           for (int i = 0; i < p.A; ++i) dl[i] = logit(i);
@@ -417,7 +418,8 @@ cudaError_t launch_init_env(int env_kind, int N, int S_d, uint2 seed, float* sta
 cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s) {
   if (env_kind == TJ_ENV_LINGAUSS) {
     constexpr int TE = 32, NT = 256;
-    const size_t smem = actor_smem_floats(TE, p.D, p.Hp, p.Ap, true, 0) * sizeof(float);
+    const bool ext = p.logits_in != nullptr;
+    const size_t smem = actor_smem_floats(TE, p.D, ext ? 0 : p.Hp, ext ? 0 : p.Ap, true, 0) * sizeof(float);
     if (smem > kSmemMax) return cudaErrorInvalidConfiguration;
     return launch_with_smem(actor_lingauss_kernel<TE, NT>, (p.N + TE - 1) / TE, NT, smem, p, s);
   }

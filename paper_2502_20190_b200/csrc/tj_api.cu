@@ -14,6 +14,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxTdRows = 1 << 20;
+constexpr int kMaxTcTdRows = 1 << 16;   // rows of Q outputs the tensor-core TD path keeps in the workspace
 
 struct Carver {
   char* base;
@@ -111,6 +112,16 @@ size_t carve(tj_ctx* x, void* base) {
     x->lgB = cv.take<float>((size_t)c.n_actions * round_up4(D));
     x->lg_stage = cv.take<float>((size_t)D * D + (size_t)c.n_actions * D);
   }
+  x->use_tc = c.weight_dtype == TJ_W_BF16 && tc_mlp_supported(D, c.hidden, c.n_actions + vh);
+  if (x->use_tc) {
+    const size_t ne = tc_weight_elems(D, c.hidden);
+    x->wtc[0] = cv.take<uint16_t>(ne);
+    x->wtc[1] = cv.take<uint16_t>(ne);
+    x->wtc_target = cv.take<uint16_t>(ne);
+    x->logits_buf = cv.take<float>((size_t)N * c.n_actions);
+    x->tdq[0] = cv.take<float>((size_t)kMaxTcTdRows * c.n_actions);
+    x->tdq[1] = cv.take<float>((size_t)kMaxTcTdRows * c.n_actions);
+  }
   return (cv.off + kAlign - 1) & ~(kAlign - 1);
 }
 
@@ -176,6 +187,8 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
 
   cudaError_t e = cudaSetDevice(cfg->device);
   if (e != cudaSuccess) { g_err = std::string("cudaSetDevice: ") + cudaGetErrorString(e); delete x; return TJ_ERR_CUDA; }
+  x->sm_count = 148;
+  cudaDeviceGetAttribute(&x->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
   auto bail = [&](cudaError_t err, const char* where) {
     g_err = std::string(where) + ": " + cudaGetErrorString(err);
     delete x;
@@ -230,11 +243,20 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
   if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->stream)) != cudaSuccess)
     return cuda_fail(x, e, "publish: repack");
+  uint16_t* dst_tc = nullptr;
+  if (x->use_tc) {
+    dst_tc = x->version == 0 ? x->wtc[x->active] : x->wtc[next];
+    if ((e = launch_pack_tc_weights(src, dst_tc, x->D, x->H, x->A, x->value_head, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: tensor-core repack");
+  }
   if (x->version != 0) x->active = next;
   x->version += 1;
   if (!x->has_target || (x->cfg.target_sync_interval > 0 && x->k - x->k_last_sync >= x->cfg.target_sync_interval)) {
     if ((e = cudaMemcpyAsync(x->wtarget, dst, x->wl.total * sizeof(float), cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: target refresh");
+    if (x->use_tc && (e = cudaMemcpyAsync(x->wtc_target, dst_tc, tc_weight_elems(x->D, x->H) * sizeof(uint16_t),
+                                          cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: target refresh (tensor-core weights)");
     x->has_target = true;
     x->k_last_sync = x->k;
   }
@@ -269,7 +291,27 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
   p.seg_logp = x->seg_logp; p.seg_val = x->seg_val;
   p.lgAt = x->lgAt; p.lgB = x->lgB; p.lg_noise_std = c.lg_noise_std; p.lg_done_norm = c.lg_done_norm;
   p.dbg_logits = dbg_logits; p.stats = x->dstats;
-  cudaError_t e = launch_actor(c.env_kind, p, x->stream);
+  cudaError_t e = cudaSuccess;
+  if (x->use_tc && c.env_kind == TJ_ENV_LINGAUSS) {
+    // network on the tensor cores, then the env/selection/insert kernel reads its outputs; one pair per step
+    const float* W = x->wbuf[x->active];
+    for (int i = 0; i < n_steps && e == cudaSuccess; ++i) {
+      TcMlpParams t{};
+      t.x = x->state; t.n = x->N; t.D = x->D; t.H = x->H; t.Aout = x->A;
+      t.wtc = x->wtc[x->active];
+      t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
+      t.out = x->logits_buf; t.error = &x->dstats->error;
+      e = launch_tc_mlp(t, x->sm_count, x->stream);
+      if (e != cudaSuccess) break;
+      ActorParams q = p;
+      q.n_steps = 1; q.t0 = x->t + i; q.cursor0 = x->cursor + (uint64_t)i * x->N;
+      q.logits_in = x->logits_buf;
+      q.dbg_logits = dbg_logits ? dbg_logits + (size_t)i * x->N * x->A : nullptr;
+      e = launch_actor(c.env_kind, q, x->stream);
+    }
+  } else {
+    e = launch_actor(c.env_kind, p, x->stream);
+  }
   if (e != cudaSuccess) return cuda_fail(x, e, "actor step");
   // host mirror of what the kernel does to versions, cursor and segment slots
   for (int i = 0; i < n_steps; ++i) {
@@ -345,7 +387,26 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = x->td_partial;
-  cudaError_t e = launch_td(p, x->stream);
+  cudaError_t e;
+  if (x->use_tc && b->n <= kMaxTcTdRows) {
+    // two tensor-core forwards (online on obs, target on next_obs), then the elementwise TD/Huber pass
+    for (int which = 0; which < 2; ++which) {
+      const float* W = which == 0 ? x->wbuf[x->active] : x->wtarget;
+      TcMlpParams t{};
+      t.x = which == 0 ? b->obs : b->next_obs; t.n = b->n; t.D = x->D; t.H = x->H; t.Aout = x->A;
+      t.wtc = which == 0 ? x->wtc[x->active] : x->wtc_target;
+      t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
+      t.out = x->tdq[which]; t.error = &x->dstats->error;
+      if ((e = launch_tc_mlp(t, x->sm_count, x->stream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
+    }
+    if ((e = launch_td_from_q(x->tdq[0], x->tdq[1], b->n, x->A, b->act, b->rew, b->done, p.gamma, p.kappa, td_out,
+                              huber_out, x->td_partial, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "TD error (elementwise)");
+    if (loss_mean_out && (e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "TD error (loss reduction)");
+    return TJ_OK;
+  }
+  e = launch_td(p, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error");
   return TJ_OK;
 }

@@ -72,6 +72,7 @@ struct ActorParams {
   const float* lgB;   // [A][Dp]
   float lg_noise_std, lg_done_norm;
   float* dbg_logits;
+  const float* logits_in;  // when set, network outputs [N][A] computed by another kernel (tensor-core path)
   DevStats* stats;
 };
 
@@ -109,6 +110,24 @@ struct SampleParams {
   int* ver;
   DevStats* stats;
 };
+
+struct TcMlpParams {
+  const float* x;          // [n][D] FP32 rows
+  int n, D, H, Aout;
+  const uint16_t* wtc;     // BF16 weight chunks in streaming order
+  const float *b1, *b2, *b3;
+  float* out;              // [n][Aout]
+  unsigned long long* error;
+};
+
+bool tc_mlp_supported(int D, int H, int Aout);
+size_t tc_weight_elems(int D, int H);
+cudaError_t launch_pack_tc_weights(const float* blob, uint16_t* dst, int D, int H, int A, int value_head, cudaStream_t s);
+cudaError_t launch_tc_mlp(const TcMlpParams& p, int sm_count, cudaStream_t s);
+cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
+                             const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
+                             cudaStream_t s);
+cudaError_t launch_td_finish(const float* partial, int n_partial, int n, float* loss_out, cudaStream_t s);
 
 // launchers (each returns the cudaGetLastError() of its launches)
 cudaError_t launch_init_env(int env_kind, int N, int S_d, uint2 seed, float* state, int* ep_step, float* ep_return,
@@ -158,6 +177,13 @@ struct tj_ctx {
   float* lgAt;
   float* lgB;
   float* lg_stage;
+  // tensor-core path (BF16 weights, supported shapes only)
+  bool use_tc;
+  int sm_count;
+  uint16_t* wtc[2];
+  uint16_t* wtc_target;
+  float* logits_buf;   // [N][A]
+  float* tdq[2];       // [kMaxTcTdRows][A] online / target outputs
   float *seg_obs, *seg_rew, *seg_logp, *seg_val;
   int* seg_act;
   uint8_t* seg_done;

@@ -371,6 +371,11 @@ cudaError_t launch_td_static(const TdParams& p_in, cudaStream_t s, bool* too_lar
   return launch_td(p, s);
 }
 
+cudaError_t launch_td_finish(const float* partial, int n_partial, int n, float* loss_out, cudaStream_t s) {
+  td_finish_kernel<<<1, 32, 0, s>>>(partial, n_partial, n, loss_out);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
                        float* adv, float* ret, cudaStream_t s) {
   gae_kernel<<<(N + 127) / 128, 128, 0, s>>>(rew, val, done, T, N, gamma, lambda, adv, ret);

@@ -1,0 +1,360 @@
+// BF16 tensor-core policy MLP (tcgen05.mma with TMEM accumulators) for wide networks.
+//
+//   out[n][A] = W3 relu(W2 relu(W1 x + b1) + b2) + b3     x: [n][D] FP32 rows,  weights BF16, accumulation FP32
+//
+// One thread block owns a tile of 128 rows (one row per TMEM lane) and walks tiles persistently.  Roles:
+//   warp 0, one lane   producer: streams pre-tiled BF16 weight chunks from global/L2 into a shared-memory ring with
+//                      bulk async copies (mbarrier complete_tx)
+//   warp 1, one lane   issues tcgen05.mma (M = 128, N <= 256, K = 16) over the ring; tcgen05.commit frees ring
+//                      slots and signals "accumulator full"
+//   warps 2-5          (128 threads, thread = row) convert the FP32 input rows to BF16 into the A-operand buffer;
+//                      after each layer read the accumulator from TMEM (tcgen05.ld), add the bias, apply ReLU,
+//                      round to BF16 and write the next layer's A operand; after the last layer write the outputs
+// Operands use the no-swizzle K-major core-matrix layout: 8 rows x 16 bytes are contiguous (128 B), cores adjacent
+// in K are 128 B apart (leading byte offset), groups of 8 rows are (K/8)*128 B apart (stride byte offset).
+// Every wait is bounded: on a timeout the block raises an abort flag, records an error, frees its TMEM and leaves.
+#include "tj_async.cuh"
+#include "tj_internal.h"
+
+namespace tj {
+
+namespace {
+
+constexpr int TC_M = 128;        // rows per tile
+constexpr int TC_KC = 32;        // K elements per weight chunk
+constexpr int TC_STAGES = 4;     // ring slots
+constexpr int TC_STAGE_BYTES = 256 * TC_KC * 2;   // largest chunk: 256 output rows
+constexpr int TC_THREADS = 192;
+constexpr int TC_N3 = 16;        // head width on the tensor cores (outputs padded to 16)
+
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  return d;                 // base offset 0, no swizzle
+}
+
+// D = F32, A = B = BF16, both K-major, M = 128
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// bounded wait that also gives up as soon as another role has raised the abort flag
+__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < (1 << 22); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  // round to nearest even; inputs are finite
+  uint32_t a = __float_as_uint(lo), b = __float_as_uint(hi);
+  a += 0x7FFFu + ((a >> 16) & 1u);
+  b += 0x7FFFu + ((b >> 16) & 1u);
+  return (a >> 16) | (b & 0xFFFF0000u);
+}
+
+struct TcSmem {
+  uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int D = p.D, H = p.H;
+  const int Kmax = D > H ? D : H;
+  uint8_t* abuf = smem_raw;                                          // [128][Kmax] bf16, core-matrix layout
+  uint8_t* ring = abuf + (size_t)TC_M * Kmax * 2;                    // TC_STAGES x TC_STAGE_BYTES
+  float* bias = reinterpret_cast<float*>(ring + TC_STAGES * TC_STAGE_BYTES);   // b1 [H], b2 [H], b3 [16]
+  TcSmem* ctl = reinterpret_cast<TcSmem*>(bias + 2 * H + TC_N3);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_tiles = (p.n + TC_M - 1) / TC_M;
+  const int n_blocks = H > 256 ? 2 : 1, NB = H / n_blocks;           // output-neuron blocks per hidden layer
+
+  if (tid == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    mbar_init(&ctl->a_ready, 128);
+    mbar_init(&ctl->acc_full, 1);
+    ctl->abort_flag = 0;
+  }
+  for (int i = tid; i < 2 * H + TC_N3; i += TC_THREADS) {
+    float v;
+    if (i < H) v = p.b1[i];
+    else if (i < 2 * H) v = p.b2[i - H];
+    else v = (i - 2 * H) < p.Aout ? p.b3[i - 2 * H] : 0.f;
+    bias[i] = v;
+  }
+  __syncthreads();
+  if (warp == 1) {   // one warp allocates all 512 TMEM columns (one block per SM) and publishes the base address
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&ctl->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  // chunk schedule of one tile, the same for producer and MMA issuer:
+  //   layer 1: n_blocks x (D/KC) chunks of NB rows; layer 2: n_blocks x (H/KC) chunks of NB rows;
+  //   layer 3: (H/KC) chunks of 16 rows
+  const int c1 = n_blocks * (D / TC_KC), c2 = n_blocks * (H / TC_KC), c3 = H / TC_KC;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer
+    uint32_t it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(p.wtc);
+      for (int c = 0; c < c1 + c2 + c3; ++c, ++it) {
+        const uint32_t bytes = (c < c1 + c2 ? NB : TC_N3) * TC_KC * 2;
+        const int s = it % TC_STAGES;
+        if (!tc_wait(&ctl->empty[s], ((it / TC_STAGES) & 1) ^ 1, abort_flag)) goto done;
+        mbar_expect_tx(&ctl->full[s], bytes);
+        bulk_copy_g2s(ring + (size_t)s * TC_STAGE_BYTES, src, bytes, &ctl->full[s]);
+        src += bytes;
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    uint32_t it = 0, layer_count = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      for (int layer = 0; layer < 3; ++layer, ++layer_count) {
+        const int K = layer == 0 ? D : H;
+        const int nb_count = layer == 2 ? 1 : n_blocks;
+        const int rows = layer == 2 ? TC_N3 : NB;
+        const uint32_t idesc = make_idesc(rows);
+        const uint32_t a_sbo = (uint32_t)(K / 8) * 128u, b_sbo = (uint32_t)(TC_KC / 8) * 128u;
+        if (!tc_wait(&ctl->a_ready, layer_count & 1, abort_flag)) goto done;
+        tc_fence_after();
+        for (int nb = 0; nb < nb_count; ++nb) {
+          for (int kc = 0; kc < K / TC_KC; ++kc, ++it) {
+            const int s = it % TC_STAGES;
+            if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
+            tc_fence_after();
+            const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
+            const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 8)) * 128u;
+#pragma unroll
+            for (int j = 0; j < TC_KC / 16; ++j) {
+              umma_bf16(tmem + (uint32_t)(nb * NB), make_desc(a_base + j * 256u, 128u, a_sbo),
+                        make_desc(b_base + j * 256u, 128u, b_sbo), idesc, (kc | j) != 0);
+            }
+            umma_commit(&ctl->empty[s]);    // the slot is free once these MMAs have read it
+          }
+        }
+        umma_commit(&ctl->acc_full);        // accumulator of this layer complete
+      }
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ operand conversion and epilogues
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int r = q * 32 + lane;                  // row of the tile = TMEM lane
+    const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
+    uint32_t layer_count = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      const long long row = (long long)tile * TC_M + r;
+      const bool live = row < p.n;
+      // layer-1 A operand: this row of x, FP32 -> BF16, 8 elements (16 bytes) at a time
+      {
+        const float* xr = p.x + (size_t)(live ? row : 0) * D;
+        uint8_t* dst = abuf + ((size_t)(r >> 3) * (D / 8)) * 128 + (r & 7) * 16;
+        for (int kg = 0; kg < D / 8; ++kg) {
+          float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+          if (live) {
+            lo = __ldg(reinterpret_cast<const float4*>(xr + kg * 8));
+            hi = __ldg(reinterpret_cast<const float4*>(xr + kg * 8 + 4));
+          }
+          uint4 v;
+          v.x = pack_bf16x2(lo.x, lo.y); v.y = pack_bf16x2(lo.z, lo.w);
+          v.z = pack_bf16x2(hi.x, hi.y); v.w = pack_bf16x2(hi.z, hi.w);
+          *reinterpret_cast<uint4*>(dst + (size_t)kg * 128) = v;
+        }
+      }
+      fence_async_smem();
+      mbar_arrive(&ctl->a_ready);
+      for (int layer = 0; layer < 3; ++layer, ++layer_count) {
+        if (!tc_wait(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
+        tc_fence_after();
+        if (layer < 2) {
+          // h = relu(acc + b) -> BF16 -> A operand of the next layer (K = H)
+          const float* b = bias + layer * H;
+          uint8_t* dst = abuf + ((size_t)(r >> 3) * (H / 8)) * 128 + (r & 7) * 16;
+          for (int c0 = 0; c0 < H; c0 += 16) {
+            uint32_t v[16];
+            tmem_ld16(t_lane + (uint32_t)c0, v);
+            tmem_ld_wait();
+            float f[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + b[c0 + j], 0.f);
+            uint4 o0, o1;
+            o0.x = pack_bf16x2(f[0], f[1]); o0.y = pack_bf16x2(f[2], f[3]);
+            o0.z = pack_bf16x2(f[4], f[5]); o0.w = pack_bf16x2(f[6], f[7]);
+            o1.x = pack_bf16x2(f[8], f[9]); o1.y = pack_bf16x2(f[10], f[11]);
+            o1.z = pack_bf16x2(f[12], f[13]); o1.w = pack_bf16x2(f[14], f[15]);
+            *reinterpret_cast<uint4*>(dst + (size_t)(c0 / 8) * 128) = o0;
+            *reinterpret_cast<uint4*>(dst + (size_t)(c0 / 8 + 1) * 128) = o1;
+          }
+          tc_fence_before();
+          fence_async_smem();
+          mbar_arrive(&ctl->a_ready);
+        } else {
+          uint32_t v[16];
+          tmem_ld16(t_lane, v);
+          tmem_ld_wait();
+          tc_fence_before();
+          if (live) {
+            float* o = p.out + (size_t)row * p.Aout;
+            for (int j = 0; j < p.Aout; ++j) o[j] = __uint_as_float(v[j]) + bias[2 * H + j];
+          }
+        }
+      }
+    }
+  }
+done:
+  __syncthreads();
+  if (tid == 0 && ctl->abort_flag) atomicExch(p.error, 2ull);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// FP32 blob -> BF16 chunks in the order the producer streams them; within a chunk of R rows x KC columns
+// element (r, k) sits at ((r/8) * (KC/8) + k/8) * 64 + (r%8) * 8 + k%8.
+__global__ void pack_tc_weights_kernel(const float* __restrict__ blob, uint16_t* __restrict__ dst, int D, int H, int A,
+                                       int value_head) {
+  const int n_blocks = H > 256 ? 2 : 1, NB = H / n_blocks;
+  const size_t n1 = (size_t)H * D, n2 = (size_t)H * H, n3 = (size_t)TC_N3 * H;
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n1 + n2 + n3) return;
+  const float* W1 = blob;
+  const float* W2 = W1 + n1 + H;
+  const float* W3 = W2 + n2 + H;
+  const float* Wv = W3 + (size_t)A * H + A;
+  size_t j = i;
+  const float* W;
+  int K, R, rows_total, n_off;
+  if (j < n1) { W = W1; K = D; R = NB; rows_total = H; }
+  else if (j < n1 + n2) { j -= n1; W = W2; K = H; R = NB; rows_total = H; }
+  else { j -= n1 + n2; W = W3; K = H; R = TC_N3; rows_total = A; }
+  const size_t chunk_elems = (size_t)R * TC_KC;
+  const size_t chunk = j / chunk_elems, within = j % chunk_elems;
+  const int chunks_per_block = K / TC_KC;
+  const int nb = (int)(chunk / chunks_per_block), kc = (int)(chunk % chunks_per_block);
+  n_off = nb * R;
+  const int core = (int)(within / 64), in_core = (int)(within % 64);
+  const int rg = core / (TC_KC / 8), kg = core % (TC_KC / 8);
+  const int r = rg * 8 + in_core / 8, k = kc * TC_KC + kg * 8 + in_core % 8;
+  const int n = n_off + r;
+  float v = 0.f;
+  if (n < rows_total) v = W[(size_t)n * K + k];
+  else if (W == W3 && value_head && n == A) v = Wv[k];
+  uint32_t u = __float_as_uint(v);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  dst[i] = (uint16_t)(u >> 16);
+}
+
+// TD error from precomputed Q rows: q = Qo[j][act], q' = max_a Qt[j][a]; per-block partial sums of the Huber loss
+__global__ void td_from_q_kernel(const float* __restrict__ q_online, const float* __restrict__ q_target, int n, int A,
+                                 const int* __restrict__ act, const float* __restrict__ rew,
+                                 const int* __restrict__ done, float gamma, float kappa, float* __restrict__ td_out,
+                                 float* __restrict__ huber_out, float* __restrict__ partial) {
+  __shared__ float hub[16];
+  const int j = blockIdx.x * 16 + threadIdx.x;
+  float h = 0.f;
+  if (threadIdx.x < 16 && j < n) {
+    int a = act[j];
+    a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+    const float q = q_online[(size_t)j * A + a];
+    float qmax = q_target[(size_t)j * A];
+    for (int i = 1; i < A; ++i) qmax = fmaxf(qmax, q_target[(size_t)j * A + i]);
+    const float y = rew[j] + gamma * (done[j] ? 0.f : 1.f) * qmax;
+    const float delta = y - q, ad = fabsf(delta);
+    h = ad <= kappa ? 0.5f * delta * delta : kappa * (ad - 0.5f * kappa);
+    if (td_out) td_out[j] = delta;
+    if (huber_out) huber_out[j] = h;
+  }
+  if (threadIdx.x < 16) hub[threadIdx.x] = h;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float sum = 0.f;
+    for (int i = 0; i < 16; ++i) sum += hub[i];
+    partial[blockIdx.x] = sum;
+  }
+}
+
+}  // namespace
+
+bool tc_mlp_supported(int D, int H, int Aout) {
+  if (D % TC_KC || H % TC_KC || D < TC_KC || H < TC_KC || H > 512 || D > 512 || Aout > TC_N3) return false;
+  const int n_blocks = H > 256 ? 2 : 1;
+  return (H / n_blocks) % 16 == 0;
+}
+
+size_t tc_weight_elems(int D, int H) { return (size_t)H * D + (size_t)H * H + (size_t)TC_N3 * H; }
+
+cudaError_t launch_pack_tc_weights(const float* blob, uint16_t* dst, int D, int H, int A, int value_head, cudaStream_t s) {
+  const size_t n = tc_weight_elems(D, H);
+  pack_tc_weights_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(blob, dst, D, H, A, value_head);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_tc_mlp(const TcMlpParams& p, int sm_count, cudaStream_t s) {
+  if (p.n <= 0) return cudaSuccess;
+  const int Kmax = p.D > p.H ? p.D : p.H;
+  const size_t smem = (size_t)TC_M * Kmax * 2 + (size_t)TC_STAGES * TC_STAGE_BYTES + (size_t)(2 * p.H + TC_N3) * 4 +
+                      sizeof(TcSmem) + 64;
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  cudaError_t e = cudaFuncSetAttribute(mlp_bf16_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const int n_tiles = (p.n + TC_M - 1) / TC_M;
+  const int grid = n_tiles < sm_count ? n_tiles : sm_count;
+  mlp_bf16_tc_kernel<<<grid, TC_THREADS, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
+                             const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
+                             cudaStream_t s) {
+  td_from_q_kernel<<<(n + 15) / 16, 32, 0, s>>>(q_online, q_target, n, A, act, rew, done, gamma, kappa, td_out, huber_out,
+                                                partial);
+  return cudaGetLastError();
+}
+
+}  // namespace tj

@@ -390,3 +390,42 @@ def test_categorical_actions_follow_the_margin_rule(env):
     same = g_act == o_acts
     close(gseg["logp"].cpu().numpy()[same], o_logp[same], RTOL_FP32, "logp")
     assert len(np.unique(g_act)) == 3
+
+
+# ------------------------------------------------------------------------------------------------ tensor cores
+@pytest.mark.parametrize("D,H,A,N", [(128, 512, 16, 300), (64, 64, 5, 130), (128, 320, 16, 128), (32, 256, 16, 257)])
+def test_bf16_tensor_core_actor_lockstep(env, D, H, A, N):
+    """BF16 weights on the tcgen05 path: network outputs within 2e-2 of the oracle (BF16-rounded weights, double
+    accumulation), actions exact outside the oracle's top-2 margin, the selection rule exact on the GPU's own
+    outputs, env step / ring / reset as in FP32."""
+    torch, orc, binding = env
+    f = _small(env_kind=2, obs_dim=D, n_actions=A, hidden=H, n_envs=N, replay_capacity=N * 4, warmup=N, weight_dtype=1,
+               max_episode_steps=5, lg_done_norm=0.75 * np.sqrt(D), minibatch=200, staleness_bound=10)
+    ctx, o = make_pair(orc, binding, **f)
+    tally = Tally()
+    for t in range(12):
+        if t % 5 == 0:
+            blob = blob_for(f, t // 5 + 1)
+            ctx.publish_weights(blob)
+            o.publish(blob)
+        r = lockstep_step(ctx, o, torch, rtol=2e-2, env_kind=2, tally=tally, logits_exact=False)
+        scale = float(np.sqrt(np.mean(r["o_logits"].astype(np.float64) ** 2)))
+        compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=2, tally=tally, act_exact=False, act_margin_scale=8 * 2e-2 * scale)
+    assert ctx.stats()["device_error"] == 0 and ctx.stats()["episodes_finished"] > 0
+    assert tally.ambiguous_act < 0.6 * tally.total          # the margin rule must still bind most decisions
+    # TD error through the same tensor-core forward
+    _, batch = ctx.replay_sample()
+    out = ctx.td_error(batch)
+    rec = np.zeros((200, 2 * D + 4), np.float32)
+    rec[:, :D] = batch["obs"].cpu().numpy()
+    rec[:, D:2 * D] = batch["next_obs"].cpu().numpy()
+    rec.view(np.int32)[:, 2 * D] = batch["act"].cpu().numpy()
+    rec[:, 2 * D + 1] = batch["rew"].cpu().numpy()
+    rec.view(np.int32)[:, 2 * D + 2] = batch["done"].cpu().numpy()
+    st, td, hub, loss, qs, qn = o.td(rec)
+    assert st == 0
+    g_td = out["td"].cpu().numpy().astype(np.float64)
+    q_scale = np.sqrt(np.mean(qs ** 2) + np.mean(qn ** 2))
+    assert np.all(np.abs(g_td - td) <= 2e-2 * (np.abs(qs) + np.abs(qn) + 2 * q_scale))
+    assert abs(float(out["loss"].item()) - loss) <= 4e-2 * (abs(loss) + q_scale)
+    assert ctx.stats()["device_error"] == 0
