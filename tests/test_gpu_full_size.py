@@ -1,0 +1,250 @@
+"""Full-size workloads in the launch configuration bench.py times (several actor steps per call, then a learner
+step and a publish).  The oracle cannot run these sizes, so every check is either on sampled environments and
+samples, recomputed one by one from the oracle's building blocks, or a property that holds at any size:
+records are self-contained (obs, action, reward, next_obs, done, version), consecutive records of one env chain
+(next_obs -> obs, or a reset drawn from Philox), the sampler's indices follow from the version tags, every sampled
+batch respects the staleness bound, gathers are bit-exact copies, counters add up.
+"""
+import numpy as np
+import pytest
+
+from parity_util import RTOL_FP32, blob_for, close, fields_for
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import oracle
+    from paper_2502_20190_b200 import binding, build
+    build.build()
+    oracle.build()
+    return torch, oracle, binding
+
+
+def _uniform(orc, x, lo, width):
+    return np.float32(np.float64(orc.u01(int(x))) * np.float64(np.float32(width)) + np.float64(np.float32(lo)))
+
+
+def _bf16_round(x):
+    """FP32 -> nearest bfloat16 (ties to even), returned as FP32."""
+    u = np.ascontiguousarray(x, np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
+def _check_ring_records(orc, f, blobs_by_version, recs, t_of_row, envs, rtol_logits, exact_logits):
+    """recs[i][j]: record of sampled env envs[j] written at actor step t_of_row[i].  CartPole / LinGauss only
+    (their observation is the state, so a record determines the whole step)."""
+    D, H, A = f["obs_dim"], f["hidden"], f["n_actions"]
+    thr = orc.explore_threshold(f["epsilon"])
+    kind = f["env_kind"]
+    n_amb = 0
+    for i, t in enumerate(t_of_row):
+        for j, e in enumerate(envs):
+            rec = recs[i][j]
+            ri = rec.view(np.int32)
+            obs, nxt = rec[:D], rec[D:2 * D]
+            a, rew, done, ver = int(ri[2 * D]), float(rec[2 * D + 1]), int(ri[2 * D + 2]), int(ri[2 * D + 3])
+            blob = blobs_by_version[ver]
+            w = orc.stream_words(f["seed"], orc.STREAM_ACTION, 0, int(e), int(t))
+            if f["weight_dtype"] == 0:
+                q = orc.mlp_forward(blob, D, H, A, obs)
+                assert a == orc.select_eps_greedy(q, w[0], w[1], thr)          # same FMA order: exact
+            else:
+                rb = blob.copy()
+                o0 = 0
+                for n_out, n_in in ((H, D), (H, H), (A, H)):
+                    rb[o0:o0 + n_out * n_in] = _bf16_round(rb[o0:o0 + n_out * n_in])
+                    o0 += n_out * n_in + n_out
+                q = orc.mlp_forward(rb, D, H, A, obs, f64=True).astype(np.float32)
+                explore = int(w[0]) < thr
+                top = np.sort(q)[::-1]
+                if explore or top[0] - top[1] > 8 * rtol_logits * float(np.sqrt(np.mean(q * q))):
+                    assert a == orc.select_eps_greedy(q, w[0], w[1], thr)
+                else:
+                    n_amb += 1
+            if kind == 0:
+                sn, r, term, margin = orc.cartpole_step(obs, a)
+            else:
+                noise = np.concatenate([orc.normal4(orc.stream_words(f["seed"], orc.STREAM_NOISE, b, int(e), int(t)))
+                                        for b in range(D // 4)])
+                sn, r, term, margin = orc.lingauss_step(obs, a, f["lg_A"], f["lg_B"], noise, f.get("lg_noise_std", 0.01),
+                                                        f.get("lg_done_norm", 4.0))
+            close(nxt, sn, RTOL_FP32, "next_obs")
+            assert abs(rew - r) <= RTOL_FP32 * (abs(r) + 1.0)
+            if margin > 8 * RTOL_FP32 and not done:
+                assert term == 0
+            if margin > 8 * RTOL_FP32 and term:
+                assert done == 1
+            # chaining: the next record's obs is this record's next_obs, or a fresh Philox draw after a done
+            if i + 1 < len(t_of_row) and t_of_row[i + 1] == t + 1:
+                nobs = recs[i + 1][j][:D]
+                if done:
+                    lo, wd = (-0.05, 0.1) if kind == 0 else (-0.1, 0.2)
+                    want = np.concatenate([[_uniform(orc, x, lo, wd) for x in
+                                            orc.stream_words(f["seed"], orc.STREAM_RESET, b, int(e), int(t))]
+                                           for b in range(D // 4)]).astype(np.float32)
+                    assert np.array_equal(nobs, want)
+                else:
+                    assert np.array_equal(nobs, nxt)
+    return n_amb
+
+
+def _run_ring_workload(env, name, n_iters, sample_envs):
+    torch, orc, binding = env
+    f = fields_for(name)
+    ctx = binding.Context(**f)
+    N, D, C_, B, S = f["n_envs"], f["obs_dim"], f["replay_capacity"], f["minibatch"], f["staleness_bound"]
+    rng = np.random.default_rng(5)
+    envs = np.unique(np.concatenate([[0, N - 1, 31, 32], rng.integers(0, N, sample_envs)]))
+    blobs = {}
+    batch = ctx.alloc_batch()
+    ring, block_ver = ctx.ring_view()
+    a_steps = 4
+    for it in range(n_iters):
+        v = it + 1
+        blobs[v] = blob_for(f, v)
+        assert ctx.publish_weights(blobs[v]) == v
+        cursor0, t0 = ctx.get_state()["cursor"], ctx.get_state()["t"]
+        ctx.actor_step(a_steps)
+        st, _ = ctx.replay_sample(batch=batch, allow=(0, -6, -7))
+        assert st == 0
+        # the sampler at full scale: staleness invariant, bit-exact gather, indices from the version tags
+        idx = batch["idx"].cpu().numpy()
+        ver = batch["ver"].cpu().numpy()
+        assert np.all(v - ver <= S) and np.all(ver >= 1)
+        valid = min(ctx.get_state()["cursor"], C_)
+        bv = block_ver[:valid // N].cpu().numpy()
+        elig = np.nonzero(v - bv <= S)[0]
+        k = ctx.get_state()["k"] - 1
+        for j in (0, 1, B // 2, B - 1):
+            x0 = int(orc.stream_words(f["seed"], orc.STREAM_SAMPLE, 0, j, k)[0])
+            r = (x0 * (len(elig) * N)) >> 32
+            assert idx[j] == elig[r // N] * N + r % N
+        rows = ring[batch["idx"][:64].long()].cpu().numpy()
+        assert np.array_equal(batch["obs"][:64].cpu().numpy(), rows[:, :D])
+        assert np.array_equal(batch["next_obs"][:64].cpu().numpy(), rows[:, D:2 * D])
+        assert np.array_equal(batch["ver"][:64].cpu().numpy(), rows.view(np.int32)[:, 2 * D + 3])
+        out = ctx.td_error(batch)
+        assert torch.isfinite(out["loss"]).all() and torch.isfinite(out["td"]).all()
+        if it == n_iters - 1:
+            slots = [[(cursor0 + s * N + int(e)) % C_ for e in envs] for s in range(a_steps)]
+            recs = [ring[torch.tensor(sl, device="cuda")].cpu().numpy() for sl in slots]
+            last = dict(recs=recs, ts=[t0 + s for s in range(a_steps)], batch=batch, out=out, v=v)
+    s = ctx.stats()
+    assert s["produced"] == n_iters * a_steps * N and s["consumed"] == n_iters * B and s["device_error"] == 0
+    assert s["actor_steps"] == n_iters * a_steps and sum(s["staleness_hist"]) == s["consumed"]
+    assert s["max_sampled_staleness"] <= S
+    return ctx, f, blobs, envs, last
+
+
+def test_cfg2_full_size(env):
+    torch, orc, binding = env
+    ctx, f, blobs, envs, last = _run_ring_workload(env, "cfg2", n_iters=12, sample_envs=40)
+    _check_ring_records(orc, f, blobs, last["recs"], last["ts"], envs, RTOL_FP32, True)
+    # TD error of sampled rows, recomputed one by one
+    b, out = last["batch"], last["out"]
+    D = 4
+    o = orc.Oracle(**f)
+    o.publish(blobs[1])
+    for v in range(2, last["v"] + 1):
+        o.publish(blobs[v])          # same cadence: the target network stays at version 1 (refresh every 1000)
+    rec = np.zeros((64, 12), np.float32)
+    rec[:, :4] = b["obs"][:64].cpu().numpy()
+    rec[:, 4:8] = b["next_obs"][:64].cpu().numpy()
+    rec.view(np.int32)[:, 8] = b["act"][:64].cpu().numpy()
+    rec[:, 9] = b["rew"][:64].cpu().numpy()
+    rec.view(np.int32)[:, 10] = b["done"][:64].cpu().numpy()
+    _, td, hub, _, qs, qn = o.td(rec)
+    g = out["td"][:64].cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(g - td) <= RTOL_FP32 * (np.abs(td) + np.abs(qs) + np.abs(qn) + 1.0))
+
+
+def test_cfg3_full_size_single_step_from_state(env):
+    """Acrobot: the observation does not determine the state bit for bit, so sampled envs are checked from a
+    state snapshot taken before a single step, after the multi-step calls have run."""
+    torch, orc, binding = env
+    ctx, f, blobs, envs, last = _run_ring_workload(env, "cfg3", n_iters=6, sample_envs=30)
+    N, D, A, H, C_ = f["n_envs"], 6, 3, f["hidden"], f["replay_capacity"]
+    st = ctx.get_state()
+    s0 = st["state"][torch.tensor(envs, device="cuda")].cpu().numpy()
+    dbg = torch.empty((N, A), dtype=torch.float32, device="cuda")
+    ctx.actor_step(1, dbg)
+    ring, _ = ctx.ring_view()
+    slots = [(st["cursor"] + int(e)) % C_ for e in envs]
+    recs = ring[torch.tensor(slots, device="cuda")].cpu().numpy()
+    logits = dbg[torch.tensor(envs, device="cuda")].cpu().numpy()
+    blob = blobs[last["v"]]
+    thr = orc.explore_threshold(f["epsilon"])
+    for j, e in enumerate(envs):
+        obs = orc.acrobot_obs(s0[j])
+        q = orc.mlp_forward(blob, D, H, A, obs)
+        close(logits[j], q, RTOL_FP32, "logits")
+        w = orc.stream_words(f["seed"], orc.STREAM_ACTION, 0, int(e), int(st["t"]))
+        a = int(recs[j].view(np.int32)[2 * D])
+        assert a == orc.select_eps_greedy(logits[j], w[0], w[1], thr)
+        sn, r, term, margin = orc.acrobot_step(s0[j], a)
+        close(recs[j][:D], obs, RTOL_FP32, "obs")
+        close(recs[j][D:2 * D], orc.acrobot_obs(sn), RTOL_FP32, "next_obs")
+        if margin > 1e-4:
+            assert float(recs[j][2 * D + 1]) == r
+
+
+def test_cfg5_full_size_tensor_core_path(env):
+    torch, orc, binding = env
+    ctx, f, blobs, envs, last = _run_ring_workload(env, "cfg5", n_iters=3, sample_envs=12)
+    n_amb = _check_ring_records(orc, f, blobs, last["recs"], last["ts"], envs, 2e-2, False)
+    assert n_amb < 0.5 * len(envs) * 4
+    s = ctx.stats()
+    # with the literal constants nearly every env terminates on every step
+    assert s["episodes_finished"] > 0.9 * s["produced"]
+
+
+def test_cfg4_full_size_segments_and_gae(env):
+    torch, orc, binding = env
+    f = fields_for("cfg4")
+    ctx = binding.Context(**f)
+    N, T, D, H, A = f["n_envs"], f["rollout_len"], 4, f["hidden"], 2
+    rng = np.random.default_rng(6)
+    envs = np.unique(np.concatenate([[0, N - 1], rng.integers(0, N, 10)]))
+    blobs = {}
+    for seg_i in range(2):
+        v = seg_i + 1
+        blobs[v] = blob_for(f, v)
+        ctx.publish_weights(blobs[v])
+        ctx.actor_step(T)
+        st, seg = ctx.segment_acquire()
+        assert st == 0 and seg["version"] == v
+        adv, ret = ctx.gae(seg["rew"], seg["val"], seg["done"], f["gamma"], f["gae_lambda"])
+        ei = torch.tensor(envs, device="cuda")
+        obs = seg["obs"][:, ei].cpu().numpy()
+        act = seg["act"][:, ei].cpu().numpy()
+        rew = seg["rew"][:, ei].cpu().numpy()
+        done = seg["done"][:, ei].cpu().numpy()
+        logp = seg["logp"][:, ei].cpu().numpy()
+        val = seg["val"][:, ei].cpu().numpy()
+        o_adv, o_ret = orc.gae(rew, val, done, f["gamma"], f["gae_lambda"])
+        close(adv[:, ei].cpu().numpy(), o_adv, RTOL_FP32, "adv")
+        close(ret[:, ei].cpu().numpy(), o_ret, RTOL_FP32, "ret")
+        n_amb = 0
+        for t in range(0, T, 9):
+            for j, e in enumerate(envs):
+                lg, v_ = orc.mlp_forward(blobs[v], D, H, A, obs[t, j], value_head=True)
+                assert val[t, j] == np.float32(v_)                       # same FMA order
+                u = orc.u01(int(orc.stream_words(f["seed"], orc.STREAM_ACTION, 0, int(e), seg_i * T + t)[0]))
+                a, lp, margin = orc.select_categorical(lg, u)
+                if margin > 8 * RTOL_FP32:
+                    assert act[t, j] == a and abs(logp[t, j] - lp) <= RTOL_FP32 * (abs(lp) + 1)
+                else:
+                    n_amb += 1
+                sn, r, term, m2 = orc.cartpole_step(obs[t, j], int(act[t, j]))
+                assert rew[t, j] == r
+                if t + 1 < T and not done[t, j]:
+                    close(obs[t + 1, j], sn, RTOL_FP32, "chained obs")
+        assert n_amb <= 2
+    s = ctx.stats()
+    assert s["produced"] == 2 * T * N and s["consumed"] == 2 * T * N and s["device_error"] == 0
