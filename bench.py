@@ -122,7 +122,6 @@ class Runner:
         self.dev_blobs = [torch.from_numpy(b).cuda() for b in blobs]
         self.host_blobs = [torch.from_numpy(b).pin_memory() for b in blobs]
         self.version = 0
-        self.launches = 0
         self.learner_ok = 0
         if not self.on_policy:
             self.batch = self.ctx.alloc_batch()
@@ -148,24 +147,20 @@ class Runner:
         else:
             self.ctx.publish_weights(blob)
         self.version += 1
-        self.launches += 1
 
     def actor(self):
         self.ctx.actor_step(self.actor_steps)
-        self.launches += 1
 
     def learner(self):
         if self.on_policy:
             st, seg = self.ctx.segment_acquire(allow=(0, -7))
             if st == 0:
                 self.ctx.gae(seg["rew"], seg["val"], seg["done"], self.w["gamma"], self.w["gae_lambda"], self.adv, self.ret)
-                self.launches += 1
                 self.learner_ok += 1
         else:
             st, _ = self.ctx.replay_sample(batch=self.batch, allow=(0, -6, -7))
             if st == 0:
                 self.ctx.td_error(self.batch, self.out)
-                self.launches += 4  # eligible list, sample+gather, TD, loss reduction
                 self.learner_ok += 1
 
     def step(self, events=None, e2e=False):
@@ -233,7 +228,7 @@ def run_ours(args):
 
     def timed_loop(K, e2e):
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-        r.launches = 0
+        launches0 = r.ctx.stats()["kernel_launches"]
         r.learner_ok = 0
         for i in range(K):
             if need_flush:
@@ -243,7 +238,7 @@ def run_ours(args):
         tot = sum(e[0].elapsed_time(e[3]) for e in evs)
         act = sum(e[0].elapsed_time(e[1]) for e in evs)
         lrn = sum(e[1].elapsed_time(e[2]) for e in evs)
-        return tot, act, lrn, r.launches, r.learner_ok
+        return tot, act, lrn, r.ctx.stats()["kernel_launches"] - launches0, r.learner_ok
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -256,6 +251,12 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     e2e_ms, _, _, _, _ = timed_loop(args.steps, True)
     barrier()
+    # the same K steps once more with the library's per-kernel CUDA events on: duration of each kernel class
+    r.ctx.set_profiling(1)
+    timed_loop(args.steps, False)
+    prof = r.ctx.stats()
+    r.ctx.set_profiling(0)
+    barrier()
 
     times = torch.tensor([tot_ms, e2e_ms, act_ms, lrn_ms], dtype=torch.float64, device="cuda")
     if world > 1:
@@ -266,18 +267,42 @@ def run_ours(args):
     consumed = (w["rollout_len"] * N if r.on_policy else w["minibatch"]) * learner_ok * world
     value = env_steps / (tot_ms * 1e-3)
     flops, nbytes = actor_algorithmic(w)
-    launch_s = act_ms * 1e-3 / K
-    units = N * r.actor_steps
-    if w["weight_dtype"] == synth.W_BF16:
-        bound, unit = "tensor", "TFLOP/s"
-        achieved = flops * units / launch_s / 1e12
-        peak = peaks["bf16_tflops_sustained"]
-        peak_note = "cuBLAS bf16 sustained, of " + peaks["source"]
-    else:
-        bound, unit = "alu", "TFLOP/s"
-        achieved = flops * units / launch_s / 1e12
-        peak = SM_COUNT * FMA_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-        peak_note = "FP32 FMA: 148 SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"
+    names = ["actor_fused", "mlp_tensor", "env_select_insert", "sample_gather", "td", "publish", "gae"]
+    kms, kcnt = prof["kernel_ms"], prof["kernel_count"]
+    total_kms = sum(kms) or 1.0
+    kernels = {names[i]: {"launches": kcnt[i], "ms": kms[i], "share": kms[i] / total_kms} for i in range(len(names)) if kcnt[i]}
+    dom = max(range(len(names)), key=lambda i: kms[i])
+    units = N * r.actor_steps                      # env-steps one actor call processes
+    fma_peak = SM_COUNT * FMA_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    mlp_flops = 2 * mlp_macs(w)
+    env_flops = flops - mlp_flops
+    S_d = w["obs_dim"] if w["env_kind"] == synth.ENV_LINGAUSS else 4
+    if dom == 1:      # tensor-core MLP: actor launches process N rows, learner launches B rows (two per step)
+        rows = K * (r.actor_steps * N + 2 * w["minibatch"])
+        achieved = mlp_flops * rows / (kms[1] * 1e-3) / 1e12
+        roof = {"kernel": "mlp_bf16_tc_kernel (tcgen05 MLP forward)", "bound": "tensor", "achieved": achieved,
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "peak_source": "cuBLAS bf16 sustained, of " + peaks["source"]}
+    elif dom == 2:    # selection + env step + insert: state read twice (obs) + written, record written, outputs read
+        per_env = 2 * S_d * 4 + 8 + (2 * w["obs_dim"] + 4) * 4 + w["n_actions"] * 4
+        gbs = per_env * units * K / (kms[2] * 1e-3) / 1e9
+        tfl = env_flops * units * K / (kms[2] * 1e-3) / 1e12
+        if gbs / peaks["hbm_gbs"] >= tfl / fma_peak:
+            roof = {"kernel": "actor_lingauss_kernel (selection + env step + insert)", "bound": "hbm", "achieved": gbs,
+                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_source": "copy bandwidth, of " + peaks["source"]}
+        else:
+            roof = {"kernel": "actor_lingauss_kernel (selection + env step + insert)", "bound": "alu", "achieved": tfl,
+                    "peak": fma_peak, "unit": "TFLOP/s",
+                    "peak_source": "FP32 FMA: 148 SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"}
+    else:             # fused FP32 actor kernel (or, for tiny workloads, whatever dominates: reported against it)
+        t_ms = kms[0] if kcnt[0] else act_ms
+        achieved = flops * units * K / (t_ms * 1e-3) / 1e12
+        roof = {"kernel": "actor_small_env_kernel (MLP + selection + env step + insert)", "bound": "alu",
+                "achieved": achieved, "peak": fma_peak, "unit": "TFLOP/s",
+                "peak_source": "FP32 FMA: 148 SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["step_hbm_frac_of_measured"] = nbytes * units / (act_ms * 1e-3 / K) / 1e9 / peaks["hbm_gbs"]
     h2d, d2h = r.e2e_bytes()
     line = {
         "metric": "env-steps/s", "value": value, "unit": "env-steps/s", "n_gpus": world, "steps": K,
@@ -293,9 +318,8 @@ def run_ours(args):
         "e2e": {"value": env_steps / (e2e_ms * 1e-3), "unit": "env-steps/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
-        "roofline": {"kernel": "actor step (policy MLP + env + ring insert)", "bound": bound, "achieved": achieved,
-                     "peak": peak, "unit": unit, "frac": achieved / peak, "traffic": None, "peak_source": peak_note,
-                     "hbm_frac_of_measured": nbytes * units / launch_s / 1e9 / peaks["hbm_gbs"]},
+        "roofline": roof,
+        "kernels": kernels,
         "clocks": clocks,
     }
     if rank == 0:
@@ -408,7 +432,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="cfg2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--workload", default="cfg5", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

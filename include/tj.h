@@ -60,6 +60,14 @@ typedef enum {
 enum { TJ_ENV_CARTPOLE = 0, TJ_ENV_ACROBOT = 1, TJ_ENV_LINGAUSS = 2 };
 enum { TJ_POLICY_EPS_GREEDY = 0, TJ_POLICY_CATEGORICAL = 1 };
 enum { TJ_W_FP32 = 0, TJ_W_BF16 = 1 };
+/* kernel classes reported by tj_stats (Sec. 3.3: performance analysis measures the production and the
+ * consumption side separately) */
+enum { TJ_K_ACTOR_FUSED = 0,  /* MLP + selection + env step + insert in one kernel (FP32 path) */
+       TJ_K_MLP_TENSOR = 1,   /* tensor-core MLP forward (actor or learner) */
+       TJ_K_ENV = 2,          /* selection + env step + insert fed by the tensor-core MLP */
+       TJ_K_SAMPLE = 3,       /* eligible list + sample + gather */
+       TJ_K_TD = 4,           /* TD error (FP32 forward, or the elementwise pass after tensor-core forwards) */
+       TJ_K_PUBLISH = 5, TJ_K_GAE = 6, TJ_KERNEL_CLASSES = 8 };
 
 /* Configuration (App. B: one configuration with distribution / training / model / environment groups). */
 typedef struct {
@@ -137,7 +145,12 @@ typedef struct {
   int64_t episodes_finished;
   double return_sum;            /* sum of the returns of finished episodes */
   int64_t staleness_hist[33];   /* sampled staleness 0..31, last bin = 32 and more */
-  int64_t device_error;         /* 0, or a code latched by a kernel's own bounds check */
+  int64_t device_error;         /* 0, or a code latched by a kernel's own bounded wait or bounds check */
+  int64_t kernel_launches;      /* kernels this context has launched since tj_create */
+  /* Per kernel class, filled while profiling is on (tj_set_profiling): launches timed and their summed
+   * duration in ms, from CUDA events recorded around each launch on the context's stream. */
+  int64_t kernel_count[TJ_KERNEL_CLASSES];
+  double kernel_ms[TJ_KERNEL_CLASSES];
 } tj_stats_t;
 
 /* Bytes (and alignment) of device memory a context with this configuration needs. */
@@ -225,6 +238,11 @@ int tj_set_state(tj_ctx *ctx, const tj_state_view *in);
 
 /* Counters (Eq. 2-3: produced vs consumed, sampled staleness).  Synchronises the stream. */
 int tj_stats(tj_ctx *ctx, tj_stats_t *host_out);
+
+/* Turn per-kernel timing on or off.  While on, every launch is bracketed by two CUDA events on the context's
+ * stream (a few microseconds of overhead per launch); tj_stats turns them into kernel_count / kernel_ms.
+ * Turning it on resets the per-class figures. */
+int tj_set_profiling(tj_ctx *ctx, int32_t on);
 
 /* Views into the ring for inspection: records [C][2D+4] (obs, next_obs, act, rew, done, ver as 32-bit words)
  * and the per-block version summary [C/N]. */

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
            "tj_last_error")
 
 
@@ -63,7 +63,8 @@ class TjStats(C.Structure):
                 ("dropped_overwritten", C.c_int64), ("starved_calls", C.c_int64), ("actor_version", C.c_int64),
                 ("learner_version", C.c_int64), ("actor_steps", C.c_int64), ("learner_steps", C.c_int64),
                 ("max_sampled_staleness", C.c_int64), ("episodes_finished", C.c_int64), ("return_sum", C.c_double),
-                ("staleness_hist", C.c_int64 * 33), ("device_error", C.c_int64)]
+                ("staleness_hist", C.c_int64 * 33), ("device_error", C.c_int64), ("kernel_launches", C.c_int64),
+                ("kernel_count", C.c_int64 * 8), ("kernel_ms", C.c_double * 8)]
 
 
 _lib = None
@@ -92,6 +93,7 @@ def load_library():
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
     L.tj_stats.argtypes = [vp, vp]
+    L.tj_set_profiling.argtypes = [vp, i32]
     L.tj_ring_view.argtypes = [vp, vp, vp, vp]
     L.tj_last_error.argtypes = [vp]
     L.tj_last_error.restype = C.c_char_p
@@ -172,6 +174,10 @@ def tj_stats(h):
     s = TjStats()
     st = load_library().tj_stats(h, C.byref(s))
     return st, s
+
+
+def tj_set_profiling(h, on: int):
+    return load_library().tj_set_profiling(h, int(on))
 
 
 def tj_ring_view(h):
@@ -354,9 +360,14 @@ class Context:
     def stats(self):
         st, s = tj_stats(self.h)
         self._check(st)
-        d = {k: getattr(s, k) for k, _ in TjStats._fields_ if k != "staleness_hist"}
-        d["staleness_hist"] = list(s.staleness_hist)
+        arrays = ("staleness_hist", "kernel_count", "kernel_ms")
+        d = {k: getattr(s, k) for k, _ in TjStats._fields_ if k not in arrays}
+        for k in arrays:
+            d[k] = list(getattr(s, k))
         return d
+
+    def set_profiling(self, on):
+        return self._check(tj_set_profiling(self.h, on))
 
     def ring_view(self):
         torch = self.torch

@@ -136,6 +136,43 @@ int cuda_fail(tj_ctx* x, cudaError_t e, const char* where) {
 
 thread_local std::string g_err;  // for failures before a context exists
 
+// Counts the launches made inside its scope and, while profiling is on, brackets them with two events.
+struct LaunchScope {
+  tj_ctx* x;
+  cudaEvent_t a = nullptr, b = nullptr;
+  int cls;
+  LaunchScope(tj_ctx* ctx, int kernel_class, int n_launches) : x(ctx), cls(kernel_class) {
+    x->hs.kernel_launches += n_launches;
+    if (!x->profiling) return;
+    a = take(); b = take();
+    if (a && b) cudaEventRecord(a, x->stream);
+  }
+  ~LaunchScope() {
+    if (!a || !b) return;
+    cudaEventRecord(b, x->stream);
+    x->spans.push_back({a, b, cls});
+  }
+  cudaEvent_t take() {
+    if (!x->ev_pool.empty()) { cudaEvent_t e = x->ev_pool.back(); x->ev_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    return cudaEventCreate(&e) == cudaSuccess ? e : nullptr;
+  }
+};
+
+// reads every finished span into the per-class totals; the stream must have been synchronised
+void drain_spans(tj_ctx* x) {
+  for (auto& sp : x->spans) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) {
+      x->hs.kernel_ms[sp.cls] += ms;
+      x->hs.kernel_count[sp.cls] += 1;
+    }
+    x->ev_pool.push_back(sp.a);
+    x->ev_pool.push_back(sp.b);
+  }
+  x->spans.clear();
+}
+
 uint64_t explore_threshold(float eps) {
   const double e = (double)eps;
   if (!(e > 0.0)) return 0;
@@ -180,7 +217,7 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
   x->n_blob = blob_floats(x->D, x->H, x->A, x->value_head);
   x->wl = make_weight_layout(x->D, x->H, x->A, x->value_head);
   x->active = 0; x->version = 0; x->k_last_sync = 0; x->has_target = false;
-  x->t = 0; x->k = 0; x->cursor = 0; x->next_consume = 0;
+  x->t = 0; x->k = 0; x->cursor = 0; x->next_consume = 0; x->profiling = false;
   std::memset(&x->hs, 0, sizeof(x->hs));
   if (cfg->replay_capacity > 0) x->h_block_ver.assign((size_t)(cfg->replay_capacity / cfg->n_envs), 0);
   else x->seg.assign((size_t)cfg->n_segments, SegSlot{});
@@ -224,7 +261,20 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
 int tj_destroy(tj_ctx* ctx) {
   if (!ctx) return TJ_ERR_INVALID_ARG;
   cudaStreamSynchronize(ctx->stream);
+  drain_spans(ctx);
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   delete ctx;
+  return TJ_OK;
+}
+
+int tj_set_profiling(tj_ctx* x, int32_t on) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (on && !x->profiling) {
+    cudaStreamSynchronize(x->stream);
+    drain_spans(x);
+    for (int i = 0; i < TJ_KERNEL_CLASSES; ++i) { x->hs.kernel_ms[i] = 0.0; x->hs.kernel_count[i] = 0; }
+  }
+  x->profiling = on != 0;
   return TJ_OK;
 }
 
@@ -239,6 +289,7 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
       return cuda_fail(x, e, "publish: host to device copy");
     src = x->blob_stage;
   }
+  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc ? 2 : 1);
   const int next = x->active ^ 1;
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
   if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->stream)) != cudaSuccess)
@@ -301,15 +352,20 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
       t.wtc = x->wtc[x->active];
       t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
       t.out = x->logits_buf; t.error = &x->dstats->error;
-      e = launch_tc_mlp(t, x->sm_count, x->stream);
+      {
+        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
+        e = launch_tc_mlp(t, x->sm_count, x->stream);
+      }
       if (e != cudaSuccess) break;
       ActorParams q = p;
       q.n_steps = 1; q.t0 = x->t + i; q.cursor0 = x->cursor + (uint64_t)i * x->N;
       q.logits_in = x->logits_buf;
       q.dbg_logits = dbg_logits ? dbg_logits + (size_t)i * x->N * x->A : nullptr;
+      LaunchScope scope(x, TJ_K_ENV, 1);
       e = launch_actor(c.env_kind, q, x->stream);
     }
   } else {
+    LaunchScope scope(x, TJ_K_ACTOR_FUSED, 1);
     e = launch_actor(c.env_kind, p, x->stream);
   }
   if (e != cudaSuccess) return cuda_fail(x, e, "actor step");
@@ -355,6 +411,7 @@ int tj_replay_sample(tj_ctx* x, int32_t staleness_bound, int32_t* idx_out, const
     return fail(x, TJ_ERR_STARVED, "no resident record within the staleness bound");
   }
   if ((uint64_t)n_elig * (uint64_t)x->N > 0xFFFFFFFFull) return fail(x, TJ_ERR_UNSUPPORTED, "eligible set too large");
+  LaunchScope scope(x, TJ_K_SAMPLE, 2);
   cudaError_t e = launch_eligible(x->block_ver, n_blocks, x->version, S, x->elig_list, x->elig_count, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "eligible list");
   SampleParams p{};
@@ -397,8 +454,10 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
       t.wtc = which == 0 ? x->wtc[x->active] : x->wtc_target;
       t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
       t.out = x->tdq[which]; t.error = &x->dstats->error;
+      LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
       if ((e = launch_tc_mlp(t, x->sm_count, x->stream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
     }
+    LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1);
     if ((e = launch_td_from_q(x->tdq[0], x->tdq[1], b->n, x->A, b->act, b->rew, b->done, p.gamma, p.kappa, td_out,
                               huber_out, x->td_partial, x->stream)) != cudaSuccess)
       return cuda_fail(x, e, "TD error (elementwise)");
@@ -406,6 +465,7 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
       return cuda_fail(x, e, "TD error (loss reduction)");
     return TJ_OK;
   }
+  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1);
   e = launch_td(p, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error");
   return TJ_OK;
@@ -426,6 +486,7 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = nullptr;
   bool too_large = false;
+  x->hs.kernel_launches += loss_mean_out ? 2 : 1;
   cudaError_t e = launch_td_static(p, x->stream, &too_large);
   if (too_large) {
     char msg[160];
@@ -443,6 +504,7 @@ int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, i
   if (!rew || !val || !done || !adv_out || !ret_out) return fail(x, TJ_ERR_INVALID_ARG, "GAE arrays must not be null");
   if (T < 0 || N < 0) return fail(x, TJ_ERR_INVALID_ARG, "T and N must not be negative");
   if (T == 0 || N == 0) return TJ_OK;
+  LaunchScope scope(x, TJ_K_GAE, 1);
   cudaError_t e = launch_gae(rew, val, done, T, N, gamma, lambda, adv_out, ret_out, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "GAE");
   return TJ_OK;
@@ -516,6 +578,7 @@ int tj_stats(tj_ctx* x, tj_stats_t* o) {
   cudaError_t e = cudaMemcpyAsync(&d, x->dstats, sizeof(d), cudaMemcpyDeviceToHost, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "read counters");
+  drain_spans(x);
   *o = x->hs;
   o->actor_version = o->learner_version = x->version;
   o->episodes_finished = (int64_t)d.episodes;

@@ -197,5 +197,9 @@ struct tj_ctx {
   std::vector<SegSlot> seg;
   int64_t next_consume;
   tj_stats_t hs;        // host-side counters
+  bool profiling;
+  std::vector<cudaEvent_t> ev_pool;                  // free events
+  struct Span { cudaEvent_t a, b; int cls; };
+  std::vector<Span> spans;                            // recorded, not yet read
   std::string err;
 };
