@@ -122,6 +122,11 @@ size_t carve(tj_ctx* x, void* base) {
     x->tdq[0] = cv.take<float>((size_t)kMaxTcTdRows * c.n_actions);
     x->tdq[1] = cv.take<float>((size_t)kMaxTcTdRows * c.n_actions);
   }
+  x->use_tc_fused = x->use_tc && c.env_kind == TJ_ENV_LINGAUSS && c.replay_capacity > 0 && tc_fused_supported(D, c.hidden, c.n_actions);
+  if (x->use_tc_fused) {
+    x->lgA_hi = cv.take<uint32_t>((size_t)D * D);
+    x->lgA_lo = cv.take<uint32_t>((size_t)D * D);
+  }
   return (cv.off + kAlign - 1) & ~(kAlign - 1);
 }
 
@@ -249,6 +254,8 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
     // B [A][D] is used as it is: D is a multiple of 4, so rows are already 16-byte aligned
     if ((e = cudaMemcpyAsync(x->lgB, stage + (size_t)D * D, sizeof(float) * A * D, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
       return bail(e, "copy B to its place");
+    if (x->use_tc_fused && (e = launch_pack_env_matrix(stage, x->lgA_hi, x->lgA_lo, D, x->stream)) != cudaSuccess)
+      return bail(e, "tile env matrix");
     if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e, "sync after LinGauss set-up");
   }
   const uint2 seed = make_uint2((uint32_t)cfg->seed, (uint32_t)(cfg->seed >> 32));
@@ -352,6 +359,20 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
       t.wtc = x->wtc[x->active];
       t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
       t.out = x->logits_buf; t.error = &x->dstats->error;
+      if (x->use_tc_fused) {
+        // one kernel per step: network, selection, A s on the tensor cores, env epilogue, insert
+        t.out = dbg_logits ? dbg_logits + (size_t)i * x->N * x->A : nullptr;
+        TcEnvParams& ev = t.env;
+        ev.fused = 1; ev.A = x->A; ev.max_ep = x->max_ep; ev.rec_words = x->rec_words; ev.version = (int)x->version;
+        ev.state = x->state; ev.ep_step = x->ep_step; ev.ep_return = x->ep_return;
+        ev.seed = p.seed; ev.explore_thr = p.explore_thr; ev.t = (unsigned long long)(x->t + i);
+        ev.ring = x->ring; ev.C = c.replay_capacity; ev.cursor = x->cursor + (uint64_t)i * x->N; ev.block_ver = x->block_ver;
+        ev.lgA_hi = x->lgA_hi; ev.lgA_lo = x->lgA_lo; ev.lgB = x->lgB;
+        ev.noise_std = c.lg_noise_std; ev.done_norm = c.lg_done_norm; ev.stats = x->dstats;
+        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
+        e = launch_tc_mlp(t, x->sm_count, x->stream);
+        continue;
+      }
       {
         LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
         e = launch_tc_mlp(t, x->sm_count, x->stream);

@@ -111,19 +111,40 @@ struct SampleParams {
   DevStats* stats;
 };
 
+struct TcEnvParams {
+  int fused;                 // 0: network only
+  int A, max_ep, rec_words, version;
+  float* state;
+  int* ep_step;
+  float* ep_return;
+  uint2 seed;
+  unsigned long long explore_thr, t;
+  float* ring;
+  long long C;
+  unsigned long long cursor;
+  int* block_ver;
+  const uint32_t *lgA_hi, *lgA_lo;   // env matrix, TF32 high / low parts, tiled
+  const float* lgB;                  // [A][D]
+  float noise_std, done_norm;
+  DevStats* stats;
+};
+
 struct TcMlpParams {
   const float* x;          // [n][D] FP32 rows
   int n, D, H, Aout;
   const uint16_t* wtc;     // BF16 weight chunks in streaming order
   const float *b1, *b2, *b3;
-  float* out;              // [n][Aout]
+  float* out;              // [n][Aout] (nullable in fused mode)
   unsigned long long* error;
+  TcEnvParams env;
 };
 
 bool tc_mlp_supported(int D, int H, int Aout);
 size_t tc_weight_elems(int D, int H);
 cudaError_t launch_pack_tc_weights(const float* blob, uint16_t* dst, int D, int H, int A, int value_head, cudaStream_t s);
 cudaError_t launch_tc_mlp(const TcMlpParams& p, int sm_count, cudaStream_t s);
+cudaError_t launch_pack_env_matrix(const float* A, uint32_t* hi, uint32_t* lo, int D, cudaStream_t s);
+bool tc_fused_supported(int D, int H, int A);
 cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
                              const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
                              cudaStream_t s);
@@ -183,6 +204,8 @@ struct tj_ctx {
   uint16_t* wtc[2];
   uint16_t* wtc_target;
   float* logits_buf;   // [N][A]
+  bool use_tc_fused;
+  uint32_t *lgA_hi, *lgA_lo;
   float* tdq[2];       // [kMaxTcTdRows][A] online / target outputs
   float *seg_obs, *seg_rew, *seg_logp, *seg_val;
   int* seg_act;

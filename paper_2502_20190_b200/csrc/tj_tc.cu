@@ -12,8 +12,14 @@
 //                      round to BF16 and write the next layer's A operand; after the last layer write the outputs
 // Operands use the no-swizzle K-major core-matrix layout: 8 rows x 16 bytes are contiguous (128 B), cores adjacent
 // in K are 128 B apart (leading byte offset), groups of 8 rows are (K/8)*128 B apart (stride byte offset).
+// Fused actor mode (linear-Gaussian env): after the head layer the same block selects the action (epsilon-greedy on the
+// accumulator row), re-reads the FP32 state row, writes it as the record's observation and splits it into TF32
+// high and low parts; A s then runs on the tensor cores as three TF32 products (hi*hi + lo*hi + hi*lo, FP32
+// accumulation, error ~2^-21 relative per term), and the epilogue threads finish the step: + B[a], tanh, Philox
+// noise, reward, done, record, reset, new state.
 // Every wait is bounded: on a timeout the block raises an abort flag, records an error, frees its TMEM and leaves.
 #include "tj_async.cuh"
+#include "tj_device.cuh"
 #include "tj_internal.h"
 
 namespace tj {
@@ -45,6 +51,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
+      : "memory");
+}
+
+// D = F32, A = B = TF32, both K-major, M = 128
+__device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
       : "memory");
 }
@@ -81,6 +100,12 @@ __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile
   return false;
 }
 
+// for whole warps (the epilogue warps run warp-wide TMEM loads): every lane waits, and the warp leaves together
+__device__ __forceinline__ bool tc_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = tc_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   // round to nearest even; inputs are finite
   uint32_t a = __float_as_uint(lo), b = __float_as_uint(hi);
@@ -89,18 +114,30 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return (a >> 16) | (b & 0xFFFF0000u);
 }
 
+// bytes of the A-operand buffer: the widest BF16 operand; in fused mode also the TF32 high+low state tile and
+// the FP32 staging rows of the stepped state
+__host__ __device__ inline size_t tc_abuf_bytes(int D, int H, bool fused) {
+  size_t n = (size_t)TC_M * (D > H ? D : H) * 2;
+  if (fused) {
+    const size_t hl = (size_t)2 * TC_M * D * 4, st = (size_t)TC_M * (D + 4) * 4;
+    if (hl > n) n = hl;
+    if (st > n) n = st;
+  }
+  return (n + 1023) & ~(size_t)1023;
+}
+
 struct TcSmem {
-  uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full;
+  uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full, rows_done;
   uint32_t tmem_base;
   int abort_flag;
 };
 
+template <bool FUSED>
 __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int D = p.D, H = p.H;
-  const int Kmax = D > H ? D : H;
   uint8_t* abuf = smem_raw;                                          // [128][Kmax] bf16, core-matrix layout
-  uint8_t* ring = abuf + (size_t)TC_M * Kmax * 2;                    // TC_STAGES x TC_STAGE_BYTES
+  uint8_t* ring = abuf + tc_abuf_bytes(D, H, FUSED);                 // TC_STAGES x TC_STAGE_BYTES
   float* bias = reinterpret_cast<float*>(ring + TC_STAGES * TC_STAGE_BYTES);   // b1 [H], b2 [H], b3 [16]
   TcSmem* ctl = reinterpret_cast<TcSmem*>(bias + 2 * H + TC_N3);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -111,6 +148,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
     mbar_init(&ctl->a_ready, 128);
     mbar_init(&ctl->acc_full, 1);
+    mbar_init(&ctl->rows_done, 128);
     ctl->abort_flag = 0;
   }
   for (int i = tid; i < 2 * H + TC_N3; i += TC_THREADS) {
@@ -135,6 +173,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
   //   layer 1: n_blocks x (D/KC) chunks of NB rows; layer 2: n_blocks x (H/KC) chunks of NB rows;
   //   layer 3: (H/KC) chunks of 16 rows
   const int c1 = n_blocks * (D / TC_KC), c2 = n_blocks * (H / TC_KC), c3 = H / TC_KC;
+  const int ce = D / TC_KC;   // fused mode: chunks of the env matrix per TF32 pass (three passes)
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ producer
@@ -148,6 +187,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         mbar_expect_tx(&ctl->full[s], bytes);
         bulk_copy_g2s(ring + (size_t)s * TC_STAGE_BYTES, src, bytes, &ctl->full[s]);
         src += bytes;
+      }
+      if (FUSED) {
+        const uint32_t bytes = (uint32_t)D * TC_KC * 4;
+        for (int c = 0; c < 3 * ce; ++c, ++it) {
+          const uint8_t* esrc = reinterpret_cast<const uint8_t*>(c < 2 * ce ? p.env.lgA_hi : p.env.lgA_lo) + (size_t)(c % ce) * bytes;
+          const int s = it % TC_STAGES;
+          if (!tc_wait(&ctl->empty[s], ((it / TC_STAGES) & 1) ^ 1, abort_flag)) goto done;
+          mbar_expect_tx(&ctl->full[s], bytes);
+          bulk_copy_g2s(ring + (size_t)s * TC_STAGE_BYTES, esrc, bytes, &ctl->full[s]);
+        }
       }
     }
   } else if (warp == 1 && lane == 0) {
@@ -179,6 +228,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         }
         umma_commit(&ctl->acc_full);        // accumulator of this layer complete
       }
+      if (FUSED) {
+        // z = A s as three TF32 products: (s_hi, A_hi), (s_lo, A_hi), (s_hi, A_lo)
+        const uint32_t idesc = make_idesc_tf32(D);
+        const uint32_t a_sbo = (uint32_t)(D / 4) * 128u, b_sbo = (uint32_t)(TC_KC / 4) * 128u;
+        const uint32_t lo_off = (uint32_t)TC_M * D * 4;
+        if (!tc_wait(&ctl->a_ready, layer_count & 1, abort_flag)) goto done;
+        tc_fence_after();
+        for (int pass = 0; pass < 3; ++pass) {
+          for (int kc = 0; kc < ce; ++kc, ++it) {
+            const int s = it % TC_STAGES;
+            if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
+            tc_fence_after();
+            const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
+            const uint32_t a_base = smem_addr(abuf) + (pass == 1 ? lo_off : 0u) + (uint32_t)(kc * (TC_KC / 4)) * 128u;
+#pragma unroll
+            for (int j = 0; j < TC_KC / 8; ++j) {
+              umma_tf32(tmem, make_desc(a_base + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, b_sbo), idesc,
+                        (pass | kc | j) != 0);
+            }
+            umma_commit(&ctl->empty[s]);
+          }
+        }
+        umma_commit(&ctl->acc_full);
+        ++layer_count;
+      }
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ operand conversion and epilogues
@@ -186,6 +260,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     const int r = q * 32 + lane;                  // row of the tile = TMEM lane
     const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
     uint32_t layer_count = 0;
+    int action = 0;
+    uint32_t tiles_done = 0;
+    unsigned long long n_episodes = 0;
+    double ret_sum = 0.0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const long long row = (long long)tile * TC_M + r;
       const bool live = row < p.n;
@@ -208,7 +286,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
       fence_async_smem();
       mbar_arrive(&ctl->a_ready);
       for (int layer = 0; layer < 3; ++layer, ++layer_count) {
-        if (!tc_wait(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
+        if (!tc_wait_warp(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
         tc_fence_after();
         if (layer < 2) {
           // h = relu(acc + b) -> BF16 -> A operand of the next layer (K = H)
@@ -237,12 +315,130 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           tmem_ld16(t_lane, v);
           tmem_ld_wait();
           tc_fence_before();
-          if (live) {
+          float qv[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) qv[j] = __uint_as_float(v[j]) + bias[2 * H + j];
+          if (live && p.out) {
             float* o = p.out + (size_t)row * p.Aout;
-            for (int j = 0; j < p.Aout; ++j) o[j] = __uint_as_float(v[j]) + bias[2 * H + j];
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (j < p.Aout) o[j] = qv[j];
+          }
+          if (FUSED) {
+            // epsilon-greedy on this row: explore iff x0 < threshold, else the first maximum
+            const uint4 w = stream_words(p.env.seed, STREAM_ACTION, 0, (uint32_t)row, p.env.t);
+            int best = 0;
+            float qb = qv[0];
+#pragma unroll
+            for (int j = 1; j < 16; ++j)
+              if (j < p.env.A && qv[j] > qb) { qb = qv[j]; best = j; }
+            action = ((unsigned long long)w.x < p.env.explore_thr) ? (int)__umulhi(w.y, (uint32_t)p.env.A) : best;
           }
         }
       }
+      if (FUSED) {
+        const TcEnvParams& ev = p.env;
+        const unsigned long long slot = (ev.cursor + (unsigned long long)(live ? row : 0)) % (unsigned long long)ev.C;
+        float* rec = ev.ring + slot * ev.rec_words;
+        // the FP32 state row once more: record's observation, and TF32 high / low parts as the A operand
+        {
+          const float* xr = p.x + (size_t)(live ? row : 0) * D;
+          uint8_t* dst_hi = abuf + ((size_t)(r >> 3) * (D / 4)) * 128 + (r & 7) * 16;
+          uint8_t* dst_lo = dst_hi + (size_t)TC_M * D * 4;
+          for (int kg = 0; kg < D / 4; ++kg) {
+            float4 sv = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (live) {
+              sv = __ldg(reinterpret_cast<const float4*>(xr + kg * 4));
+              *reinterpret_cast<float4*>(rec + kg * 4) = sv;
+            }
+            float4 hi, lo;
+            hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
+            hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
+            hi.z = __uint_as_float(__float_as_uint(sv.z) & 0xFFFFE000u); lo.z = sv.z - hi.z;
+            hi.w = __uint_as_float(__float_as_uint(sv.w) & 0xFFFFE000u); lo.w = sv.w - hi.w;
+            *reinterpret_cast<float4*>(dst_hi + (size_t)kg * 128) = hi;
+            *reinterpret_cast<float4*>(dst_lo + (size_t)kg * 128) = lo;
+          }
+        }
+        fence_async_smem();
+        mbar_arrive(&ctl->a_ready);
+        if (!tc_wait_warp(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
+        ++layer_count;
+        tc_fence_after();
+        // s' = tanh(z + B[a]) + noise, 16 components at a time; kept in shared memory until `done` is known
+        float* sb = reinterpret_cast<float*>(abuf) + (size_t)r * (D + 4);
+        const float* Ba = ev.lgB + (size_t)action * D;
+        float sq = 0.f;
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t v[16];
+          tmem_ld16(t_lane + (uint32_t)c0, v);
+          tmem_ld_wait();
+          float sn[16];
+#pragma unroll
+          for (int b4 = 0; b4 < 4; ++b4) {
+            const uint4 w = stream_words(ev.seed, STREAM_NOISE, (uint32_t)(c0 / 4 + b4), (uint32_t)row, ev.t);
+            const float2 z01 = box_muller(w.x, w.y), z23 = box_muller(w.z, w.w);
+            const float4 bb = __ldg(reinterpret_cast<const float4*>(Ba + c0 + 4 * b4));
+            sn[4 * b4 + 0] = tanhf(__uint_as_float(v[4 * b4 + 0]) + bb.x) + ev.noise_std * z01.x;
+            sn[4 * b4 + 1] = tanhf(__uint_as_float(v[4 * b4 + 1]) + bb.y) + ev.noise_std * z01.y;
+            sn[4 * b4 + 2] = tanhf(__uint_as_float(v[4 * b4 + 2]) + bb.z) + ev.noise_std * z23.x;
+            sn[4 * b4 + 3] = tanhf(__uint_as_float(v[4 * b4 + 3]) + bb.w) + ev.noise_std * z23.y;
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) sq = fmaf(sn[j], sn[j], sq);
+#pragma unroll
+          for (int b4 = 0; b4 < 4; ++b4) {
+            const float4 o = make_float4(sn[4 * b4], sn[4 * b4 + 1], sn[4 * b4 + 2], sn[4 * b4 + 3]);
+            *reinterpret_cast<float4*>(sb + c0 + 4 * b4) = o;
+            if (live) *reinterpret_cast<float4*>(rec + D + c0 + 4 * b4) = o;
+          }
+        }
+        tc_fence_before();
+        if (live) {
+          const float rew = -sq / (float)D;
+          int ep = ev.ep_step[row] + 1;
+          float ep_ret = ev.ep_return[row] + rew;
+          const int done = (sqrtf(sq) > ev.done_norm || ep >= ev.max_ep) ? 1 : 0;
+          *reinterpret_cast<float4*>(rec + 2 * D) =
+              make_float4(__int_as_float(action), rew, __int_as_float(done), __int_as_float(ev.version));
+          float* st = ev.state + (size_t)row * D;
+          if (done) {
+            n_episodes += 1;
+            ret_sum += (double)ep_ret;
+            ep_ret = 0.f;
+            ep = 0;
+            for (int b4 = 0; b4 < D / 4; ++b4) {
+              const uint4 w = stream_words(ev.seed, STREAM_RESET, (uint32_t)b4, (uint32_t)row, ev.t);
+              *reinterpret_cast<float4*>(st + 4 * b4) = make_float4(uniform_range(w.x, -0.1f, 0.2f), uniform_range(w.y, -0.1f, 0.2f),
+                                                                    uniform_range(w.z, -0.1f, 0.2f), uniform_range(w.w, -0.1f, 0.2f));
+            }
+          } else {
+            for (int b4 = 0; b4 < D / 4; ++b4)
+              *reinterpret_cast<float4*>(st + 4 * b4) = *reinterpret_cast<const float4*>(sb + 4 * b4);
+          }
+          ev.ep_step[row] = ep;
+          ev.ep_return[row] = ep_ret;
+        }
+        // the staging rows alias the next tile's operand buffer: every row must be consumed before it is rewritten
+        mbar_arrive(&ctl->rows_done);
+        if (!tc_wait_warp(&ctl->rows_done, tiles_done & 1, abort_flag)) goto done;
+        ++tiles_done;
+      }
+    }
+    if (FUSED) {
+      // episode statistics: one atomic pair per warp
+      unsigned long long n = n_episodes;
+      double rs = ret_sum;
+      for (int o = 16; o > 0; o >>= 1) {
+        n += __shfl_down_sync(0xffffffffu, n, o);
+        rs += __shfl_down_sync(0xffffffffu, rs, o);
+      }
+      if (lane == 0 && n) {
+        atomicAdd(&p.env.stats->episodes, n);
+        atomicAdd(&p.env.stats->return_sum, rs);
+      }
+      if (blockIdx.x == 0 && tid == 64)
+        p.env.block_ver[(p.env.cursor % (unsigned long long)p.env.C) / (unsigned long long)p.n] = p.env.version;
     }
   }
 done:
@@ -337,16 +533,43 @@ cudaError_t launch_pack_tc_weights(const float* blob, uint16_t* dst, int D, int 
 
 cudaError_t launch_tc_mlp(const TcMlpParams& p, int sm_count, cudaStream_t s) {
   if (p.n <= 0) return cudaSuccess;
-  const int Kmax = p.D > p.H ? p.D : p.H;
-  const size_t smem = (size_t)TC_M * Kmax * 2 + (size_t)TC_STAGES * TC_STAGE_BYTES + (size_t)(2 * p.H + TC_N3) * 4 +
+  const bool fused = p.env.fused != 0;
+  const size_t smem = tc_abuf_bytes(p.D, p.H, fused) + (size_t)TC_STAGES * TC_STAGE_BYTES + (size_t)(2 * p.H + TC_N3) * 4 +
                       sizeof(TcSmem) + 64;
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
-  cudaError_t e = cudaFuncSetAttribute(mlp_bf16_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kernel = fused ? mlp_bf16_tc_kernel<true> : mlp_bf16_tc_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int n_tiles = (p.n + TC_M - 1) / TC_M;
   const int grid = n_tiles < sm_count ? n_tiles : sm_count;
-  mlp_bf16_tc_kernel<<<grid, TC_THREADS, smem, s>>>(p);
+  kernel<<<grid, TC_THREADS, smem, s>>>(p);
   return cudaGetLastError();
+}
+
+// the env matrix A [D][D] as TF32 high and low parts, tiled in chunks of D rows x KC columns:
+// element (r, k) of chunk kc sits at ((r/8) * (KC/4) + (k%KC)/4) * 32 + (r%8) * 4 + k%4
+__global__ void pack_env_matrix_kernel(const float* __restrict__ A, uint32_t* __restrict__ hi, uint32_t* __restrict__ lo, int D) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= D * D) return;
+  const int chunk_elems = D * TC_KC;
+  const int kc = i / chunk_elems, within = i % chunk_elems;
+  const int core = within / 32, in_core = within % 32;
+  const int rg = core / (TC_KC / 4), kg = core % (TC_KC / 4);
+  const int r = rg * 8 + in_core / 4, k = kc * TC_KC + kg * 4 + in_core % 4;
+  const float v = A[(size_t)r * D + k];
+  const float h = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
+  hi[i] = __float_as_uint(h);
+  lo[i] = __float_as_uint(v - h);
+}
+
+cudaError_t launch_pack_env_matrix(const float* A, uint32_t* hi, uint32_t* lo, int D, cudaStream_t s) {
+  pack_env_matrix_kernel<<<(D * D + 255) / 256, 256, 0, s>>>(A, hi, lo, D);
+  return cudaGetLastError();
+}
+
+bool tc_fused_supported(int D, int H, int A) {
+  return tc_mlp_supported(D, H, A) && D <= 128 && A <= TC_N3 &&
+         tc_abuf_bytes(D, H, true) + (size_t)TC_STAGES * TC_STAGE_BYTES + (size_t)(2 * H + TC_N3) * 4 + 256 <= 227 * 1024;
 }
 
 cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
