@@ -7,7 +7,7 @@
 //                      bulk async copies (mbarrier complete_tx)
 //   warp 1, one lane   issues tcgen05.mma (M = 128, N <= 256, K = 16) over the ring; tcgen05.commit frees ring
 //                      slots and signals "accumulator full"
-//   warps 2-5          (128 threads, thread = row) convert the FP32 input rows to BF16 into the A-operand buffer;
+//   warps 2-9          (256 threads, two per row, each owning half of the columns) convert the FP32 input rows to BF16 into the A-operand buffer;
 //                      after each layer read the accumulator from TMEM (tcgen05.ld), add the bias, apply ReLU,
 //                      round to BF16 and write the next layer's A operand; after the last layer write the outputs
 // Operands use the no-swizzle K-major core-matrix layout: 8 rows x 16 bytes are contiguous (128 B), cores adjacent
@@ -30,7 +30,8 @@ constexpr int TC_M = 128;        // rows per tile
 constexpr int TC_KC = 32;        // K elements per weight chunk
 constexpr int TC_STAGES = 4;     // ring slots
 constexpr int TC_STAGE_BYTES = 256 * TC_KC * 2;   // largest chunk: 256 output rows
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;   // producer warp, MMA warp, eight epilogue warps
+constexpr int TC_EPI_THREADS = 256;
 constexpr int TC_N3 = 16;        // head width on the tensor cores (outputs padded to 16)
 
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -100,18 +101,34 @@ __device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile
   return false;
 }
 
+// Box-Muller pair with the hardware approximations (ex2/lg2/sin/cos units).  The noise enters the state scaled by
+// noise_std (0.01), so an absolute error of ~1e-6 in a normal is 1e-8 in the state, far inside the FP32 tolerance.
+__device__ __forceinline__ float2 box_muller_fast(uint32_t a, uint32_t b) {
+  const float r = sqrtf(-2.0f * __logf(u01(a)));
+  // angle 2*pi*u - pi lies in (-pi, pi) where the approximations are most accurate; cos/sin(theta) = -cos/sin(theta - pi)
+  const float th = fmaf(6.28318530717958647692f, u01(b), -3.14159265358979323846f);
+  float s, c;
+  __sincosf(th, &s, &c);
+  return make_float2(-r * c, -r * s);
+}
+
+// tanh(x) = 1 - 2 / (exp(2x) + 1) with the hardware exponential: absolute error ~2e-7 for the |x| that occur
+__device__ __forceinline__ float tanh_fast(float x) {
+  const float xc = fminf(fmaxf(x, -15.f), 15.f);
+  return 1.0f - __fdividef(2.0f, __expf(2.0f * xc) + 1.0f);
+}
+
 // for whole warps (the epilogue warps run warp-wide TMEM loads): every lane waits, and the warp leaves together
 __device__ __forceinline__ bool tc_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   const bool ok = tc_wait(bar, parity, abort_flag);
   return __all_sync(0xffffffffu, ok);
 }
 
+// two FP32 values -> packed BF16 pair (round to nearest even), `lo` in the low half
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  // round to nearest even; inputs are finite
-  uint32_t a = __float_as_uint(lo), b = __float_as_uint(hi);
-  a += 0x7FFFu + ((a >> 16) & 1u);
-  b += 0x7FFFu + ((b >> 16) & 1u);
-  return (a >> 16) | (b & 0xFFFF0000u);
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
 }
 
 // bytes of the A-operand buffer: the widest BF16 operand; in fused mode also the TF32 high+low state tile and
@@ -127,7 +144,8 @@ __host__ __device__ inline size_t tc_abuf_bytes(int D, int H, bool fused) {
 }
 
 struct TcSmem {
-  uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full, rows_done;
+  uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full, rows_done, pair_sync;
+  float sq[2][TC_M];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -146,9 +164,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
 
   if (tid == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-    mbar_init(&ctl->a_ready, 128);
+    mbar_init(&ctl->a_ready, TC_EPI_THREADS);
     mbar_init(&ctl->acc_full, 1);
-    mbar_init(&ctl->rows_done, 128);
+    mbar_init(&ctl->rows_done, TC_EPI_THREADS);
+    mbar_init(&ctl->pair_sync, TC_EPI_THREADS);
     ctl->abort_flag = 0;
   }
   for (int i = tid; i < 2 * H + TC_N3; i += TC_THREADS) {
@@ -171,8 +190,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
 
   // chunk schedule of one tile, the same for producer and MMA issuer:
   //   layer 1: n_blocks x (D/KC) chunks of NB rows; layer 2: n_blocks x (H/KC) chunks of NB rows;
-  //   layer 3: (H/KC) chunks of 16 rows
-  const int c1 = n_blocks * (D / TC_KC), c2 = n_blocks * (H / TC_KC), c3 = H / TC_KC;
+  //   layer 3: one chunk of 16 rows x H columns
+  const int c1 = n_blocks * (D / TC_KC), c2 = n_blocks * (H / TC_KC), c3 = 1;
   const int ce = D / TC_KC;   // fused mode: chunks of the env matrix per TF32 pass (three passes)
 
   if (warp == 0 && lane == 0) {
@@ -181,7 +200,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
       const uint8_t* src = reinterpret_cast<const uint8_t*>(p.wtc);
       for (int c = 0; c < c1 + c2 + c3; ++c, ++it) {
-        const uint32_t bytes = (c < c1 + c2 ? NB : TC_N3) * TC_KC * 2;
+        const uint32_t bytes = c < c1 + c2 ? (uint32_t)NB * TC_KC * 2 : (uint32_t)TC_N3 * H * 2;
         const int s = it % TC_STAGES;
         if (!tc_wait(&ctl->empty[s], ((it / TC_STAGES) & 1) ^ 1, abort_flag)) goto done;
         mbar_expect_tx(&ctl->full[s], bytes);
@@ -190,8 +209,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
       }
       if (FUSED) {
         const uint32_t bytes = (uint32_t)D * TC_KC * 4;
-        for (int c = 0; c < 3 * ce; ++c, ++it) {
-          const uint8_t* esrc = reinterpret_cast<const uint8_t*>(c < 2 * ce ? p.env.lgA_hi : p.env.lgA_lo) + (size_t)(c % ce) * bytes;
+        for (int c = 0; c < 2 * ce; ++c, ++it) {
+          const uint8_t* esrc = reinterpret_cast<const uint8_t*>(c < ce ? p.env.lgA_hi : p.env.lgA_lo) + (size_t)(c % ce) * bytes;
           const int s = it % TC_STAGES;
           if (!tc_wait(&ctl->empty[s], ((it / TC_STAGES) & 1) ^ 1, abort_flag)) goto done;
           mbar_expect_tx(&ctl->full[s], bytes);
@@ -211,19 +230,32 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         const uint32_t a_sbo = (uint32_t)(K / 8) * 128u, b_sbo = (uint32_t)(TC_KC / 8) * 128u;
         if (!tc_wait(&ctl->a_ready, layer_count & 1, abort_flag)) goto done;
         tc_fence_after();
-        for (int nb = 0; nb < nb_count; ++nb) {
-          for (int kc = 0; kc < K / TC_KC; ++kc, ++it) {
-            const int s = it % TC_STAGES;
-            if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
-            tc_fence_after();
-            const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
-            const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 8)) * 128u;
+        if (layer == 2) {
+          // the head's weights arrive as one chunk: 16 rows x H columns
+          const int s = it % TC_STAGES;
+          if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
+          tc_fence_after();
+          const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
+          for (int j = 0; j < H / 16; ++j)
+            umma_bf16(tmem, make_desc(smem_addr(abuf) + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, a_sbo), idesc,
+                      j != 0);
+          umma_commit(&ctl->empty[s]);
+          ++it;
+        } else {
+          for (int nb = 0; nb < nb_count; ++nb) {
+            for (int kc = 0; kc < K / TC_KC; ++kc, ++it) {
+              const int s = it % TC_STAGES;
+              if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
+              tc_fence_after();
+              const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
+              const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 8)) * 128u;
 #pragma unroll
-            for (int j = 0; j < TC_KC / 16; ++j) {
-              umma_bf16(tmem + (uint32_t)(nb * NB), make_desc(a_base + j * 256u, 128u, a_sbo),
-                        make_desc(b_base + j * 256u, 128u, b_sbo), idesc, (kc | j) != 0);
+              for (int j = 0; j < TC_KC / 16; ++j) {
+                umma_bf16(tmem + (uint32_t)(nb * NB), make_desc(a_base + j * 256u, 128u, a_sbo),
+                          make_desc(b_base + j * 256u, 128u, b_sbo), idesc, (kc | j) != 0);
+              }
+              umma_commit(&ctl->empty[s]);    // the slot is free once these MMAs have read it
             }
-            umma_commit(&ctl->empty[s]);    // the slot is free once these MMAs have read it
           }
         }
         umma_commit(&ctl->acc_full);        // accumulator of this layer complete
@@ -235,17 +267,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         const uint32_t lo_off = (uint32_t)TC_M * D * 4;
         if (!tc_wait(&ctl->a_ready, layer_count & 1, abort_flag)) goto done;
         tc_fence_after();
-        for (int pass = 0; pass < 3; ++pass) {
+        for (int half = 0; half < 2; ++half) {       // chunks of A_hi (used with s_hi and s_lo), then of A_lo (with s_hi)
           for (int kc = 0; kc < ce; ++kc, ++it) {
             const int s = it % TC_STAGES;
             if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
             tc_fence_after();
             const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
-            const uint32_t a_base = smem_addr(abuf) + (pass == 1 ? lo_off : 0u) + (uint32_t)(kc * (TC_KC / 4)) * 128u;
+            const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 4)) * 128u;
 #pragma unroll
             for (int j = 0; j < TC_KC / 8; ++j) {
               umma_tf32(tmem, make_desc(a_base + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, b_sbo), idesc,
-                        (pass | kc | j) != 0);
+                        (half | kc | j) != 0);
+              if (half == 0)
+                umma_tf32(tmem, make_desc(a_base + lo_off + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, b_sbo),
+                          idesc, true);
             }
             umma_commit(&ctl->empty[s]);
           }
@@ -256,24 +291,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ operand conversion and epilogues
+    // Eight warps: two per TMEM lane quarter.  A row (TMEM lane) is shared by two threads, each owning one
+    // half of the columns / components (hsel).
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    const int hsel = (warp - 2) >> 2;             // which half of the columns this thread handles
     const int r = q * 32 + lane;                  // row of the tile = TMEM lane
     const uint32_t t_lane = tmem + ((uint32_t)(q * 32) << 16);
     uint32_t layer_count = 0;
     int action = 0;
-    uint32_t tiles_done = 0;
+    uint32_t tiles_done = 0, pair_count = 0;
     unsigned long long n_episodes = 0;
     double ret_sum = 0.0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const long long row = (long long)tile * TC_M + r;
       const bool live = row < p.n;
-      // layer-1 A operand: this row of x, FP32 -> BF16, 8 elements (16 bytes) at a time
+      // layer-1 A operand: this row of x, FP32 -> BF16, 8 elements (16 bytes) at a time.  In fused mode
+      // (D <= 128) the thread keeps its half row in registers: it is the record's observation and the TF32
+      // operand later in the tile, so the state is read from memory once.
+      float4 keep[FUSED ? 16 : 1];
       {
         const float* xr = p.x + (size_t)(live ? row : 0) * D;
         uint8_t* dst = abuf + ((size_t)(r >> 3) * (D / 8)) * 128 + (r & 7) * 16;
-        for (int kg = 0; kg < D / 8; ++kg) {
+        const int g0 = hsel * (D / 16), g1 = g0 + D / 16;
+        if (FUSED) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            keep[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (live && i < D / 8) keep[i] = __ldg(reinterpret_cast<const float4*>(xr + g0 * 8 + i * 4));
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < 8; ++gi) {
+          const int kg = g0 + gi;
+          if (kg >= g1) break;
           float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-          if (live) {
+          if (FUSED) {
+            lo = keep[2 * gi];
+            hi = keep[2 * gi + 1];
+          } else if (live) {
             lo = __ldg(reinterpret_cast<const float4*>(xr + kg * 8));
             hi = __ldg(reinterpret_cast<const float4*>(xr + kg * 8 + 4));
           }
@@ -289,23 +344,30 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         if (!tc_wait_warp(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
         tc_fence_after();
         if (layer < 2) {
-          // h = relu(acc + b) -> BF16 -> A operand of the next layer (K = H)
+          // h = relu(acc + b) -> BF16 -> A operand of the next layer (K = H); 32 columns per TMEM round trip
           const float* b = bias + layer * H;
           uint8_t* dst = abuf + ((size_t)(r >> 3) * (H / 8)) * 128 + (r & 7) * 16;
-          for (int c0 = 0; c0 < H; c0 += 16) {
-            uint32_t v[16];
+          const int c_begin = hsel * (H / 2), c_end = c_begin + H / 2;
+          for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+            uint32_t v[32];
+            const bool two = c0 + 32 <= c_end;
             tmem_ld16(t_lane + (uint32_t)c0, v);
+            if (two) tmem_ld16(t_lane + (uint32_t)(c0 + 16), v + 16);
             tmem_ld_wait();
-            float f[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) f[j] = fmaxf(__uint_as_float(v[j]) + b[c0 + j], 0.f);
-            uint4 o0, o1;
-            o0.x = pack_bf16x2(f[0], f[1]); o0.y = pack_bf16x2(f[2], f[3]);
-            o0.z = pack_bf16x2(f[4], f[5]); o0.w = pack_bf16x2(f[6], f[7]);
-            o1.x = pack_bf16x2(f[8], f[9]); o1.y = pack_bf16x2(f[10], f[11]);
-            o1.z = pack_bf16x2(f[12], f[13]); o1.w = pack_bf16x2(f[14], f[15]);
-            *reinterpret_cast<uint4*>(dst + (size_t)(c0 / 8) * 128) = o0;
-            *reinterpret_cast<uint4*>(dst + (size_t)(c0 / 8 + 1) * 128) = o1;
+            for (int hh = 0; hh < 2; ++hh) {
+              if (hh == 1 && !two) break;
+              const int cc = c0 + 16 * hh;
+              uint32_t o[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float f0 = fmaxf(__uint_as_float(v[16 * hh + 2 * j]) + b[cc + 2 * j], 0.f);
+                const float f1 = fmaxf(__uint_as_float(v[16 * hh + 2 * j + 1]) + b[cc + 2 * j + 1], 0.f);
+                o[j] = pack_bf16x2(f0, f1);
+              }
+              *reinterpret_cast<uint4*>(dst + (size_t)(cc / 8) * 128) = make_uint4(o[0], o[1], o[2], o[3]);
+              *reinterpret_cast<uint4*>(dst + (size_t)(cc / 8 + 1) * 128) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
           }
           tc_fence_before();
           fence_async_smem();
@@ -318,7 +380,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           float qv[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) qv[j] = __uint_as_float(v[j]) + bias[2 * H + j];
-          if (live && p.out) {
+          if (live && p.out && hsel == 0) {
             float* o = p.out + (size_t)row * p.Aout;
 #pragma unroll
             for (int j = 0; j < 16; ++j)
@@ -342,15 +404,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         float* rec = ev.ring + slot * ev.rec_words;
         // the FP32 state row once more: record's observation, and TF32 high / low parts as the A operand
         {
-          const float* xr = p.x + (size_t)(live ? row : 0) * D;
           uint8_t* dst_hi = abuf + ((size_t)(r >> 3) * (D / 4)) * 128 + (r & 7) * 16;
           uint8_t* dst_lo = dst_hi + (size_t)TC_M * D * 4;
-          for (int kg = 0; kg < D / 4; ++kg) {
-            float4 sv = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live) {
-              sv = __ldg(reinterpret_cast<const float4*>(xr + kg * 4));
-              *reinterpret_cast<float4*>(rec + kg * 4) = sv;
-            }
+          const int g0 = hsel * (D / 8);
+#pragma unroll
+          for (int gi = 0; gi < 16; ++gi) {
+            if (gi >= D / 8) break;
+            const int kg = g0 + gi;
+            const float4 sv = keep[gi];
+            if (live) *reinterpret_cast<float4*>(rec + kg * 4) = sv;
             float4 hi, lo;
             hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
             hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
@@ -369,7 +431,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         float* sb = reinterpret_cast<float*>(abuf) + (size_t)r * (D + 4);
         const float* Ba = ev.lgB + (size_t)action * D;
         float sq = 0.f;
-        for (int c0 = 0; c0 < D; c0 += 16) {
+        const int c_begin = hsel * (D / 2), c_end = c_begin + D / 2;
+        for (int c0 = c_begin; c0 < c_end; c0 += 16) {
           uint32_t v[16];
           tmem_ld16(t_lane + (uint32_t)c0, v);
           tmem_ld_wait();
@@ -377,12 +440,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
 #pragma unroll
           for (int b4 = 0; b4 < 4; ++b4) {
             const uint4 w = stream_words(ev.seed, STREAM_NOISE, (uint32_t)(c0 / 4 + b4), (uint32_t)row, ev.t);
-            const float2 z01 = box_muller(w.x, w.y), z23 = box_muller(w.z, w.w);
+            const float2 z01 = box_muller_fast(w.x, w.y), z23 = box_muller_fast(w.z, w.w);
             const float4 bb = __ldg(reinterpret_cast<const float4*>(Ba + c0 + 4 * b4));
-            sn[4 * b4 + 0] = tanhf(__uint_as_float(v[4 * b4 + 0]) + bb.x) + ev.noise_std * z01.x;
-            sn[4 * b4 + 1] = tanhf(__uint_as_float(v[4 * b4 + 1]) + bb.y) + ev.noise_std * z01.y;
-            sn[4 * b4 + 2] = tanhf(__uint_as_float(v[4 * b4 + 2]) + bb.z) + ev.noise_std * z23.x;
-            sn[4 * b4 + 3] = tanhf(__uint_as_float(v[4 * b4 + 3]) + bb.w) + ev.noise_std * z23.y;
+            sn[4 * b4 + 0] = tanh_fast(__uint_as_float(v[4 * b4 + 0]) + bb.x) + ev.noise_std * z01.x;
+            sn[4 * b4 + 1] = tanh_fast(__uint_as_float(v[4 * b4 + 1]) + bb.y) + ev.noise_std * z01.y;
+            sn[4 * b4 + 2] = tanh_fast(__uint_as_float(v[4 * b4 + 2]) + bb.z) + ev.noise_std * z23.x;
+            sn[4 * b4 + 3] = tanh_fast(__uint_as_float(v[4 * b4 + 3]) + bb.w) + ev.noise_std * z23.y;
           }
 #pragma unroll
           for (int j = 0; j < 16; ++j) sq = fmaf(sn[j], sn[j], sq);
@@ -394,30 +457,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           }
         }
         tc_fence_before();
+        // the two halves of a row exchange their partial squared norms (low half first in the sum)
+        ctl->sq[hsel][r] = sq;
+        // both threads of a row read the episode counters before the barrier; only one writes them after it
+        const int ep0 = live ? ev.ep_step[row] : 0;
+        const float ret0 = live ? ev.ep_return[row] : 0.f;
+        mbar_arrive(&ctl->pair_sync);
+        if (!tc_wait_warp(&ctl->pair_sync, pair_count & 1, abort_flag)) goto done;
+        ++pair_count;
+        sq = ctl->sq[0][r] + ctl->sq[1][r];
         if (live) {
           const float rew = -sq / (float)D;
-          int ep = ev.ep_step[row] + 1;
-          float ep_ret = ev.ep_return[row] + rew;
+          int ep = ep0 + 1;
+          float ep_ret = ret0 + rew;
           const int done = (sqrtf(sq) > ev.done_norm || ep >= ev.max_ep) ? 1 : 0;
-          *reinterpret_cast<float4*>(rec + 2 * D) =
-              make_float4(__int_as_float(action), rew, __int_as_float(done), __int_as_float(ev.version));
           float* st = ev.state + (size_t)row * D;
+          const int b_begin = hsel * (D / 8), b_end = b_begin + D / 8;
           if (done) {
-            n_episodes += 1;
-            ret_sum += (double)ep_ret;
             ep_ret = 0.f;
             ep = 0;
-            for (int b4 = 0; b4 < D / 4; ++b4) {
+            for (int b4 = b_begin; b4 < b_end; ++b4) {
               const uint4 w = stream_words(ev.seed, STREAM_RESET, (uint32_t)b4, (uint32_t)row, ev.t);
               *reinterpret_cast<float4*>(st + 4 * b4) = make_float4(uniform_range(w.x, -0.1f, 0.2f), uniform_range(w.y, -0.1f, 0.2f),
                                                                     uniform_range(w.z, -0.1f, 0.2f), uniform_range(w.w, -0.1f, 0.2f));
             }
           } else {
-            for (int b4 = 0; b4 < D / 4; ++b4)
+            for (int b4 = b_begin; b4 < b_end; ++b4)
               *reinterpret_cast<float4*>(st + 4 * b4) = *reinterpret_cast<const float4*>(sb + 4 * b4);
           }
-          ev.ep_step[row] = ep;
-          ev.ep_return[row] = ep_ret;
+          if (hsel == 0) {
+            *reinterpret_cast<float4*>(rec + 2 * D) =
+                make_float4(__int_as_float(action), rew, __int_as_float(done), __int_as_float(ev.version));
+            if (done) {
+              n_episodes += 1;
+              ret_sum += (double)(ret0 + rew);
+            }
+            ev.ep_step[row] = ep;
+            ev.ep_return[row] = ep_ret;
+          }
         }
         // the staging rows alias the next tile's operand buffer: every row must be consumed before it is rewritten
         mbar_arrive(&ctl->rows_done);
@@ -452,7 +529,8 @@ done:
 }
 
 // FP32 blob -> BF16 chunks in the order the producer streams them; within a chunk of R rows x KC columns
-// element (r, k) sits at ((r/8) * (KC/8) + k/8) * 64 + (r%8) * 8 + k%8.
+// element (r, k) sits at ((r/8) * (KC/8) + k/8) * 64 + (r%8) * 8 + k%8.  Hidden layers: R = NB, KC = 32;
+// head: one chunk with R = 16, KC = H.
 __global__ void pack_tc_weights_kernel(const float* __restrict__ blob, uint16_t* __restrict__ dst, int D, int H, int A,
                                        int value_head) {
   const int n_blocks = H > 256 ? 2 : 1, NB = H / n_blocks;
@@ -469,14 +547,15 @@ __global__ void pack_tc_weights_kernel(const float* __restrict__ blob, uint16_t*
   if (j < n1) { W = W1; K = D; R = NB; rows_total = H; }
   else if (j < n1 + n2) { j -= n1; W = W2; K = H; R = NB; rows_total = H; }
   else { j -= n1 + n2; W = W3; K = H; R = TC_N3; rows_total = A; }
-  const size_t chunk_elems = (size_t)R * TC_KC;
+  const int KCc = W == W3 ? H : TC_KC;               // columns per chunk (the head is one chunk)
+  const size_t chunk_elems = (size_t)R * KCc;
   const size_t chunk = j / chunk_elems, within = j % chunk_elems;
-  const int chunks_per_block = K / TC_KC;
+  const int chunks_per_block = K / KCc;
   const int nb = (int)(chunk / chunks_per_block), kc = (int)(chunk % chunks_per_block);
   n_off = nb * R;
   const int core = (int)(within / 64), in_core = (int)(within % 64);
-  const int rg = core / (TC_KC / 8), kg = core % (TC_KC / 8);
-  const int r = rg * 8 + in_core / 8, k = kc * TC_KC + kg * 8 + in_core % 8;
+  const int rg = core / (KCc / 8), kg = core % (KCc / 8);
+  const int r = rg * 8 + in_core / 8, k = kc * KCc + kg * 8 + in_core % 8;
   const int n = n_off + r;
   float v = 0.f;
   if (n < rows_total) v = W[(size_t)n * K + k];
