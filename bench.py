@@ -103,13 +103,41 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of per-rank timings over all ranks (the job runs as long as its slowest replica)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def min_over_ranks(values, device):
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+    return [float(x) for x in t.tolist()]
+
+
+def aggregate_throughput(units_per_replica, world, max_ms):
+    """Whole-job rate of `world` independent replicas that each processed units_per_replica in max_ms."""
+    return units_per_replica * world / (max_ms * 1e-3)
+
+
 # --------------------------------------------------------------------------------------------- our arm
 class Runner:
     """Drives one context through the workload's call pattern."""
 
-    def __init__(self, name, torch, binding, device_index):
+    def __init__(self, name, torch, binding, device_index, n_envs=0):
         self.torch, self.name = torch, name
-        self.w = synth.WORKLOADS[name]
+        self.w = dict(synth.WORKLOADS[name])
+        if n_envs:
+            if self.w["replay_capacity"]:
+                self.w["replay_capacity"] = self.w["replay_capacity"] // self.w["n_envs"] * n_envs
+            self.w["n_envs"] = n_envs
         self.f = synth.config_fields(self.w, device=device_index)
         self.ctx = binding.Context(**self.f)
         self.on_policy = self.w["replay_capacity"] == 0
@@ -211,7 +239,8 @@ def run_ours(args):
     peaks = load_peaks()
     name = args.workload
     w = synth.WORKLOADS[name]
-    r = Runner(name, torch, binding, local)
+    r = Runner(name, torch, binding, local, args.envs)
+    w = r.w
     N = w["n_envs"]
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     ring_bytes = w["replay_capacity"] * (2 * w["obs_dim"] + 4) * 4
@@ -258,12 +287,11 @@ def run_ours(args):
     r.ctx.set_profiling(0)
     barrier()
 
-    times = torch.tensor([tot_ms, e2e_ms, act_ms, lrn_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    tot_ms, e2e_ms, act_ms, lrn_ms = [float(x) for x in times.tolist()]
+    tot_ms, e2e_ms, act_ms, lrn_ms = max_over_ranks([tot_ms, e2e_ms, act_ms, lrn_ms], "cuda")
+    learner_ok = int(min_over_ranks([learner_ok], "cuda")[0])
     K = args.steps
     env_steps = N * r.actor_steps * K * world
+    assert abs(aggregate_throughput(N * r.actor_steps * K, world, tot_ms) - env_steps / (tot_ms * 1e-3)) < 1e-6 * env_steps
     consumed = (w["rollout_len"] * N if r.on_policy else w["minibatch"]) * learner_ok * world
     value = env_steps / (tot_ms * 1e-3)
     flops, nbytes = actor_algorithmic(w)
@@ -434,6 +462,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="cfg5", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--envs", type=int, default=0, help="profiling aid: run the workload with this many envs (ring scaled to the same number of steps)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
