@@ -28,7 +28,7 @@ namespace {
 
 constexpr int TC_M = 128;        // rows per tile
 constexpr int TC_KC = 32;        // K elements per weight chunk
-constexpr int TC_STAGES = 4;     // ring slots
+constexpr int TC_STAGES = 5;     // ring slots
 constexpr int TC_STAGE_BYTES = 256 * TC_KC * 2;   // largest chunk: 256 output rows
 constexpr int TC_THREADS = 320;   // producer warp, MMA warp, eight epilogue warps
 constexpr int TC_EPI_THREADS = 256;
@@ -302,18 +302,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     uint32_t tiles_done = 0, pair_count = 0;
     unsigned long long n_episodes = 0;
     double ret_sum = 0.0;
+    float4 keep[FUSED ? 16 : 1];   // this thread's half row of the FP32 state (fused mode)
+    bool have_row = false;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const long long row = (long long)tile * TC_M + r;
       const bool live = row < p.n;
       // layer-1 A operand: this row of x, FP32 -> BF16, 8 elements (16 bytes) at a time.  In fused mode
       // (D <= 128) the thread keeps its half row in registers: it is the record's observation and the TF32
       // operand later in the tile, so the state is read from memory once.
-      float4 keep[FUSED ? 16 : 1];
       {
         const float* xr = p.x + (size_t)(live ? row : 0) * D;
         uint8_t* dst = abuf + ((size_t)(r >> 3) * (D / 8)) * 128 + (r & 7) * 16;
         const int g0 = hsel * (D / 16), g1 = g0 + D / 16;
-        if (FUSED) {
+        if (FUSED && !have_row) {      // first tile of this block; later tiles were fetched during the previous env epilogue
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             keep[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -412,7 +413,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
             if (gi >= D / 8) break;
             const int kg = g0 + gi;
             const float4 sv = keep[gi];
-            if (live) *reinterpret_cast<float4*>(rec + kg * 4) = sv;
             float4 hi, lo;
             hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
             hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
@@ -424,6 +424,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         }
         fence_async_smem();
         mbar_arrive(&ctl->a_ready);
+        // while the TF32 products run: the record's observation, then the next tile's row of the state
+        if (live) {
+#pragma unroll
+          for (int gi = 0; gi < 16; ++gi)
+            if (gi < D / 8) *reinterpret_cast<float4*>(rec + (hsel * (D / 8) + gi) * 4) = keep[gi];
+        }
+        {
+          const long long nrow = (long long)(tile + (int)gridDim.x) * TC_M + r;
+          have_row = true;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            keep[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (nrow < p.n && i < D / 8) keep[i] = __ldg(reinterpret_cast<const float4*>(p.x + (size_t)nrow * D + hsel * (D / 2) + i * 4));
+          }
+        }
         if (!tc_wait_warp(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
         ++layer_count;
         tc_fence_after();
