@@ -7,7 +7,7 @@
 //                      bulk async copies (mbarrier complete_tx)
 //   warp 1, one lane   issues tcgen05.mma (M = 128, N <= 256, K = 16) over the ring; tcgen05.commit frees ring
 //                      slots and signals "accumulator full"
-//   warps 2-9          (256 threads, two per row, each owning half of the columns) convert the FP32 input rows to BF16 into the A-operand buffer;
+//   warps 2-9          (256 threads, TC_SPLIT = 2 per row, each owning half of the columns) convert the FP32 input rows to BF16 into the A-operand buffer;
 //                      after each layer read the accumulator from TMEM (tcgen05.ld), add the bias, apply ReLU,
 //                      round to BF16 and write the next layer's A operand; after the last layer write the outputs
 // Operands use the no-swizzle K-major core-matrix layout: 8 rows x 16 bytes are contiguous (128 B), cores adjacent
@@ -30,8 +30,10 @@ constexpr int TC_M = 128;        // rows per tile
 constexpr int TC_KC = 32;        // K elements per weight chunk
 constexpr int TC_STAGES = 5;     // ring slots
 constexpr int TC_STAGE_BYTES = 256 * TC_KC * 2;   // largest chunk: 256 output rows
-constexpr int TC_THREADS = 320;   // producer warp, MMA warp, eight epilogue warps
-constexpr int TC_EPI_THREADS = 256;
+constexpr int TC_SPLIT = 2;         // epilogue threads per row (each owns 1/TC_SPLIT of the columns); 4 measured no faster
+constexpr int TC_EPI_THREADS = 128 * TC_SPLIT;
+constexpr int TC_THREADS = 64 + TC_EPI_THREADS;   // producer warp, MMA warp, 4 * TC_SPLIT epilogue warps
+constexpr int TC_KEEP = 32 / TC_SPLIT;            // float4 registers holding a thread's share of a 128-wide state row
 constexpr int TC_N3 = 16;        // head width on the tensor cores (outputs padded to 16)
 
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -145,7 +147,7 @@ __host__ __device__ inline size_t tc_abuf_bytes(int D, int H, bool fused) {
 
 struct TcSmem {
   uint64_t full[TC_STAGES], empty[TC_STAGES], a_ready, acc_full, rows_done, pair_sync;
-  float sq[2][TC_M];
+  float sq[TC_SPLIT][TC_M];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -291,8 +293,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ operand conversion and epilogues
-    // Eight warps: two per TMEM lane quarter.  A row (TMEM lane) is shared by two threads, each owning one
-    // half of the columns / components (hsel).
+    // 4 * TC_SPLIT warps: TC_SPLIT per TMEM lane quarter.  A row (TMEM lane) is shared by TC_SPLIT threads, each
+    // owning one share of the columns / components (hsel).
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     const int hsel = (warp - 2) >> 2;             // which half of the columns this thread handles
     const int r = q * 32 + lane;                  // row of the tile = TMEM lane
@@ -302,7 +304,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
     uint32_t tiles_done = 0, pair_count = 0;
     unsigned long long n_episodes = 0;
     double ret_sum = 0.0;
-    float4 keep[FUSED ? 16 : 1];   // this thread's half row of the FP32 state (fused mode)
+    float4 keep[FUSED ? TC_KEEP : 1];   // this thread's half row of the FP32 state (fused mode)
     bool have_row = false;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const long long row = (long long)tile * TC_M + r;
@@ -313,16 +315,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
       {
         const float* xr = p.x + (size_t)(live ? row : 0) * D;
         uint8_t* dst = abuf + ((size_t)(r >> 3) * (D / 8)) * 128 + (r & 7) * 16;
-        const int g0 = hsel * (D / 16), g1 = g0 + D / 16;
+        const int g0 = hsel * (D / (8 * TC_SPLIT)), g1 = g0 + D / (8 * TC_SPLIT);
         if (FUSED && !have_row) {      // first tile of this block; later tiles were fetched during the previous env epilogue
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
+          for (int i = 0; i < TC_KEEP; ++i) {
             keep[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (live && i < D / 8) keep[i] = __ldg(reinterpret_cast<const float4*>(xr + g0 * 8 + i * 4));
+            if (live && i < D / (4 * TC_SPLIT)) keep[i] = __ldg(reinterpret_cast<const float4*>(xr + g0 * 8 + i * 4));
           }
         }
 #pragma unroll
-        for (int gi = 0; gi < 8; ++gi) {
+        for (int gi = 0; gi < (FUSED ? TC_KEEP / 2 : 16 / TC_SPLIT); ++gi) {
           const int kg = g0 + gi;
           if (kg >= g1) break;
           float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
@@ -348,7 +350,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           // h = relu(acc + b) -> BF16 -> A operand of the next layer (K = H); 32 columns per TMEM round trip
           const float* b = bias + layer * H;
           uint8_t* dst = abuf + ((size_t)(r >> 3) * (H / 8)) * 128 + (r & 7) * 16;
-          const int c_begin = hsel * (H / 2), c_end = c_begin + H / 2;
+          const int c_begin = hsel * (H / TC_SPLIT), c_end = c_begin + H / TC_SPLIT;
           for (int c0 = c_begin; c0 < c_end; c0 += 32) {
             uint32_t v[32];
             const bool two = c0 + 32 <= c_end;
@@ -407,10 +409,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         {
           uint8_t* dst_hi = abuf + ((size_t)(r >> 3) * (D / 4)) * 128 + (r & 7) * 16;
           uint8_t* dst_lo = dst_hi + (size_t)TC_M * D * 4;
-          const int g0 = hsel * (D / 8);
+          const int g0 = hsel * (D / (4 * TC_SPLIT));
 #pragma unroll
-          for (int gi = 0; gi < 16; ++gi) {
-            if (gi >= D / 8) break;
+          for (int gi = 0; gi < TC_KEEP; ++gi) {
+            if (gi >= D / (4 * TC_SPLIT)) break;
             const int kg = g0 + gi;
             const float4 sv = keep[gi];
             float4 hi, lo;
@@ -427,16 +429,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         // while the TF32 products run: the record's observation, then the next tile's row of the state
         if (live) {
 #pragma unroll
-          for (int gi = 0; gi < 16; ++gi)
-            if (gi < D / 8) *reinterpret_cast<float4*>(rec + (hsel * (D / 8) + gi) * 4) = keep[gi];
+          for (int gi = 0; gi < TC_KEEP; ++gi)
+            if (gi < D / (4 * TC_SPLIT)) *reinterpret_cast<float4*>(rec + (hsel * (D / (4 * TC_SPLIT)) + gi) * 4) = keep[gi];
         }
         {
           const long long nrow = (long long)(tile + (int)gridDim.x) * TC_M + r;
           have_row = true;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
+          for (int i = 0; i < TC_KEEP; ++i) {
             keep[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (nrow < p.n && i < D / 8) keep[i] = __ldg(reinterpret_cast<const float4*>(p.x + (size_t)nrow * D + hsel * (D / 2) + i * 4));
+            if (nrow < p.n && i < D / (4 * TC_SPLIT))
+              keep[i] = __ldg(reinterpret_cast<const float4*>(p.x + (size_t)nrow * D + hsel * (D / TC_SPLIT) + i * 4));
           }
         }
         if (!tc_wait_warp(&ctl->acc_full, layer_count & 1, abort_flag)) goto done;
@@ -446,7 +449,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         float* sb = reinterpret_cast<float*>(abuf) + (size_t)r * (D + 4);
         const float* Ba = ev.lgB + (size_t)action * D;
         float sq = 0.f;
-        const int c_begin = hsel * (D / 2), c_end = c_begin + D / 2;
+        const int c_begin = hsel * (D / TC_SPLIT), c_end = c_begin + D / TC_SPLIT;
         for (int c0 = c_begin; c0 < c_end; c0 += 16) {
           uint32_t v[16];
           tmem_ld16(t_lane + (uint32_t)c0, v);
@@ -480,14 +483,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
         mbar_arrive(&ctl->pair_sync);
         if (!tc_wait_warp(&ctl->pair_sync, pair_count & 1, abort_flag)) goto done;
         ++pair_count;
-        sq = ctl->sq[0][r] + ctl->sq[1][r];
+        sq = ctl->sq[0][r];
+#pragma unroll
+        for (int h2 = 1; h2 < TC_SPLIT; ++h2) sq += ctl->sq[h2][r];
         if (live) {
           const float rew = -sq / (float)D;
           int ep = ep0 + 1;
           float ep_ret = ret0 + rew;
           const int done = (sqrtf(sq) > ev.done_norm || ep >= ev.max_ep) ? 1 : 0;
           float* st = ev.state + (size_t)row * D;
-          const int b_begin = hsel * (D / 8), b_end = b_begin + D / 8;
+          const int b_begin = hsel * (D / (4 * TC_SPLIT)), b_end = b_begin + D / (4 * TC_SPLIT);
           if (done) {
             ep_ret = 0.f;
             ep = 0;
@@ -612,7 +617,8 @@ __global__ void td_from_q_kernel(const float* __restrict__ q_online, const float
 }  // namespace
 
 bool tc_mlp_supported(int D, int H, int Aout) {
-  if (D % TC_KC || H % TC_KC || D < TC_KC || H < TC_KC || H > 512 || D > 512 || Aout > TC_N3) return false;
+  if (D % TC_KC || H % TC_KC || D < TC_KC || H < TC_KC || H > 512 || D > 128 || Aout > TC_N3) return false;
+  if (H % (16 * TC_SPLIT) || D % (8 * TC_SPLIT)) return false;   // every epilogue thread owns whole 16-column groups
   const int n_blocks = H > 256 ? 2 : 1;
   return (H / n_blocks) % 16 == 0;
 }
@@ -662,7 +668,7 @@ cudaError_t launch_pack_env_matrix(const float* A, uint32_t* hi, uint32_t* lo, i
 }
 
 bool tc_fused_supported(int D, int H, int A) {
-  return tc_mlp_supported(D, H, A) && D <= 128 && A <= TC_N3 &&
+  return tc_mlp_supported(D, H, A) && D <= 128 && D % (16 * TC_SPLIT) == 0 && A <= TC_N3 &&
          tc_abuf_bytes(D, H, true) + (size_t)TC_STAGES * TC_STAGE_BYTES + (size_t)(2 * H + TC_N3) * 4 + 256 <= 227 * 1024;
 }
 
