@@ -87,7 +87,7 @@ __device__ __forceinline__ float4 reset4(uint2 seed, uint32_t block, uint32_t e,
 // ------------------------------------------------------------------------------------------------
 // CartPole / Acrobot: one thread owns one environment (state in registers).
 // ------------------------------------------------------------------------------------------------
-template <int TE, int NT, int EPT, int ENV, int STAGE>
+template <int TE, int NT, int EPT, int NPT, int ENV, int STAGE>
 __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p) {
   extern __shared__ __align__(128) float smem[];
   __shared__ __align__(8) uint64_t wbar;
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
         if (k < p.D) sm.xs[k * TE + tid] = owner ? obs[k] : 0.f;
     }
     __syncthreads();
-    mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+    mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
     if (owner) {
       auto logit = [&](int i) { return sm.out[i * TE + tid]; };
       if (p.dbg_logits) {
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
           if (k < p.D) sm.xs[k * TE + tid] = owner ? o2[k] : 0.f;
       }
       __syncthreads();
-      mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2)>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
+      mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, p.D, p.H, p.Hp, p.Aout, p.Ap, sm.xs, sm.h1, sm.h2, sm.out);
       if (owner) {
         const int slot = (int)((long long)(t / (unsigned long long)p.T) % p.G);
         p.seg_val[((size_t)slot * (p.T + 1) + p.T) * p.N + e] = sm.out[p.A * TE + tid];
@@ -398,12 +398,12 @@ cudaError_t launch_with_smem(K kernel, int grid, int threads, size_t smem_bytes,
 constexpr size_t kSmemMax = 227 * 1024 - 1024;   // per block, leaving room for static shared memory
 constexpr size_t kSmemTwoPerSm = 112 * 1024;     // two resident blocks per SM
 
-template <int TE, int NT, int EPT, int ENV>
+template <int TE, int NT, int EPT, int NPT, int ENV>
 cudaError_t launch_small(int stage, size_t smem, const ActorParams& p, cudaStream_t s) {
   const int grid = (p.N + TE - 1) / TE;
-  if (stage == 2) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 2>, grid, NT, smem, p, s);
-  if (stage == 1) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 1>, grid, NT, smem, p, s);
-  return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, ENV, 0>, grid, NT, smem, p, s);
+  if (stage == 2) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, NPT, ENV, 2>, grid, NT, smem, p, s);
+  if (stage == 1) return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, NPT, ENV, 1>, grid, NT, smem, p, s);
+  return launch_with_smem(actor_small_env_kernel<TE, NT, EPT, NPT, ENV, 0>, grid, NT, smem, p, s);
 }
 
 }  // namespace
@@ -434,13 +434,18 @@ cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s) {
     if (smem <= (st == 0 ? kSmemMax : kSmemTwoPerSm) || (st == 2 && smem <= kSmemMax && p.H <= 160)) { stage = st; break; }
     if (st == 0) return cudaErrorInvalidConfiguration;
   }
-  // Small N: 16 envs x 128 threads, 4 envs per thread (more warps; the problem is latency-bound).
-  // Large N: 32 envs x 256 threads, 8 envs per thread (each weight fetched feeds twice the FMAs).
-  if (env_kind == TJ_ENV_CARTPOLE)
-    return small_tile ? launch_small<16, 128, 4, TJ_ENV_CARTPOLE>(stage, smem, p, s)
-                      : launch_small<32, 256, 8, TJ_ENV_CARTPOLE>(stage, smem, p, s);
-  return small_tile ? launch_small<16, 128, 4, TJ_ENV_ACROBOT>(stage, smem, p, s)
-                    : launch_small<32, 256, 8, TJ_ENV_ACROBOT>(stage, smem, p, s);
+  // Small N: 16 envs x 128 threads, 4 envs x 4 neurons per thread (more warps; the problem is latency-bound).
+  // Large N: 32 envs per block, 8 envs per thread; wide layers (hidden >= 192) use 8 x 8 register tiles on 128
+  // threads (64 FMAs per four operand loads), narrower ones 4 neurons per thread on 256 threads.
+  const bool wide = p.H >= 192;
+  if (env_kind == TJ_ENV_CARTPOLE) {
+    if (small_tile) return launch_small<16, 128, 4, 4, TJ_ENV_CARTPOLE>(stage, smem, p, s);
+    if (wide) return launch_small<32, 128, 8, 8, TJ_ENV_CARTPOLE>(stage, smem, p, s);
+    return launch_small<32, 256, 8, 4, TJ_ENV_CARTPOLE>(stage, smem, p, s);
+  }
+  if (small_tile) return launch_small<16, 128, 4, 4, TJ_ENV_ACROBOT>(stage, smem, p, s);
+  if (wide) return launch_small<32, 128, 8, 8, TJ_ENV_ACROBOT>(stage, smem, p, s);
+  return launch_small<32, 256, 8, 4, TJ_ENV_ACROBOT>(stage, smem, p, s);
 }
 
 }  // namespace tj

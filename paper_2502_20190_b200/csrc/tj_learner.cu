@@ -158,7 +158,7 @@ __device__ __forceinline__ MlpWeights td_stage(const TdParams& p, const float* W
   return w;
 }
 
-template <int TE, int NT, int STAGE>
+template <int TE, int NT, int EPT, int NPT, int STAGE>
 __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   extern __shared__ __align__(128) float smem[];
   __shared__ __align__(8) uint64_t wbar;
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   }
   if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) return;
   __syncthreads();
-  mlp_forward_tile<TE, NT, 4, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < n_here) {
     int a = p.act[j0 + tid];
     a = a < 0 ? 0 : (a >= p.A ? p.A - 1 : a);
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   }
   if (STAGE > 0 && !mbar_wait_bounded(&wbar, 1)) return;
   __syncthreads();
-  mlp_forward_tile<TE, NT, 4, (STAGE > 0), (STAGE == 2)>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
+  mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < TE) {
     float h = 0.f;
     if (tid < n_here) {
@@ -311,31 +311,37 @@ cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s) {
 
 int td_grid(int n) { return (n + kTdTile - 1) / kTdTile; }
 
-template <int STAGE>
+template <int TE, int NT, int EPT, int NPT, int STAGE>
 cudaError_t launch_td_stage(const TdParams& p, size_t smem, int grid, cudaStream_t s) {
-  auto kernel = td_kernel<kTdTile, kTdThreads, STAGE>;
+  auto kernel = td_kernel<TE, NT, EPT, NPT, STAGE>;
   if (smem > 48 * 1024) {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
   }
-  kernel<<<grid, kTdThreads, smem, s>>>(p);
+  kernel<<<grid, NT, smem, s>>>(p);
   return cudaGetLastError();
 }
 
-cudaError_t launch_td(const TdParams& p, cudaStream_t s) {
-  constexpr int TE = kTdTile;
+// tile: 16 rows x 128 threads with 4 x 4 register tiles; wide layers (hidden >= 192) 32 rows x 128 threads, 8 x 8
+template <int TE, int NT, int EPT, int NPT>
+cudaError_t launch_td_tile(const TdParams& p, cudaStream_t s, int* grid_out) {
   const int Dx = (p.D + 3) & ~3;
   const size_t acts = (size_t)Dx * TE + 2 * (size_t)p.Hp * TE + (size_t)p.Ap * TE + 2 * TE;
   const size_t limit = 226 * 1024;
   const size_t smem2 = (acts + p.w_total) * sizeof(float);
   const size_t smem1 = (acts + p.w_total - (p.off_b2 - p.off_W2t)) * sizeof(float);
   const size_t smem0 = acts * sizeof(float);
-  const int grid = td_grid(p.n);
-  cudaError_t err;
-  if (smem2 <= 112 * 1024) err = launch_td_stage<2>(p, smem2, grid, s);
-  else if (smem1 <= limit) err = launch_td_stage<1>(p, smem1, grid, s);
-  else if (smem0 <= limit) err = launch_td_stage<0>(p, smem0, grid, s);
-  else return cudaErrorInvalidConfiguration;
+  const int grid = (p.n + TE - 1) / TE;
+  *grid_out = grid;
+  if (smem2 <= 112 * 1024) return launch_td_stage<TE, NT, EPT, NPT, 2>(p, smem2, grid, s);
+  if (smem1 <= limit) return launch_td_stage<TE, NT, EPT, NPT, 1>(p, smem1, grid, s);
+  if (smem0 <= limit) return launch_td_stage<TE, NT, EPT, NPT, 0>(p, smem0, grid, s);
+  return cudaErrorInvalidConfiguration;
+}
+
+cudaError_t launch_td(const TdParams& p, cudaStream_t s) {
+  int grid = 0;
+  cudaError_t err = p.H >= 192 ? launch_td_tile<32, 128, 8, 8>(p, s, &grid) : launch_td_tile<kTdTile, kTdThreads, 4, 4>(p, s, &grid);
   if (err != cudaSuccess) return err;
   if (p.loss_out) {
     td_finish_kernel<<<1, 32, 0, s>>>(p.partial, grid, p.n, p.loss_out);

@@ -36,44 +36,60 @@ __device__ __forceinline__ float load_w1(const float* p) {
 //   W_SMEM / B_SMEM: whether Wt / b sit in shared memory (else global, read-only path)
 //   EPT: environments per thread (4 or 8).  A thread owns EPT environments x 4 neurons; with 8 environments each
 //   weight fetched feeds twice as many FMAs, which is what shared-memory (or L2) bandwidth asks for.
-template <int TE, int NT, int EPT, int ACT, bool ENV_BIAS, bool W_SMEM, bool B_SMEM = W_SMEM>
+//   NPT: neurons per thread (4 or 8): 8 x 8 register tiles do 64 FMAs per two activation and two weight loads.
+template <int TE, int NT, int EPT, int ACT, bool ENV_BIAS, bool W_SMEM, bool B_SMEM = W_SMEM, int NPT = 4>
 __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const float* __restrict__ b, int ldw, int K,
                                             int n_out, const float* __restrict__ x, float* __restrict__ y,
                                             const int* __restrict__ bias_row) {
-  constexpr int EG = TE / EPT, NG = NT / EG, XV = EPT / 4;
+  constexpr int EG = TE / EPT, NG = NT / EG, XV = EPT / 4, WV = NPT / 4;
   const int eg = threadIdx.x % EG, ng = threadIdx.x / EG;
-  for (int i0 = ng * 4; i0 < n_out; i0 += NG * 4) {
-    float acc[4][EPT];  // [neuron][env]
-    if (ENV_BIAS) {
+  for (int i0 = ng * NPT; i0 < n_out; i0 += NG * NPT) {
+    float acc[NPT][EPT];  // [neuron][env]
+    bool wv_ok[WV];       // a thread's second group of four neurons may lie beyond the padded width
 #pragma unroll
-      for (int e = 0; e < EPT; ++e) {
-        const float4 bb = __ldg(reinterpret_cast<const float4*>(b + (size_t)bias_row[eg * EPT + e] * ldw + i0));
-        acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w;
+    for (int u = 0; u < WV; ++u) wv_ok[u] = i0 + 4 * u < ldw;
+#pragma unroll
+    for (int u = 0; u < WV; ++u) {
+      if (ENV_BIAS) {
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+          float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (wv_ok[u]) bb = __ldg(reinterpret_cast<const float4*>(b + (size_t)bias_row[eg * EPT + e] * ldw + i0 + 4 * u));
+          acc[4 * u][e] = bb.x; acc[4 * u + 1][e] = bb.y; acc[4 * u + 2][e] = bb.z; acc[4 * u + 3][e] = bb.w;
+        }
+      } else {
+        float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (wv_ok[u]) bb = load_w4<B_SMEM>(b + i0 + 4 * u);
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) {
+          acc[4 * u][e] = bb.x; acc[4 * u + 1][e] = bb.y; acc[4 * u + 2][e] = bb.z; acc[4 * u + 3][e] = bb.w;
+        }
       }
-    } else {
-      const float4 bb = load_w4<B_SMEM>(b + i0);
-#pragma unroll
-      for (int e = 0; e < EPT; ++e) { acc[0][e] = bb.x; acc[1][e] = bb.y; acc[2][e] = bb.z; acc[3][e] = bb.w; }
     }
     const float* xp = x + eg * EPT;
     const float* wp = Wt + i0;
 #pragma unroll 8
     for (int k = 0; k < K; ++k) {
-      float xe[EPT];
+      float xe[EPT], wn[NPT];
 #pragma unroll
       for (int v = 0; v < XV; ++v) {
         const float4 xv = *reinterpret_cast<const float4*>(xp + k * TE + 4 * v);
         xe[4 * v] = xv.x; xe[4 * v + 1] = xv.y; xe[4 * v + 2] = xv.z; xe[4 * v + 3] = xv.w;
       }
-      const float4 wv = load_w4<W_SMEM>(wp + (size_t)k * ldw);
-      const float wn[4] = {wv.x, wv.y, wv.z, wv.w};
 #pragma unroll
-      for (int n = 0; n < 4; ++n)
+      for (int u = 0; u < WV; ++u) {
+        float4 wv = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (wv_ok[u]) wv = load_w4<W_SMEM>(wp + (size_t)k * ldw + 4 * u);
+        wn[4 * u] = wv.x; wn[4 * u + 1] = wv.y; wn[4 * u + 2] = wv.z; wn[4 * u + 3] = wv.w;
+      }
+#pragma unroll
+      for (int n = 0; n < NPT; ++n)
 #pragma unroll
         for (int e = 0; e < EPT; ++e) acc[n][e] = fmaf(wn[n], xe[e], acc[n][e]);
     }
 #pragma unroll
-    for (int n = 0; n < 4; ++n)
+    for (int n = 0; n < NPT; ++n) {
+      if (!wv_ok[n / 4]) continue;
 #pragma unroll
       for (int v = 0; v < XV; ++v) {
         float4 o;
@@ -81,6 +97,7 @@ __device__ __forceinline__ void dense_layer(const float* __restrict__ Wt, const 
         o.z = activate<ACT>(acc[n][4 * v + 2]); o.w = activate<ACT>(acc[n][4 * v + 3]);
         *reinterpret_cast<float4*>(y + (size_t)(i0 + n) * TE + eg * EPT + 4 * v) = o;
       }
+    }
   }
 }
 
@@ -106,12 +123,12 @@ struct MlpWeights {
 
 // Policy forward for the tile: x [D][TE] -> h1 -> h2 -> out [Ap][TE]; ends with a barrier.
 // SMALL_SMEM: W1t, the biases and W3t are in shared memory;  W2_SMEM: W2t is too.
-template <int TE, int NT, int EPT, bool SMALL_SMEM, bool W2_SMEM>
+template <int TE, int NT, int EPT, bool SMALL_SMEM, bool W2_SMEM, int NPT = 4>
 __device__ __forceinline__ void mlp_forward_tile(const MlpWeights& w, int D, int H, int Hp, int Aout, int Ap,
                                                  const float* x, float* h1, float* h2, float* out) {
-  dense_layer<TE, NT, EPT, ACT_RELU, false, SMALL_SMEM>(w.W1t, w.b1, Hp, D, H, x, h1, nullptr);
+  dense_layer<TE, NT, EPT, ACT_RELU, false, SMALL_SMEM, SMALL_SMEM, NPT>(w.W1t, w.b1, Hp, D, H, x, h1, nullptr);
   __syncthreads();
-  dense_layer<TE, NT, EPT, ACT_RELU, false, W2_SMEM, SMALL_SMEM>(w.W2t, w.b2, Hp, H, H, h1, h2, nullptr);
+  dense_layer<TE, NT, EPT, ACT_RELU, false, W2_SMEM, SMALL_SMEM, NPT>(w.W2t, w.b2, Hp, H, H, h1, h2, nullptr);
   __syncthreads();
   if (Aout <= 8) head_layer<TE, NT, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out);
   else dense_layer<TE, NT, EPT, ACT_NONE, false, SMALL_SMEM>(w.W3t, w.b3, Ap, H, Aout, h2, out, nullptr);
