@@ -28,6 +28,10 @@ import numpy as np  # noqa: E402
 from paper_2502_20190_b200 import synth  # noqa: E402
 
 SM_COUNT, FMA_LANES_PER_SM = 148, 128
+# dram__bytes (read + write) per env-step of the fused tensor-core actor launch, from one ncu capture of the kernel as
+# it stands (113,664 envs: 185.8 MB per launch); traffic grows with the number of envs.  Set to None when the kernel
+# changes.  See profiles/cfg5_fused_tensor_core_actor.md.
+NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": 1634.6}
 L2_FLUSH_BYTES = 256 << 20
 
 
@@ -329,7 +333,9 @@ def run_ours(args):
                 "achieved": achieved, "peak": fma_peak, "unit": "TFLOP/s",
                 "peak_source": "FP32 FMA: 148 SMs x 128 lanes x 2 flop x max SM clock (derived, not measured)"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    per_env = NCU_DRAM_BYTES_PER_ENV_STEP.get(name) if dom == 1 else None
+    roof["traffic"] = per_env * N if per_env else None
+    roof["traffic_note"] = "bytes per fused actor launch (N env-steps), ncu capture at 113,664 envs scaled by N" if per_env else None
     roof["step_hbm_frac_of_measured"] = nbytes * units / (act_ms * 1e-3 / K) / 1e9 / peaks["hbm_gbs"]
     h2d, d2h = r.e2e_bytes()
     line = {
