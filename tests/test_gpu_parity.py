@@ -429,3 +429,24 @@ def test_bf16_tensor_core_actor_lockstep(env, D, H, A, N):
     assert np.all(np.abs(g_td - td) <= 2e-2 * (np.abs(qs) + np.abs(qn) + 2 * q_scale))
     assert abs(float(out["loss"].item()) - loss) <= 4e-2 * (abs(loss) + q_scale)
     assert ctx.stats()["device_error"] == 0
+
+
+def test_launch_counter_and_kernel_timing(env):
+    torch, orc, binding = env
+    f = _small()
+    ctx = binding.Context(**f)
+    ctx.publish_weights(blob_for(f, 1))
+    base = ctx.stats()["kernel_launches"]
+    assert base >= 1 and sum(ctx.stats()["kernel_count"]) == 0
+    ctx.set_profiling(1)
+    ctx.actor_step(3)
+    _, batch = ctx.replay_sample()
+    ctx.td_error(batch)
+    s = ctx.stats()
+    # one fused actor launch, eligible list + sample/gather, TD + loss reduction
+    assert s["kernel_launches"] - base == 1 + 2 + 2
+    assert s["kernel_count"][0] == 1 and s["kernel_count"][3] == 1 and s["kernel_count"][4] == 1
+    assert all(s["kernel_ms"][i] > 0 for i in (0, 3, 4))
+    ctx.set_profiling(0)
+    ctx.actor_step(1)
+    assert ctx.stats()["kernel_count"][0] == 1 and ctx.stats()["kernel_launches"] - base == 6
