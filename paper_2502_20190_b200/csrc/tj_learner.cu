@@ -129,6 +129,40 @@ __global__ void sample_gather_kernel(const SampleParams p) {
   if (lane == 0 && p.idx_out) p.idx_out[j] = slot;
 }
 
+// The same gather with 128-bit accesses (obs_dim a multiple of 4, 16-byte aligned outputs): LPD lanes share one
+// draw and copy the record's 16-byte chunks -- obs, next_obs, then the (act, rew, done, ver) tail.
+template <int LPD>
+__global__ void sample_gather_vec_kernel(const SampleParams p) {
+  const int lane = threadIdx.x & 31, sub = lane % LPD;
+  const int j = (int)((((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (32 / LPD)) + lane / LPD;
+  if (j >= p.B) return;
+  const unsigned long long nE = (unsigned long long)(*p.elig_count) * (unsigned long long)p.N;
+  const uint4 w = stream_words(p.seed, STREAM_SAMPLE, 0, (uint32_t)j, (unsigned long long)p.k);
+  const uint32_t r = __umulhi(w.x, (uint32_t)nE);
+  const int slot = p.elig_list[r / (uint32_t)p.N] * p.N + (int)(r % (uint32_t)p.N);
+  const float4* rec = reinterpret_cast<const float4*>(p.ring + (size_t)slot * p.rec_words);
+  const int dq = p.D / 4;                         // chunks per observation
+  float4* obs = reinterpret_cast<float4*>(p.obs + (size_t)j * p.D);
+  float4* nxt = reinterpret_cast<float4*>(p.next_obs + (size_t)j * p.D);
+  for (int c = sub; c <= 2 * dq; c += LPD) {
+    const float4 v = __ldcs(rec + c);             // sampled rows are not reused: streaming load
+    if (c < dq) obs[c] = v;
+    else if (c < 2 * dq) nxt[c - dq] = v;
+    else {
+      const int ver = __float_as_int(v.w);
+      p.act[j] = __float_as_int(v.x);
+      p.rew[j] = v.y;
+      p.done[j] = __float_as_int(v.z);
+      p.ver[j] = ver;
+      long long stale = p.v_learner - (long long)ver;
+      if (stale < 0) stale = 0;
+      atomicAdd(&p.stats->hist[stale > 32 ? 32 : stale], 1ull);
+      atomicMax(&p.stats->max_stale, (unsigned long long)stale);
+    }
+  }
+  if (sub == 0 && p.idx_out) p.idx_out[j] = slot;
+}
+
 // TD error on a tile of TE samples: online forward on obs, target forward on next_obs.
 // STAGE as in the actor kernel: 0 = parameters from global memory, 1 = all but the HxH matrix staged in shared
 // memory, 2 = all staged.  The staging buffer is filled twice (online, then target parameters).
@@ -305,6 +339,16 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s) {
   const int warps_per_block = 8;
+  const bool aligned = ((reinterpret_cast<uintptr_t>(p.obs) | reinterpret_cast<uintptr_t>(p.next_obs)) & 15) == 0;
+  if (p.D % 4 == 0 && aligned) {
+    if (p.rec_words <= 32) {      // a few chunks per record: four lanes per draw, eight draws per warp
+      const int draws_per_block = warps_per_block * 8;
+      sample_gather_vec_kernel<4><<<(p.B + draws_per_block - 1) / draws_per_block, warps_per_block * 32, 0, s>>>(p);
+    } else {
+      sample_gather_vec_kernel<32><<<(p.B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(p);
+    }
+    return cudaGetLastError();
+  }
   sample_gather_kernel<<<(p.B + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(p);
   return cudaGetLastError();
 }
