@@ -84,7 +84,7 @@ typedef struct {
   const float *host_lg_A;        /* LinGauss: A [D][D], HOST pointer, copied at create */
   const float *host_lg_B;        /* LinGauss: B [A][D], HOST pointer, copied at create */
   /* model group */
-  int32_t hidden;                /* H, width of both hidden ReLU layers */
+  int32_t hidden;                /* H, width of both hidden ReLU layers (1..768) */
   int32_t policy_kind;           /* TJ_POLICY_*: Q head, or softmax head + value head */
   int32_t weight_dtype;          /* TJ_W_FP32: FP32 FMA in a fixed rounding order; TJ_W_BF16: tensor cores */
   float epsilon;                 /* exploration rate (eps-greedy) */
@@ -167,8 +167,9 @@ int tj_destroy(tj_ctx *ctx);
 /* Learner -> actor hand-over of parameters (Sec. 3.1: the learner stores the model and a trigger decides
  * when to send it; dependency I as an asynchronous exchange).  `blob` holds FP32
  *   [W1 HxD, b1 H, W2 HxH, b2 H, W3 AxH, b3 A (, Wv 1xH, bv 1 when policy_kind = categorical)]
- * row-major (out x in); nbytes must match exactly.  on_device = 0: host pointer (copied before return);
- * 1: device pointer (read on the stream).  The new parameters become version+1 (returned in version_out)
+ * row-major (out x in); nbytes must match exactly.  on_device = 0: host pointer, copied with an asynchronous
+ * host-to-device copy on the stream (pageable memory is staged before the call returns; pinned memory must stay
+ * unchanged until the stream has passed the copy); 1: device pointer (read on the stream).  The new parameters become version+1 (returned in version_out)
  * and are what the actor uses from its next call and what the learner's online forward uses.  The target
  * network takes the same parameters on the first publish and then on the first publish after
  * target_sync_interval further learner steps.  With TJ_W_BF16 the weight matrices are rounded to bfloat16

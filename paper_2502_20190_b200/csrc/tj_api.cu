@@ -35,7 +35,7 @@ const char* validate(const tj_config* c) {
   if (!c) return "null config";
   if (c->struct_size != sizeof(tj_config)) return "struct_size does not match this library's tj_config";
   if (c->n_envs < 1) return "n_envs must be positive";
-  if (c->hidden < 1 || c->hidden > 4096) return "hidden out of range";
+  if (c->hidden < 1 || c->hidden > 768) return "hidden out of range (1..768: two activation tiles must fit in shared memory)";
   if (c->n_actions < 1 || c->n_actions > 64) return "n_actions out of range";
   switch (c->env_kind) {
     case TJ_ENV_CARTPOLE:
