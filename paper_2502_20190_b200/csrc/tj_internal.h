@@ -156,7 +156,6 @@ cudaError_t launch_init_env(int env_kind, int N, int S_d, uint2 seed, float* sta
 cudaError_t launch_pack_weights(const float* blob, float* dst, const WeightLayout& L, int value_head, int bf16,
                                 cudaStream_t s);
 cudaError_t launch_actor(int env_kind, const ActorParams& p, cudaStream_t s);
-size_t actor_td_scratch_floats(int n);
 cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_learner, long long bound, int* elig_list,
                             int* elig_count, cudaStream_t s);
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
