@@ -236,7 +236,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           // the head's weights arrive as one chunk: 16 rows x H columns
           const int s = it % TC_STAGES;
           if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
-          tc_fence_after();
           const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
           for (int j = 0; j < H / 16; ++j)
             umma_bf16(tmem, make_desc(smem_addr(abuf) + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, a_sbo), idesc,
@@ -248,7 +247,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
             for (int kc = 0; kc < K / TC_KC; ++kc, ++it) {
               const int s = it % TC_STAGES;
               if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
-              tc_fence_after();
               const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
               const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 8)) * 128u;
 #pragma unroll
@@ -273,7 +271,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
           for (int kc = 0; kc < ce; ++kc, ++it) {
             const int s = it % TC_STAGES;
             if (!tc_wait(&ctl->full[s], (it / TC_STAGES) & 1, abort_flag)) goto done;
-            tc_fence_after();
             const uint32_t b_base = smem_addr(ring + (size_t)s * TC_STAGE_BYTES);
             const uint32_t a_base = smem_addr(abuf) + (uint32_t)(kc * (TC_KC / 4)) * 128u;
 #pragma unroll
