@@ -127,6 +127,11 @@ size_t carve(tj_ctx* x, void* base) {
     x->lgA_hi = cv.take<uint32_t>((size_t)D * D);
     x->lgA_lo = cv.take<uint32_t>((size_t)D * D);
   }
+  x->use_tc_pipelined = x->use_tc_fused && tc_pipelined_supported(D, c.hidden, c.n_actions);
+  if (x->use_tc_pipelined) {
+    x->wtc_pipe[0] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
+    x->wtc_pipe[1] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
+  }
   return (cv.off + kAlign - 1) & ~(kAlign - 1);
 }
 
@@ -296,7 +301,7 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
       return cuda_fail(x, e, "publish: host to device copy");
     src = x->blob_stage;
   }
-  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc ? 2 : 1);
+  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : 1));
   const int next = x->active ^ 1;
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
   if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->stream)) != cudaSuccess)
@@ -306,6 +311,10 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
     dst_tc = x->version == 0 ? x->wtc[x->active] : x->wtc[next];
     if ((e = launch_pack_tc_weights(src, dst_tc, x->D, x->H, x->A, x->value_head, x->stream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: tensor-core repack");
+    if (x->use_tc_pipelined &&
+        (e = launch_pack_pipelined_weights(src, x->version == 0 ? x->wtc_pipe[x->active] : x->wtc_pipe[next], x->D, x->H, x->A,
+                                           x->stream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: tensor-core repack (pipelined actor)");
   }
   if (x->version != 0) x->active = next;
   x->version += 1;
@@ -370,7 +379,12 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
         ev.lgA_hi = x->lgA_hi; ev.lgA_lo = x->lgA_lo; ev.lgB = x->lgB;
         ev.noise_std = c.lg_noise_std; ev.done_norm = c.lg_done_norm; ev.stats = x->dstats;
         LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
-        e = launch_tc_mlp(t, x->sm_count, x->stream);
+        if (x->use_tc_pipelined) {
+          t.wtc = x->wtc_pipe[x->active];
+          e = launch_actor_tc_pipelined(t, x->sm_count, x->stream);
+        } else {
+          e = launch_tc_mlp(t, x->sm_count, x->stream);
+        }
         continue;
       }
       {

@@ -145,6 +145,10 @@ cudaError_t launch_pack_tc_weights(const float* blob, uint16_t* dst, int D, int 
 cudaError_t launch_tc_mlp(const TcMlpParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_pack_env_matrix(const float* A, uint32_t* hi, uint32_t* lo, int D, cudaStream_t s);
 bool tc_fused_supported(int D, int H, int A);
+// pipelined fused actor (obs_dim 128, hidden a multiple of 128): its own weight chunk order
+bool tc_pipelined_supported(int D, int H, int A);
+cudaError_t launch_pack_pipelined_weights(const float* blob, uint16_t* dst, int D, int H, int A, cudaStream_t s);
+cudaError_t launch_actor_tc_pipelined(const TcMlpParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
                              const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
                              cudaStream_t s);
@@ -204,6 +208,8 @@ struct tj_ctx {
   uint16_t* wtc_target;
   float* logits_buf;   // [N][A]
   bool use_tc_fused;
+  bool use_tc_pipelined;
+  uint16_t* wtc_pipe[2];   // weight chunks in the pipelined actor's order, double buffered like wtc
   uint32_t *lgA_hi, *lgA_lo;
   float* tdq[2];       // [kMaxTcTdRows][A] online / target outputs
   float *seg_obs, *seg_rew, *seg_logp, *seg_val;

@@ -18,9 +18,8 @@
 // accumulation, error ~2^-21 relative per term), and the epilogue threads finish the step: + B[a], tanh, Philox
 // noise, reward, done, record, reset, new state.
 // Every wait is bounded: on a timeout the block raises an abort flag, records an error, frees its TMEM and leaves.
-#include "tj_async.cuh"
-#include "tj_device.cuh"
 #include "tj_internal.h"
+#include "tj_tc.cuh"
 
 namespace tj {
 
@@ -35,103 +34,6 @@ constexpr int TC_EPI_THREADS = 128 * TC_SPLIT;
 constexpr int TC_THREADS = 64 + TC_EPI_THREADS;   // producer warp, MMA warp, 4 * TC_SPLIT epilogue warps
 constexpr int TC_KEEP = 32 / TC_SPLIT;            // float4 registers holding a thread's share of a 128-wide state row
 constexpr int TC_N3 = 16;        // head width on the tensor cores (outputs padded to 16)
-
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
-  return d;                 // base offset 0, no swizzle
-}
-
-// D = F32, A = B = BF16, both K-major, M = 128
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_M >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
-      : "memory");
-}
-
-// D = F32, A = B = TF32, both K-major, M = 128
-__device__ __forceinline__ uint32_t make_idesc_tf32(int n) {
-  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_M >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
-      : "memory");
-}
-
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// bounded wait that also gives up as soon as another role has raised the abort flag
-__device__ __forceinline__ bool tc_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < (1 << 22); ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63) == 63 && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
-}
-
-// Box-Muller pair with the hardware approximations (ex2/lg2/sin/cos units).  The noise enters the state scaled by
-// noise_std (0.01), so an absolute error of ~1e-6 in a normal is 1e-8 in the state, far inside the FP32 tolerance.
-__device__ __forceinline__ float2 box_muller_fast(uint32_t a, uint32_t b) {
-  const float r = sqrtf(-2.0f * __logf(u01(a)));
-  // angle 2*pi*u - pi lies in (-pi, pi) where the approximations are most accurate; cos/sin(theta) = -cos/sin(theta - pi)
-  const float th = fmaf(6.28318530717958647692f, u01(b), -3.14159265358979323846f);
-  float s, c;
-  __sincosf(th, &s, &c);
-  return make_float2(-r * c, -r * s);
-}
-
-// tanh(x) = 1 - 2 / (exp(2x) + 1) with the hardware exponential: absolute error ~2e-7 for the |x| that occur
-__device__ __forceinline__ float tanh_fast(float x) {
-  const float xc = fminf(fmaxf(x, -15.f), 15.f);
-  return 1.0f - __fdividef(2.0f, __expf(2.0f * xc) + 1.0f);
-}
-
-// for whole warps (the epilogue warps run warp-wide TMEM loads): every lane waits, and the warp leaves together
-__device__ __forceinline__ bool tc_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  const bool ok = tc_wait(bar, parity, abort_flag);
-  return __all_sync(0xffffffffu, ok);
-}
-
-// two FP32 values -> packed BF16 pair (round to nearest even), `lo` in the low half
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  uint32_t d;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-  return d;
-}
 
 // bytes of the A-operand buffer: the widest BF16 operand; in fused mode also the TF32 high+low state tile and
 // the FP32 staging rows of the stepped state
