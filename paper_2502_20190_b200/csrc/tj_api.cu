@@ -131,6 +131,7 @@ size_t carve(tj_ctx* x, void* base) {
   if (x->use_tc_pipelined) {
     x->wtc_pipe[0] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
     x->wtc_pipe[1] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
+    x->z_scratch = cv.take<float>(tc_pipelined_scratch_floats());
   }
   return (cv.off + kAlign - 1) & ~(kAlign - 1);
 }
@@ -381,6 +382,7 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
         LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
         if (x->use_tc_pipelined) {
           t.wtc = x->wtc_pipe[x->active];
+          ev.z_scratch = x->z_scratch;
           e = launch_actor_tc_pipelined(t, x->sm_count, x->stream);
         } else {
           e = launch_tc_mlp(t, x->sm_count, x->stream);

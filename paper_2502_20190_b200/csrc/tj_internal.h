@@ -127,6 +127,7 @@ struct TcEnvParams {
   const float* lgB;                  // [A][D]
   float noise_std, done_norm;
   DevStats* stats;
+  float* z_scratch;                  // pipelined actor: per thread block two tiles of z, [2][32][128][4] floats
 };
 
 struct TcMlpParams {
@@ -149,6 +150,7 @@ bool tc_fused_supported(int D, int H, int A);
 bool tc_pipelined_supported(int D, int H, int A);
 cudaError_t launch_pack_pipelined_weights(const float* blob, uint16_t* dst, int D, int H, int A, cudaStream_t s);
 cudaError_t launch_actor_tc_pipelined(const TcMlpParams& p, int sm_count, cudaStream_t s);
+size_t tc_pipelined_scratch_floats();   // z scratch for the largest grid the launcher uses
 cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
                              const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
                              cudaStream_t s);
@@ -210,6 +212,7 @@ struct tj_ctx {
   bool use_tc_fused;
   bool use_tc_pipelined;
   uint16_t* wtc_pipe[2];   // weight chunks in the pipelined actor's order, double buffered like wtc
+  float* z_scratch;
   uint32_t *lgA_hi, *lgA_lo;
   float* tdq[2];       // [kMaxTcTdRows][A] online / target outputs
   float *seg_obs, *seg_rew, *seg_logp, *seg_val;
