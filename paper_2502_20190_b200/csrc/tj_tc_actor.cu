@@ -28,9 +28,12 @@ namespace {
 constexpr int PA_M = 128;                  // rows per tile
 constexpr int PA_D = 128;                  // observation / state width this kernel is built for
 constexpr int PA_NB = 128;                 // neurons per accumulator block
-constexpr int PA_KC = 64;                  // K elements per weight chunk (128 x 64 BF16 = 16 KB)
-constexpr int PA_STAGES = 4;
-constexpr int PA_STAGE_BYTES = 16384;
+constexpr int PA_KC = 128;                 // K elements per weight chunk (128 x 128 BF16 = 32 KB)
+constexpr int PA_W_BYTES = PA_NB * PA_KC * 2;              // bytes of a hidden-layer weight chunk
+constexpr int PA_Z_BYTES = 16384;                          // bytes of an env-matrix chunk (128 x 32 TF32)
+constexpr int PA_STAGE_BYTES = PA_W_BYTES > PA_Z_BYTES ? PA_W_BYTES : PA_Z_BYTES;
+constexpr int PA_STAGES = 65536 / PA_STAGE_BYTES;
+constexpr uint32_t PA_B_SBO = (PA_KC / 8) * 128;           // bytes between 8-row groups of a weight chunk
 constexpr int PA_X_BYTES = PA_M * PA_D * 2;
 constexpr int PA_U_BYTES = 131072;
 constexpr int PA_THREADS = 640;            // warps 0-3: producer, MMA issuer, two idle; 4-11 network; 12-19 env
@@ -67,6 +70,9 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_tiles = (p.n + PA_M - 1) / PA_M;
   const int n_hb = H / PA_NB;            // 128-neuron blocks per hidden layer
+  // Thread blocks walk the neuron blocks of a layer in rotated order, so that at any moment they stream different
+  // parts of the weights from L2 (the arithmetic per neuron is unchanged)
+  const int rot = (int)(blockIdx.x % (unsigned)n_hb);
   const int n_kc2 = H / PA_KC;           // 64-wide K chunks of layer 2 (layer 1 has two)
 
   if (tid == 0) {
@@ -104,15 +110,19 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       // layer 2 (H/64 chunks per block), head
       uint32_t it = 0;
       const uint32_t head_bytes = (uint32_t)PA_N3 * H * 2;
-      const int n1 = n_hb * 2, n2 = n_hb * n_kc2;
+      const int n1 = n_hb * (PA_D / PA_KC), n2 = n_hb * n_kc2;
       for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
         for (int c = 0; c < n1 + 8 + n2 + 1; ++c, ++it) {
           const uint8_t* src;
-          uint32_t bytes = PA_STAGE_BYTES;
-          if (c < n1) src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)c * PA_STAGE_BYTES;
-          else if (c < n1 + 8) src = reinterpret_cast<const uint8_t*>(c - n1 < 4 ? ev.lgA_hi : ev.lgA_lo) + (size_t)((c - n1) & 3) * PA_STAGE_BYTES;
-          else if (c < n1 + 8 + n2) src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(c - 8) * PA_STAGE_BYTES;
-          else { src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(n1 + n2) * PA_STAGE_BYTES; bytes = head_bytes; }
+          uint32_t bytes = PA_W_BYTES;
+          constexpr int cpb1 = PA_D / PA_KC;
+          if (c < n1) src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(((c / cpb1 + rot) % n_hb) * cpb1 + c % cpb1) * PA_W_BYTES;
+          else if (c < n1 + 8) { src = reinterpret_cast<const uint8_t*>(c - n1 < 4 ? ev.lgA_hi : ev.lgA_lo) + (size_t)((c - n1) & 3) * PA_Z_BYTES; bytes = PA_Z_BYTES; }
+          else if (c < n1 + 8 + n2) {
+            const int idx = c - n1 - 8;
+            src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(n1 + ((idx / n_kc2 + rot) % n_hb) * n_kc2 + idx % n_kc2) * PA_W_BYTES;
+          }
+          else { src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(n1 + n2) * PA_W_BYTES; bytes = head_bytes; }
           const int s = it % PA_STAGES;
           if (!tc_wait(&ctl->empty[s], ((it / PA_STAGES) & 1) ^ 1, abort_flag)) goto done;
           mbar_expect_tx(&ctl->full[s], bytes);
@@ -141,14 +151,14 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           if (!acquire(u)) goto done;
           tc_fence_after();
           const uint32_t acc = tmem + ((u & 1) ? PA_COL_ACC1 : PA_COL_ACC0);
-          for (int c = 0; c < 2; ++c, ++it) {
+          for (int c = 0; c < PA_D / PA_KC; ++c, ++it) {
             const int s = it % PA_STAGES;
             if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
             const uint32_t b_base = smem_addr(ring + (size_t)s * PA_STAGE_BYTES);
             const uint32_t a_base = x_addr + (uint32_t)(c * (PA_KC / 8)) * 128u;
 #pragma unroll
             for (int j = 0; j < PA_KC / 16; ++j)
-              umma_bf16(acc, make_desc(a_base + j * 256u, 128u, 2048u), make_desc(b_base + j * 256u, 128u, 1024u), idesc_h,
+              umma_bf16(acc, make_desc(a_base + j * 256u, 128u, 2048u), make_desc(b_base + j * 256u, 128u, PA_B_SBO), idesc_h,
                         (c | j) != 0);
             umma_commit(&ctl->empty[s]);
           }
@@ -195,7 +205,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
             const uint32_t a_col = tmem + PA_COL_HB + (uint32_t)(c * (PA_KC / 2));
 #pragma unroll
             for (int j = 0; j < PA_KC / 16; ++j)
-              umma_bf16_ts(acc, a_col + (uint32_t)(j * 8), make_desc(b_base + j * 256u, 128u, 1024u), idesc_h, (c | j) != 0);
+              umma_bf16_ts(acc, a_col + (uint32_t)(j * 8), make_desc(b_base + j * 256u, 128u, PA_B_SBO), idesc_h, (c | j) != 0);
             umma_commit(&ctl->empty[s]);
           }
           umma_commit((u & 1) ? &ctl->acc_full[1] : &ctl->acc_full[0]);
@@ -249,45 +259,8 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       fence_async_smem();
       mbar_arrive_warp(&ctl->x_ready);
     };
-    // TF32 high / low parts of a tile's rows -> U (A operand of z = A s); the FP32 row is the record's observation
-    auto convert_u = [&](int tile) {
-#pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        const int rr = nw * 16 + g * 8 + c_r8;
-        const long long row = (long long)tile * PA_M + rr;
-        const bool live = row < p.n;
-        const float* xr = p.x + (size_t)(live ? row : 0) * D;
-        float4 v[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = live ? __ldg(reinterpret_cast<const float4*>(xr + (c_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        uint8_t* dhi = ubuf + ((size_t)(rr >> 3) * (D / 4)) * 128 + (rr & 7) * 16;
-        uint8_t* dlo = dhi + (size_t)PA_M * D * 4;
-        const unsigned long long slot = (ev.cursor + (unsigned long long)(live ? row : 0)) % (unsigned long long)ev.C;
-        float* rec = ev.ring + slot * ev.rec_words;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int k4 = c_kq + 4 * i;
-          const float4 sv = v[i];
-          float4 hi, lo;
-          hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
-          hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
-          hi.z = __uint_as_float(__float_as_uint(sv.z) & 0xFFFFE000u); lo.z = sv.z - hi.z;
-          hi.w = __uint_as_float(__float_as_uint(sv.w) & 0xFFFFE000u); lo.w = sv.w - hi.w;
-          *reinterpret_cast<float4*>(dhi + (size_t)k4 * 128) = hi;
-          *reinterpret_cast<float4*>(dlo + (size_t)k4 * 128) = lo;
-          if (live) *reinterpret_cast<float4*>(rec + k4 * 4) = sv;
-        }
-      }
-      fence_async_smem();
-      mbar_arrive_warp(&ctl->u_ready);
-    };
-    if ((int)blockIdx.x < n_tiles) {
-      convert_x(blockIdx.x);
-      convert_u(blockIdx.x);
-    }
+    if ((int)blockIdx.x < n_tiles) convert_x(blockIdx.x);
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tiles) {
-      const long long row = (long long)tile * PA_M + r;
-      const bool live = row < p.n;
       const int next_tile = tile + (int)gridDim.x;
       {
         // pull the rows of the tile after the next towards L2
@@ -324,23 +297,23 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           continue;
         }
         const int layer = u < n_hb ? 0 : 1;
-        const int b = layer == 0 ? u : u - n_hb - 1;
+        const int b = ((layer == 0 ? u : u - n_hb - 1) + rot) % n_hb;   // neuron block of this use
         const float* bias = layer == 0 ? p.b1 : p.b2;
         const int c0 = b * PA_NB + hsel * 64;          // first of this thread's 64 columns
+        uint32_t v[64];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) tmem_ld16(t_acc + (uint32_t)(g * 16), v + 16 * g);
+        tmem_ld_wait();
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
-          uint32_t v[32];
-          tmem_ld16(t_acc + (uint32_t)(hh * 32), v);
-          tmem_ld16(t_acc + (uint32_t)(hh * 32 + 16), v + 16);
-          tmem_ld_wait();
           uint32_t o[16];
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
             const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + c0 + hh * 32 + 4 * j4));
-            const float f0 = fmaxf(__uint_as_float(v[4 * j4 + 0]) + bb.x, 0.f);
-            const float f1 = fmaxf(__uint_as_float(v[4 * j4 + 1]) + bb.y, 0.f);
-            const float f2 = fmaxf(__uint_as_float(v[4 * j4 + 2]) + bb.z, 0.f);
-            const float f3 = fmaxf(__uint_as_float(v[4 * j4 + 3]) + bb.w, 0.f);
+            const float f0 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 0]) + bb.x, 0.f);
+            const float f1 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 1]) + bb.y, 0.f);
+            const float f2 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 2]) + bb.z, 0.f);
+            const float f3 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 3]) + bb.w, 0.f);
             o[2 * j4] = pack_bf16x2(f0, f1);
             o[2 * j4 + 1] = pack_bf16x2(f2, f3);
           }
@@ -358,11 +331,6 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         tc_fence_before();
         mbar_arrive_warp(&ctl->acc_empty[buf]);
       }
-      if (next_tile < n_tiles) {
-        // U is read by this tile's head until it completes
-        if (!tc_wait_elect(&ctl->head_full, tiles & 1, abort_flag)) goto done;
-        convert_u(next_tile);
-      }
     }
   } else {
     // ------------------------------------------------------------------ env warps
@@ -370,6 +338,39 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
     const int ew = warp - 12;                      // 0..7; the first four also read the head outputs (one TMEM quarter each)
     const int e_r8 = lane >> 2, e_kq = lane & 3;   // env step: eight rows x four 16-byte pieces per warp instruction
     uint32_t tiles = 0;
+    // TF32 high / low parts of a tile's rows -> U (A operand of z = A s); the FP32 row is the record's observation
+    auto convert_u = [&](int tile) {
+#pragma unroll
+      for (int g = 0; g < 2; ++g) {
+        const int rr = ew * 16 + g * 8 + e_r8;
+        const long long row = (long long)tile * PA_M + rr;
+        const bool live = row < p.n;
+        const float* xr = p.x + (size_t)(live ? row : 0) * D;
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = live ? __ldg(reinterpret_cast<const float4*>(xr + (e_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        uint8_t* dhi = ubuf + ((size_t)(rr >> 3) * (D / 4)) * 128 + (rr & 7) * 16;
+        uint8_t* dlo = dhi + (size_t)PA_M * D * 4;
+        const unsigned long long slot = (ev.cursor + (unsigned long long)(live ? row : 0)) % (unsigned long long)ev.C;
+        float* rec = ev.ring + slot * ev.rec_words;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int k4 = e_kq + 4 * i;
+          const float4 sv = v[i];
+          float4 hi, lo;
+          hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
+          hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
+          hi.z = __uint_as_float(__float_as_uint(sv.z) & 0xFFFFE000u); lo.z = sv.z - hi.z;
+          hi.w = __uint_as_float(__float_as_uint(sv.w) & 0xFFFFE000u); lo.w = sv.w - hi.w;
+          *reinterpret_cast<float4*>(dhi + (size_t)k4 * 128) = hi;
+          *reinterpret_cast<float4*>(dlo + (size_t)k4 * 128) = lo;
+          if (live) *reinterpret_cast<float4*>(rec + k4 * 4) = sv;
+        }
+      }
+      fence_async_smem();
+      mbar_arrive_warp(&ctl->u_ready);
+    };
+    if ((int)blockIdx.x < n_tiles) convert_u(blockIdx.x);
     unsigned long long n_episodes = 0;
     double ret_sum = 0.0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tiles) {
@@ -403,7 +404,10 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         mbar_arrive_warp(&ctl->act_ready);
       } else {
         mbar_arrive_warp(&ctl->env_taken);         // this warp has finished the previous tile
+        if (!tc_wait_elect(&ctl->head_full, tiles & 1, abort_flag)) goto done;
       }
+      // the head of this tile is complete, so U is free: the next tile's TF32 parts go in before this tile's env step
+      if (tile + (int)gridDim.x < n_tiles) convert_u(tile + (int)gridDim.x);
       if (!tc_wait_elect(&ctl->act_ready, tiles & 1, abort_flag)) goto done;
       // z was stored long before the head finished; the wait orders the loads below after those stores
       if (!tc_wait_elect(&ctl->z_stored, tiles & 1, abort_flag)) goto done;
