@@ -28,10 +28,10 @@ import numpy as np  # noqa: E402
 from paper_2502_20190_b200 import synth  # noqa: E402
 
 SM_COUNT, FMA_LANES_PER_SM = 148, 128
-# dram__bytes (read + write) per env-step of the fused tensor-core actor launch, from one ncu capture of the kernel as
-# it stands (113,664 envs: 185.8 MB per launch); traffic grows with the number of envs.  Set to None when the kernel
-# changes.  See profiles/cfg5_fused_tensor_core_actor.md.
-NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": 1634.6}
+# dram__bytes (read + write) per env-step of the pipelined tensor-core actor launch, from one ncu capture of the kernel as
+# it stands (113,664 envs: 1.318 TB/s over 188.9 us = 249.0 MB per launch); traffic grows with the number of envs.  Set to
+# None when the kernel changes.  See profiles/cfg5_pipelined_tensor_core_actor.md.
+NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": 2190.7}
 L2_FLUSH_BYTES = 256 << 20
 
 
@@ -312,7 +312,8 @@ def run_ours(args):
     if dom == 1:      # tensor-core MLP: actor launches process N rows, learner launches B rows (two per step)
         rows = K * (r.actor_steps * N + 2 * w["minibatch"])
         achieved = mlp_flops * rows / (kms[1] * 1e-3) / 1e12
-        roof = {"kernel": "mlp_bf16_tc_kernel (tcgen05 MLP forward)", "bound": "tensor", "achieved": achieved,
+        roof = {"kernel": "actor_tc_pipelined_kernel (fused tcgen05 actor step; the TD forwards of mlp_bf16_tc_kernel share the class)",
+                "bound": "tensor", "achieved": achieved,
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "peak_source": "cuBLAS bf16 sustained, of " + peaks["source"]}
     elif dom == 2:    # selection + env step + insert: state read twice (obs) + written, record written, outputs read
