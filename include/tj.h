@@ -217,7 +217,9 @@ int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_
  *   - every call, from every context on the device, shares the one array.  Each call rewrites the part it
  *     reads, so nothing needs clearing between calls, but two calls that overlap on the GPU (different
  *     streams) race on it: keep them on one stream or order them with events;
- *   - results equal tj_td_error's (same kernels, same summation order). */
+ *   - in an FP32 context the results equal tj_td_error's (same kernels, same summation order); in a BF16 context this
+ *     call still runs the FP32 kernels on the BF16-rounded weights, so it agrees with tj_td_error's tensor-core
+ *     result within the BF16 tolerance only. */
 int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
 
 /* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
