@@ -394,7 +394,7 @@ def test_categorical_actions_follow_the_margin_rule(env):
 
 # ------------------------------------------------------------------------------------------------ tensor cores
 @pytest.mark.parametrize("D,H,A,N", [(128, 512, 16, 300), (64, 64, 5, 130), (128, 320, 16, 128), (32, 256, 16, 257),
-                                     (128, 256, 16, 300), (128, 128, 7, 200)])
+                                     (128, 256, 16, 300), (128, 128, 7, 200), (128, 384, 9, 140)])
 def test_bf16_tensor_core_actor_lockstep(env, D, H, A, N):
     """BF16 weights on the tcgen05 path: network outputs within 2e-2 of the oracle (BF16-rounded weights, double
     accumulation), actions exact outside the oracle's top-2 margin, the selection rule exact on the GPU's own
