@@ -281,6 +281,28 @@ def td_one(q_sel, q_next_max, r, done, gamma, kappa):
     return float(td.value), float(hub.value)
 
 
+def sgd_step(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, gamma, kappa, lr):
+    """One minibatch update of Algorithm 1's form (semi-gradient of the mean Huber loss); returns (theta_new, loss)."""
+    theta = np.ascontiguousarray(theta, np.float32)
+    theta_target = np.ascontiguousarray(theta_target, np.float32)
+    obs = np.ascontiguousarray(obs, np.float32)
+    next_obs = np.ascontiguousarray(next_obs, np.float32)
+    act = np.ascontiguousarray(act, np.int32)
+    done = np.ascontiguousarray(done, np.int32)
+    rew = np.ascontiguousarray(rew, np.float32)
+    n = act.size
+    assert theta.size == blob_floats(D, H, A) == theta_target.size and obs.size == n * D == next_obs.size
+    out = np.zeros_like(theta)
+    loss = C.c_double()
+    fn = lib().orc_sgd_step
+    fn.restype = None
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                   C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_void_p, C.c_void_p]
+    fn(_p(theta), _p(theta_target), D, H, A, _p(obs), _p(act), _p(rew), _p(next_obs), _p(done), n, float(gamma),
+       float(kappa), float(lr), _p(out), C.byref(loss))
+    return out, loss.value
+
+
 def gae(rew, val, done, gamma, lam):
     rew = np.ascontiguousarray(rew, np.float32)
     val = np.ascontiguousarray(val, np.float32)

@@ -314,6 +314,84 @@ void orc_td_one(double q_sel, double q_next_max, double r, int done, double gamm
 }
 
 /* ===================================================================== */
+/* Learner update (Algorithm 1: theta <- theta + alpha * delta * grad V(s; theta)), as one minibatch step:   */
+/*   L(theta) = mean_j Huber(delta_j),  delta_j = r_j + gamma (1 - done_j) max_a Q(s'_j, a; theta_target)     */
+/*                                               - Q(s_j, a_j; theta)                                         */
+/*   theta <- theta - lr * dL/dtheta, the target term held constant (semi-gradient).                          */
+/* dHuber/ddelta = clip(delta, -kappa, kappa), so dL/dQ(s_j, a_j) = -clip(delta_j) / n: with kappa = inf,     */
+/* n = 1 and theta_target = theta this is Algorithm 1's update line.  Everything in double from the FP32      */
+/* inputs; the new parameters are rounded to FP32 once, at the end.                                           */
+/* ===================================================================== */
+void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                  const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
+                  double kappa, double lr, float *theta_out, double *loss_mean) {
+  const size_t nW1 = (size_t)H * D, nW2 = (size_t)H * H, nW3 = (size_t)A * H;
+  const size_t o_b1 = nW1, o_W2 = o_b1 + H, o_b2 = o_W2 + nW2, o_W3 = o_b2 + H, o_b3 = o_W3 + nW3, total = o_b3 + A;
+  double *grad = (double *)calloc(total, sizeof(double));
+  double *h1 = (double *)malloc(sizeof(double) * H), *h2 = (double *)malloc(sizeof(double) * H);
+  double *dh1 = (double *)malloc(sizeof(double) * H), *dh2 = (double *)malloc(sizeof(double) * H);
+  double *qn = (double *)malloc(sizeof(double) * A);
+  const float *W1 = theta, *b1 = theta + o_b1, *W2 = theta + o_W2, *b2 = theta + o_b2, *W3 = theta + o_W3, *b3 = theta + o_b3;
+  double loss = 0.0;
+  for (int j = 0; j < n; ++j) {
+    const float *x = obs + (size_t)j * D;
+    int a = act[j];
+    if (a < 0) a = 0;
+    if (a >= A) a = A - 1;
+    /* online forward, activations kept */
+    for (int i = 0; i < H; ++i) {
+      double s = (double)b1[i];
+      for (int k = 0; k < D; ++k) s += (double)W1[(size_t)i * D + k] * (double)x[k];
+      h1[i] = s > 0.0 ? s : 0.0;
+    }
+    for (int i = 0; i < H; ++i) {
+      double s = (double)b2[i];
+      for (int k = 0; k < H; ++k) s += (double)W2[(size_t)i * H + k] * h1[k];
+      h2[i] = s > 0.0 ? s : 0.0;
+    }
+    double q = (double)b3[a];
+    for (int k = 0; k < H; ++k) q += (double)W3[(size_t)a * H + k] * h2[k];
+    /* target: max over the target network's outputs at the next observation */
+    orc_mlp_forward_f64(theta_target, D, H, A, 0, next_obs + (size_t)j * D, qn, NULL);
+    double qmax = qn[0];
+    for (int i = 1; i < A; ++i)
+      if (qn[i] > qmax) qmax = qn[i];
+    double delta, hub;
+    orc_td_one(q, qmax, (double)rew[j], done[j], gamma, kappa, &delta, &hub);
+    loss += hub;
+    /* dL/dq = -clip(delta, -kappa, kappa) / n */
+    double c = delta > kappa ? kappa : (delta < -kappa ? -kappa : delta);
+    const double g = -c / (double)n;
+    /* head row a */
+    grad[o_b3 + a] += g;
+    for (int k = 0; k < H; ++k) {
+      grad[o_W3 + (size_t)a * H + k] += g * h2[k];
+      dh2[k] = h2[k] > 0.0 ? g * (double)W3[(size_t)a * H + k] : 0.0;
+    }
+    /* layer 2 */
+    for (int k = 0; k < H; ++k) dh1[k] = 0.0;
+    for (int i = 0; i < H; ++i) {
+      if (dh2[i] == 0.0) continue;
+      grad[o_b2 + i] += dh2[i];
+      for (int k = 0; k < H; ++k) {
+        grad[o_W2 + (size_t)i * H + k] += dh2[i] * h1[k];
+        dh1[k] += dh2[i] * (double)W2[(size_t)i * H + k];
+      }
+    }
+    /* layer 1 */
+    for (int i = 0; i < H; ++i) {
+      const double d = h1[i] > 0.0 ? dh1[i] : 0.0;
+      if (d == 0.0) continue;
+      grad[o_b1 + i] += d;
+      for (int k = 0; k < D; ++k) grad[(size_t)i * D + k] += d * (double)x[k];
+    }
+  }
+  for (size_t i = 0; i < total; ++i) theta_out[i] = (float)((double)theta[i] - lr * grad[i]);
+  if (loss_mean) *loss_mean = loss / (double)n;
+  free(grad); free(h1); free(h2); free(dh1); free(dh2); free(qn);
+}
+
+/* ===================================================================== */
 /* GAE: delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;                      */
 /*      A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0; R_t = A_t + V_t */
 /* arrays are time-major: rew[T][N], val[T+1][N], done[T][N]              */

@@ -111,6 +111,11 @@ int orc_select_categorical(const float *logits, int A, float u, double *logp, do
 
 void orc_td_one(double q_sel, double q_next_max, double r, int done, double gamma, double kappa, double *td,
                 double *huber);
+/* Algorithm 1's update line as one minibatch semi-gradient step on the mean Huber loss; theta blobs in the layout above
+ * (no value head); theta_out may not alias theta */
+void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                  const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
+                  double kappa, double lr, float *theta_out, double *loss_mean);
 void orc_gae(const float *rew, const float *val, const uint8_t *done, int T, int N, double gamma, double lambda,
              double *adv, double *ret);
 
