@@ -67,7 +67,9 @@ enum { TJ_K_ACTOR_FUSED = 0,  /* MLP + selection + env step + insert in one kern
        TJ_K_ENV = 2,          /* selection + env step + insert fed by the tensor-core MLP */
        TJ_K_SAMPLE = 3,       /* eligible list + sample + gather */
        TJ_K_TD = 4,           /* TD error (FP32 forward, or the elementwise pass after tensor-core forwards) */
-       TJ_K_PUBLISH = 5, TJ_K_GAE = 6, TJ_KERNEL_CLASSES = 8 };
+       TJ_K_PUBLISH = 5, TJ_K_GAE = 6,
+       TJ_K_SGD = 7,          /* learner update: forward with kept activations, backward, parameter update */
+       TJ_KERNEL_CLASSES = 8 };
 
 /* Configuration (App. B: one configuration with distribution / training / model / environment groups). */
 typedef struct {
@@ -221,6 +223,17 @@ int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_
  *     call still runs the FP32 kernels on the BF16-rounded weights, so it agrees with tj_td_error's tensor-core
  *     result within the BF16 tolerance only. */
 int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
+
+/* Learner, step 2, update half (Algorithm 1: theta <- theta + alpha * delta * grad V(s; theta)) as one minibatch
+ * semi-gradient step on the mean Huber loss of tj_td_error:
+ *   L = mean_j Huber(delta_j; huber_delta),  delta_j = r_j + gamma (1 - done_j) max_a Q(s'_j, a; theta_target) - Q(s_j, a_j; theta)
+ *   theta <- theta - lr * dL/dtheta   (the target term is a constant; dHuber/ddelta = clip(delta, -huber_delta, huber_delta))
+ * With huber_delta = inf, one row and theta_target = theta this is Algorithm 1's update line.
+ * theta (in/out) and theta_target: device FP32 blobs in the tj_publish_weights layout, distinct buffers, owned by the
+ * caller; nothing in the context changes -- publish theta afterwards to hand it to the actor.  batch.n <= the configured
+ * minibatch.  loss_mean_out (nullable, device): the loss before the update.  FP32 arithmetic, every sum in a fixed order.
+ * TJ_ERR_UNSUPPORTED for BF16 contexts, segment mode and the categorical policy. */
+int tj_sgd_step(tj_ctx *ctx, const tj_batch *batch, float lr, float *theta, const float *theta_target, float *loss_mean_out);
 
 /* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
  *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0;

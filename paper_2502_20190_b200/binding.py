@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
            "tj_last_error")
 
 
@@ -89,6 +89,7 @@ def load_library():
     L.tj_td_error.argtypes = [vp, vp, vp, vp, vp]
     L.tj_td_error_static.argtypes = [vp, vp, vp, vp, vp]
     L.tj_gae.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
+    L.tj_sgd_step.argtypes = [vp, vp, f32, vp, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
@@ -148,6 +149,11 @@ def tj_td_error(h, batch: TjBatch, td_ptr: int, huber_ptr: int, loss_ptr: int):
 def tj_td_error_static(h, batch: TjBatch, td_ptr: int, huber_ptr: int, loss_ptr: int):
     """tj_td_error with the reduction scratch inside the library image (at most 65,536 rows; allocates nothing)."""
     return load_library().tj_td_error_static(h, C.byref(batch), td_ptr or None, huber_ptr or None, loss_ptr or None)
+
+
+def tj_sgd_step(h, batch: TjBatch, lr: float, theta_ptr: int, theta_target_ptr: int, loss_ptr: int):
+    """One learner update (Algorithm 1's update line as a minibatch semi-gradient step) on device blobs, in place."""
+    return load_library().tj_sgd_step(h, C.byref(batch), lr, theta_ptr, theta_target_ptr, loss_ptr or None)
 
 
 def tj_gae(h, rew_ptr, val_ptr, done_ptr, T, N, gamma, lam, adv_ptr, ret_ptr):
@@ -317,6 +323,15 @@ class Context:
         self._check(tj_td_error(self.h, batch["c"], out["td"].data_ptr(), out["huber"].data_ptr(),
                                 out["loss"].data_ptr()))
         return out
+
+    def sgd_step(self, batch, lr, theta, theta_target):
+        """theta (updated in place) and theta_target: float32 device tensors in the publish layout; returns the loss tensor"""
+        torch = self.torch
+        assert theta.dtype == torch.float32 and theta_target.dtype == torch.float32
+        assert theta.is_contiguous() and theta_target.is_contiguous() and theta.numel() == theta_target.numel()
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        self._check(tj_sgd_step(self.h, batch["c"], float(lr), theta.data_ptr(), theta_target.data_ptr(), loss.data_ptr()))
+        return loss
 
     def gae(self, rew, val, done, gamma, lam, adv=None, ret=None):
         torch = self.torch

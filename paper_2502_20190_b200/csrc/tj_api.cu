@@ -98,6 +98,12 @@ size_t carve(tj_ctx* x, void* base) {
     x->block_ver = cv.take<int>(nb);
     x->elig_list = cv.take<int>(nb);
     x->elig_count = cv.take<int>(1);
+    x->sgd_rows = 0;
+    x->sgd_scratch = nullptr;
+    if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_EPS_GREEDY && sgd_supported(D, c.hidden, c.n_actions)) {
+      x->sgd_rows = c.minibatch;
+      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(c.minibatch, c.hidden));
+    }
   } else {
     const size_t TN = (size_t)c.rollout_len * N, G = c.n_segments;
     x->seg_obs = cv.take<float>(G * TN * D);
@@ -532,6 +538,29 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
     return fail(x, TJ_ERR_INVALID_ARG, msg);
   }
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error (library scratch)");
+  return TJ_OK;
+}
+
+int tj_sgd_step(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
+  if (!theta || !theta_target) return fail(x, TJ_ERR_INVALID_ARG, "parameter blobs must not be null");
+  if (theta == theta_target) return fail(x, TJ_ERR_INVALID_ARG, "theta and theta_target must be different buffers");
+  if (!(lr >= 0.f)) return fail(x, TJ_ERR_INVALID_ARG, "lr must not be negative");
+  if (!x->sgd_scratch) return fail(x, TJ_ERR_UNSUPPORTED, "the learner update is implemented for FP32 replay contexts with the Q head");
+  if (b->n < 1 || b->n > x->sgd_rows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be between 1 and the configured minibatch");
+  SgdParams p{};
+  p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A;
+  p.theta = theta; p.theta_target = theta_target;
+  p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
+  p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
+  const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
+  p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH; p.g = p.dh2 + RH; p.partial = p.g + rows;
+  LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 8 : 7);
+  cudaError_t e = launch_sgd_step(p, lr, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
+  if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
+    return cuda_fail(x, e, "learner update (loss reduction)");
   return TJ_OK;
 }
 

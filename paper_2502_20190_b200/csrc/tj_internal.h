@@ -93,6 +93,21 @@ struct TdParams {
   float* partial;  // scratch: one float per thread block
 };
 
+struct SgdParams {
+  int n, D, H, A;
+  float* theta;                // online parameters, publish layout, updated in place
+  const float* theta_target;   // target parameters, same layout
+  const float* obs;
+  const int* act;
+  const float* rew;
+  const float* next_obs;
+  const int* done;
+  float gamma, kappa;
+  float *h1, *h2, *dh1, *dh2;  // scratch [n][H] each
+  float* g;                    // scratch [n]: dL/dq of the selected action
+  float* partial;              // scratch: one Huber partial sum per 16 rows
+};
+
 struct SampleParams {
   int B, D, N, rec_words;
   uint2 seed;
@@ -167,6 +182,10 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
 cudaError_t launch_td(const TdParams& p, cudaStream_t s);
 int td_grid(int n);
+size_t sgd_scratch_floats(int max_rows, int H);
+int sgd_partial_count(int n);
+bool sgd_supported(int D, int H, int A);
+cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s);
 int td_static_max_rows();
 cudaError_t launch_td_static(const TdParams& p, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
@@ -199,6 +218,8 @@ struct tj_ctx {
   int* elig_list;
   int* elig_count;
   float* td_partial;
+  float* sgd_scratch;   // learner update: activations and their gradients for one minibatch (FP32 replay contexts)
+  int sgd_rows;         // rows the scratch holds
   tj::DevStats* dstats;
   float* lgAt;
   float* lgB;

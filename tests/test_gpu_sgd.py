@@ -1,0 +1,111 @@
+"""GPU parity for the learner update (tj_sgd_step) against the oracle's orc_sgd_step.
+
+The two sides get the same parameter blobs and the same minibatch (sampled by the GPU context from its own ring, whose
+contents are parity-checked elsewhere).  Compared: the parameter *change* per group and the loss.  Tolerance: the GPU
+accumulates each gradient entry over the n rows in FP32 (n sequential fused multiply-adds, error <= n * 2^-24 of the sum of
+term magnitudes in the worst case, ~sqrt(n) * 2^-24 typically), the oracle in double; 1e-5 relative to each entry plus
+1e-5 of the group's rms covers n up to a few thousand with the inputs used here, and is the FP32 tolerance of every other
+test."""
+import numpy as np
+import pytest
+
+from parity_util import RTOL_FP32, blob_for, close, fields_for
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import oracle
+    from paper_2502_20190_b200 import binding, build
+    build.build()
+    oracle.build()
+    return torch, oracle, binding
+
+
+def _groups(D, H, A):
+    n1, n2, n3 = H * D, H * H, A * H
+    names = ["W1", "b1", "W2", "b2", "W3", "b3"]
+    sizes = [n1, H, n2, H, n3, A]
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    return [(names[i], int(offs[i]), int(offs[i + 1])) for i in range(6)]
+
+
+@pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (1, 6, 3, 96, 50, 333), (2, 16, 5, 200, 40, 77),
+                                            (0, 4, 2, 256, 128, 1024)])
+def test_sgd_step_matches_oracle(env, kind, D, A, H, N, B):
+    torch, orc, binding = env
+    f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, epsilon=0.3, seed=777, replay_capacity=N * 16,
+                   minibatch=B, staleness_bound=20, warmup=N, target_sync_interval=1000, gamma=0.99, huber_delta=1.0,
+                   max_episode_steps=9)
+    ctx = binding.Context(**f)
+    theta_t = blob_for(f, 1)            # the first publish also becomes the target
+    theta = blob_for(f, 2)
+    ctx.publish_weights(theta_t)
+    ctx.actor_step(6)
+    ctx.publish_weights(theta)
+    ctx.actor_step(6)
+    _, batch = ctx.replay_sample()
+    dev = ctx.device
+    th = torch.from_numpy(theta.copy()).to(dev)
+    tt = torch.from_numpy(theta_t.copy()).to(dev)
+    lr = 0.05
+    loss = ctx.sgd_step(batch, lr, th, tt)
+    torch.cuda.synchronize()
+    g_new = th.cpu().numpy()
+    o_new, o_loss = orc.sgd_step(theta, theta_t, D, H, A, batch["obs"].cpu().numpy(), batch["act"].cpu().numpy(),
+                                 batch["rew"].cpu().numpy(), batch["next_obs"].cpu().numpy(), batch["done"].cpu().numpy(),
+                                 0.99, 1.0, lr)
+    assert np.array_equal(tt.cpu().numpy(), theta_t)                        # the target blob is read only
+    assert abs(float(loss.item()) - o_loss) <= 2 * RTOL_FP32 * (abs(o_loss) + 1e-3)
+    dg = g_new.astype(np.float64) - theta.astype(np.float64)
+    do = o_new.astype(np.float64) - theta.astype(np.float64)
+    # the FP32 rounding of theta_new itself (half an ulp of theta, on both sides) is part of the comparison floor
+    ulp = np.spacing(np.abs(theta).astype(np.float32)).astype(np.float64)
+    for name, a, b in _groups(D, H, A):
+        assert np.abs(do[a:b]).max() > 0, name                               # every group moves
+        rms = np.sqrt(np.mean(do[a:b] ** 2))
+        err = np.abs(dg[a:b] - do[a:b])
+        bound = RTOL_FP32 * np.abs(do[a:b]) + RTOL_FP32 * rms + ulp[a:b]
+        assert np.all(err <= bound), "%s: worst %.3e over bound %.3e" % (name, err.max(), bound[np.argmax(err - bound)])
+    # a second step from the updated parameters stays on the oracle's trajectory
+    loss2 = ctx.sgd_step(batch, lr, th, tt)
+    o_new2, o_loss2 = orc.sgd_step(o_new, theta_t, D, H, A, batch["obs"].cpu().numpy(), batch["act"].cpu().numpy(),
+                                   batch["rew"].cpu().numpy(), batch["next_obs"].cpu().numpy(), batch["done"].cpu().numpy(),
+                                   0.99, 1.0, lr)
+    assert abs(float(loss2.item()) - o_loss2) <= 1e-4 * (abs(o_loss2) + 1e-3)
+    close(th.cpu().numpy(), o_new2, 1e-4, "theta after two steps")
+    assert ctx.stats()["device_error"] == 0
+
+
+def test_sgd_step_argument_checks(env):
+    torch, orc, binding = env
+    f = fields_for(env_kind=0, n_envs=32, obs_dim=4, n_actions=2, hidden=32, epsilon=0.1, seed=5, replay_capacity=32 * 8,
+                   minibatch=64, staleness_bound=8, warmup=32, target_sync_interval=10, gamma=0.99, huber_delta=1.0)
+    ctx = binding.Context(**f)
+    blob = blob_for(f, 1)
+    ctx.publish_weights(blob)
+    ctx.actor_step(4)
+    _, batch = ctx.replay_sample()
+    th = torch.from_numpy(blob.copy()).to(ctx.device)
+    st = binding.tj_sgd_step(ctx.h, batch["c"], 0.1, th.data_ptr(), th.data_ptr(), 0)
+    assert st == binding.TJ_ERR_INVALID_ARG                                  # theta and target must differ
+    big = ctx.alloc_batch(65)
+    tt = th.clone()
+    st = binding.tj_sgd_step(ctx.h, big["c"], 0.1, th.data_ptr(), tt.data_ptr(), 0)
+    assert st == binding.TJ_ERR_INVALID_ARG and "minibatch" in binding.tj_last_error(ctx.h)
+    # lr = 0 leaves the parameters untouched
+    before = th.clone()
+    ctx.sgd_step(batch, 0.0, th, tt)
+    assert torch.equal(before, th)
+    # a BF16 context refuses the call
+    f2 = fields_for(env_kind=2, n_envs=128, obs_dim=32, n_actions=4, hidden=64, epsilon=0.1, seed=5, replay_capacity=128 * 4,
+                    minibatch=64, staleness_bound=8, warmup=128, target_sync_interval=10, gamma=0.99, huber_delta=1.0,
+                    weight_dtype=1)
+    c2 = binding.Context(**f2)
+    b2 = c2.alloc_batch(8)
+    st = binding.tj_sgd_step(c2.h, b2["c"], 0.1, th.data_ptr(), tt.data_ptr(), 0)
+    assert st == binding.TJ_ERR_UNSUPPORTED
