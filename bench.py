@@ -135,7 +135,7 @@ def aggregate_throughput(units_per_replica, world, max_ms):
 class Runner:
     """Drives one context through the workload's call pattern."""
 
-    def __init__(self, name, torch, binding, device_index, n_envs=0):
+    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False):
         self.torch, self.name = torch, name
         self.w = dict(synth.WORKLOADS[name])
         if n_envs:
@@ -155,6 +155,13 @@ class Runner:
         self.host_blobs = [torch.from_numpy(b).pin_memory() for b in blobs]
         self.version = 0
         self.learner_ok = 0
+        # --with-update: the learner also takes a gradient step (tj_sgd_step) and the published parameters are the ones it
+        # trains, instead of the pre-drawn pool (FP32 replay workloads only)
+        self.with_update = bool(with_update) and self.w["replay_capacity"] > 0 and self.w["weight_dtype"] == synth.W_FP32
+        if self.with_update:
+            self.theta = self.dev_blobs[0].clone()
+            self.theta_target = self.dev_blobs[0].clone()
+            self.lr = 1e-3
         if not self.on_policy:
             self.batch = self.ctx.alloc_batch()
             B = self.w["minibatch"]
@@ -171,6 +178,12 @@ class Runner:
         self.publish(False)
 
     def publish(self, from_host):
+        if self.with_update:
+            self.ctx.publish_weights(self.theta)
+            self.version += 1
+            if self.version % 1000 == 0:
+                self.theta_target.copy_(self.theta)
+            return
         blob = (self.host_blobs if from_host else self.dev_blobs)[self.version % self.n_pool]
         if from_host:
             from paper_2502_20190_b200 import binding as b
@@ -193,6 +206,8 @@ class Runner:
             st, _ = self.ctx.replay_sample(batch=self.batch, allow=(0, -6, -7))
             if st == 0:
                 self.ctx.td_error(self.batch, self.out)
+                if self.with_update:
+                    self.ctx.sgd_step(self.batch, self.lr, self.theta, self.theta_target)
                 self.learner_ok += 1
 
     def step(self, events=None, e2e=False):
@@ -217,7 +232,7 @@ class Runner:
             events[3].record()
 
     def e2e_bytes(self):
-        h2d = self.host_blobs[0].numel() * 4
+        h2d = 0 if self.with_update else self.host_blobs[0].numel() * 4
         d2h = 4 if self.on_policy else (self.w["minibatch"] + 1) * 4
         return h2d, d2h
 
@@ -243,7 +258,7 @@ def run_ours(args):
     peaks = load_peaks()
     name = args.workload
     w = synth.WORKLOADS[name]
-    r = Runner(name, torch, binding, local, args.envs)
+    r = Runner(name, torch, binding, local, args.envs, args.with_update)
     w = r.w
     N = w["n_envs"]
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
@@ -299,7 +314,7 @@ def run_ours(args):
     consumed = (w["rollout_len"] * N if r.on_policy else w["minibatch"]) * learner_ok * world
     value = env_steps / (tot_ms * 1e-3)
     flops, nbytes = actor_algorithmic(w)
-    names = ["actor_fused", "mlp_tensor", "env_select_insert", "sample_gather", "td", "publish", "gae"]
+    names = ["actor_fused", "mlp_tensor", "env_select_insert", "sample_gather", "td", "publish", "gae", "sgd_update"]
     kms, kcnt = prof["kernel_ms"], prof["kernel_count"]
     total_kms = sum(kms) or 1.0
     kernels = {names[i]: {"launches": kcnt[i], "ms": kms[i], "share": kms[i] / total_kms} for i in range(len(names)) if kcnt[i]}
@@ -345,7 +360,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "bf16" if w["weight_dtype"] == synth.W_BF16 else "f32", "data": "synthetic",
         "config": {"workload": name, "n_envs": N, "actor_steps_per_step": r.actor_steps,
                    "minibatch": w.get("minibatch"), "mlp": "%d-%d-%d-%d" % (w["obs_dim"], w["hidden"], w["hidden"], w["n_actions"]),
-                   "replicas": world,
+                   "replicas": world, "learner_update": r.with_update,
                    "l2": "flushed between steps (256 MiB write outside the per-step event pairs)" if need_flush
                    else "ring larger than L2"},
         "consumed_samples_per_s": consumed / (tot_ms * 1e-3),
@@ -470,6 +485,7 @@ def main():
     ap.add_argument("--workload", default="cfg5", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--envs", type=int, default=0, help="profiling aid: run the workload with this many envs (ring scaled to the same number of steps)")
+    ap.add_argument("--with-update", action="store_true", help="FP32 replay workloads: the learner step also runs tj_sgd_step and publishes the parameters it trains")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()

@@ -555,8 +555,8 @@ int tj_sgd_step(tj_ctx* x, const tj_batch* b, float lr, float* theta, const floa
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
-  p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH; p.g = p.dh2 + RH; p.partial = p.g + rows;
-  LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 8 : 7);
+  p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH; p.g = p.dh2 + RH; p.partial = p.g + rows * 16; p.grad_partial = p.partial + rows / 16 + 64;
+  LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 15 : 14);
   cudaError_t e = launch_sgd_step(p, lr, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
   if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)

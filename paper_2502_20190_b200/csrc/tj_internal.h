@@ -104,8 +104,9 @@ struct SgdParams {
   const int* done;
   float gamma, kappa;
   float *h1, *h2, *dh1, *dh2;  // scratch [n][H] each
-  float* g;                    // scratch [n]: dL/dq of the selected action
+  float* g;                    // scratch [n][A]: dL/dq, non-zero at the selected action only
   float* partial;              // scratch: one Huber partial sum per 16 rows
+  float* grad_partial;         // scratch: per row range partial sums of one gradient matrix
 };
 
 struct SampleParams {

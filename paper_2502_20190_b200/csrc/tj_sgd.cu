@@ -15,35 +15,49 @@ namespace {
 constexpr int SG_ROWS = 16;       // minibatch rows per thread block in the forward and backward kernels
 constexpr int SG_THREADS = 256;
 
+constexpr int SG_KT = 32;         // K columns of the weight tile staged in shared memory
+
 // one dense layer for SG_ROWS rows at once: out[i][r] = (relu)(b[i] + sum_k W[i][k] in[k][r]); activations live in shared
-// memory k-major, so a step of the inner loop is one weight times 16 broadcast values
+// memory k-major, so a step of the inner loop is one weight times 16 broadcast values.  The weights (row-major out x in)
+// pass through a 256 x 32 shared-memory tile so that the global loads run along k, 128 contiguous bytes per row.
 template <bool RELU>
 __device__ __forceinline__ void sg_dense(const float* __restrict__ W, const float* __restrict__ b, int n_out, int n_in,
-                                         const float* in, float* out) {
-  for (int i = threadIdx.x; i < n_out; i += SG_THREADS) {
+                                         const float* in, float* out, float* wt) {
+  for (int i0 = 0; i0 < n_out; i0 += SG_THREADS) {
+    const int i = i0 + threadIdx.x;
     float acc[SG_ROWS];
-    const float bi = b[i];
+    const float bi = i < n_out ? b[i] : 0.f;
 #pragma unroll
     for (int r = 0; r < SG_ROWS; ++r) acc[r] = bi;
-    const float* w = W + (size_t)i * n_in;
-    for (int k = 0; k < n_in; ++k) {
-      const float wk = __ldg(w + k);
-      const float4* a = reinterpret_cast<const float4*>(in + (size_t)k * SG_ROWS);
+    for (int k0 = 0; k0 < n_in; k0 += SG_KT) {
+      __syncthreads();
+      for (int t = threadIdx.x; t < SG_THREADS * SG_KT; t += SG_THREADS) {
+        const int ii = t / SG_KT, kk = t % SG_KT;
+        wt[ii * (SG_KT + 1) + kk] = (i0 + ii < n_out && k0 + kk < n_in) ? __ldg(W + (size_t)(i0 + ii) * n_in + k0 + kk) : 0.f;
+      }
+      __syncthreads();
+      const int kn = n_in - k0 < SG_KT ? n_in - k0 : SG_KT;
+      for (int kk = 0; kk < kn; ++kk) {
+        const float wk = wt[threadIdx.x * (SG_KT + 1) + kk];
+        const float4* a = reinterpret_cast<const float4*>(in + (size_t)(k0 + kk) * SG_ROWS);
 #pragma unroll
-      for (int r4 = 0; r4 < SG_ROWS / 4; ++r4) {
-        const float4 v = a[r4];
-        acc[4 * r4 + 0] = fmaf(wk, v.x, acc[4 * r4 + 0]);
-        acc[4 * r4 + 1] = fmaf(wk, v.y, acc[4 * r4 + 1]);
-        acc[4 * r4 + 2] = fmaf(wk, v.z, acc[4 * r4 + 2]);
-        acc[4 * r4 + 3] = fmaf(wk, v.w, acc[4 * r4 + 3]);
+        for (int r4 = 0; r4 < SG_ROWS / 4; ++r4) {
+          const float4 v = a[r4];
+          acc[4 * r4 + 0] = fmaf(wk, v.x, acc[4 * r4 + 0]);
+          acc[4 * r4 + 1] = fmaf(wk, v.y, acc[4 * r4 + 1]);
+          acc[4 * r4 + 2] = fmaf(wk, v.z, acc[4 * r4 + 2]);
+          acc[4 * r4 + 3] = fmaf(wk, v.w, acc[4 * r4 + 3]);
+        }
       }
     }
+    if (i < n_out) {
 #pragma unroll
-    for (int r = 0; r < SG_ROWS; ++r) out[(size_t)i * SG_ROWS + r] = RELU ? fmaxf(acc[r], 0.f) : acc[r];
+      for (int r = 0; r < SG_ROWS; ++r) out[(size_t)i * SG_ROWS + r] = RELU ? fmaxf(acc[r], 0.f) : acc[r];
+    }
   }
 }
 
-// shared memory: xs [D][16] | a1 [H][16] | a2 [H][16] | qs [A][16]
+// shared memory: xs [D][16] | a1 [H][16] | a2 [H][16] | qs [A][16] | weight tile [256][33]
 __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams p) {
   extern __shared__ __align__(16) float sg_sm[];
   const int D = p.D, H = p.H, A = p.A;
@@ -51,6 +65,7 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
   float* a1 = xs + (size_t)D * SG_ROWS;
   float* a2 = a1 + (size_t)H * SG_ROWS;
   float* qs = a2 + (size_t)H * SG_ROWS;
+  float* wt = qs + (size_t)A * SG_ROWS;
   __shared__ float qsel[SG_ROWS], hub[SG_ROWS];
   const int row0 = blockIdx.x * SG_ROWS;
   const float *W1 = p.theta, *b1 = W1 + (size_t)H * D, *W2 = b1 + H, *b2 = W2 + (size_t)H * H, *W3 = b2 + H, *b3 = W3 + (size_t)A * H;
@@ -62,11 +77,11 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
     xs[i] = row0 + r < p.n ? p.obs[(size_t)(row0 + r) * D + k] : 0.f;
   }
   __syncthreads();
-  sg_dense<true>(W1, b1, H, D, xs, a1);
+  sg_dense<true>(W1, b1, H, D, xs, a1, wt);
   __syncthreads();
-  sg_dense<true>(W2, b2, H, H, a1, a2);
+  sg_dense<true>(W2, b2, H, H, a1, a2, wt);
   __syncthreads();
-  sg_dense<false>(W3, b3, A, H, a2, qs);
+  sg_dense<false>(W3, b3, A, H, a2, qs, wt);
   for (int i = threadIdx.x; i < H * SG_ROWS; i += SG_THREADS) {
     const int k = i / SG_ROWS, r = i % SG_ROWS;
     if (row0 + r < p.n) {
@@ -87,11 +102,11 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
     xs[i] = row0 + r < p.n ? p.next_obs[(size_t)(row0 + r) * D + k] : 0.f;
   }
   __syncthreads();
-  sg_dense<true>(T1, tb1, H, D, xs, a1);
+  sg_dense<true>(T1, tb1, H, D, xs, a1, wt);
   __syncthreads();
-  sg_dense<true>(T2, tb2, H, H, a1, a2);
+  sg_dense<true>(T2, tb2, H, H, a1, a2, wt);
   __syncthreads();
-  sg_dense<false>(T3, tb3, A, H, a2, qs);
+  sg_dense<false>(T3, tb3, A, H, a2, qs, wt);
   __syncthreads();
   if (threadIdx.x < SG_ROWS) {
     const int r = threadIdx.x, j = row0 + r;
@@ -102,7 +117,10 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
       const float y = p.rew[j] + p.gamma * (p.done[j] ? 0.f : 1.f) * qmax;
       const float delta = y - qsel[r], ad = fabsf(delta);
       h = ad <= p.kappa ? 0.5f * delta * delta : p.kappa * (ad - 0.5f * p.kappa);
-      p.g[j] = -fminf(fmaxf(delta, -p.kappa), p.kappa) / (float)p.n;
+      const float gj = -fminf(fmaxf(delta, -p.kappa), p.kappa) / (float)p.n;
+      int a = p.act[j];
+      a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+      for (int i = 0; i < A; ++i) p.g[(size_t)j * A + i] = i == a ? gj : 0.f;
     }
     hub[r] = h;
   }
@@ -128,7 +146,7 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_backward_kernel(const SgdParam
     const int j = row0 + threadIdx.x;
     int a = j < p.n ? p.act[j] : 0;
     as[threadIdx.x] = a < 0 ? 0 : (a >= A ? A - 1 : a);
-    gs[threadIdx.x] = j < p.n ? p.g[j] : 0.f;
+    gs[threadIdx.x] = j < p.n ? p.g[(size_t)j * A + as[threadIdx.x]] : 0.f;
   }
   __syncthreads();
   // dh2[r][i] = g_r W3[a_r][i] where h2 > 0
@@ -165,20 +183,26 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_backward_kernel(const SgdParam
   }
 }
 
-// C[m][n] -= lr * sum_j A[j][m] * Bm[j][n]   (C row-major M x N; A n_rows x M with row stride lda; Bm n_rows x N, stride ldb)
-// 32 x 32 tile per block, 256 threads, each 2 x 2; rows j in ascending order
-__global__ void __launch_bounds__(256) sgd_update_matrix_kernel(float* __restrict__ Cm, int M, int N, const float* __restrict__ Am,
-                                                                int lda, const float* __restrict__ Bm, int ldb, int n_rows,
-                                                                float lr) {
+constexpr int SG_SPLITS = 32;     // at most this many row ranges per gradient product (partial sums go through scratch)
+
+// P[z][m][n] = sum over the rows j of range z of A[j][m] * Bm[j][n]   (A n_rows x M with row stride lda; Bm n_rows x N,
+// stride ldb; Bm == nullptr stands for a column of ones, N = 1: a bias gradient).  32 x 32 tile per block, 256 threads,
+// each 2 x 2; rows in ascending order.  The row ranges (blockIdx.z) make the reduction over the minibatch parallel; the
+// second kernel adds the partial sums in range order, so the result does not depend on the launch.
+__global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, int M, int N, const float* __restrict__ Am,
+                                                               int lda, const float* __restrict__ Bm, int ldb, int n_rows,
+                                                               int rows_per_range) {
   __shared__ float As[32][33], Bs[32][33];
   const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int j_begin = blockIdx.z * rows_per_range;
+  const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
   float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-  for (int j0 = 0; j0 < n_rows; j0 += 32) {
+  for (int j0 = j_begin; j0 < j_end; j0 += 32) {
     for (int i = threadIdx.x; i < 32 * 32; i += 256) {
       const int jj = i >> 5, c = i & 31, j = j0 + jj;
-      As[jj][c] = (j < n_rows && m0 + c < M) ? Am[(size_t)j * lda + m0 + c] : 0.f;
-      Bs[jj][c] = (j < n_rows && n0 + c < N) ? Bm[(size_t)j * ldb + n0 + c] : 0.f;
+      As[jj][c] = (j < j_end && m0 + c < M) ? Am[(size_t)j * lda + m0 + c] : 0.f;
+      Bs[jj][c] = (j < j_end && n0 + c < N) ? (Bm ? Bm[(size_t)j * ldb + n0 + c] : 1.f) : 0.f;
     }
     __syncthreads();
 #pragma unroll 8
@@ -196,55 +220,38 @@ __global__ void __launch_bounds__(256) sgd_update_matrix_kernel(float* __restric
 #pragma unroll
     for (int v = 0; v < 2; ++v) {
       const int m = m0 + ty + 16 * u, n = n0 + tx + 16 * v;
-      if (m < M && n < N) Cm[(size_t)m * N + n] -= lr * acc[u][v];
+      if (m < M && n < N) P[((size_t)blockIdx.z * M + m) * N + n] = acc[u][v];
     }
 }
 
-// b[m] -= lr * sum_j A[j][m]
-__global__ void sgd_update_bias_kernel(float* __restrict__ b, int M, const float* __restrict__ Am, int lda, int n_rows, float lr) {
-  const int m = blockIdx.x * blockDim.x + threadIdx.x;
-  if (m >= M) return;
+// C[i] -= lr * (P[0][i] + P[1][i] + ...), the partial sums added in range order
+__global__ void sgd_apply_kernel(float* __restrict__ Cm, const float* __restrict__ P, int count, int n_ranges, float lr) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
   float s = 0.f;
-  for (int j = 0; j < n_rows; ++j) s += Am[(size_t)j * lda + m];
-  b[m] -= lr * s;
-}
-
-// head: W3[a][i] -= lr * sum_{j: a_j = a} g_j h2[j][i];  b3[a] -= lr * sum_{j: a_j = a} g_j.   grid (ceil(H/128), A)
-__global__ void sgd_update_head_kernel(const SgdParams p, float lr) {
-  const int H = p.H, A = p.A, a = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
-  float* W3 = p.theta + (size_t)H * p.D + H + (size_t)H * H + H;
-  float* b3 = W3 + (size_t)A * H;
-  float s = 0.f, sb = 0.f;
-  for (int j = 0; j < p.n; ++j) {
-    int aj = p.act[j];
-    aj = aj < 0 ? 0 : (aj >= A ? A - 1 : aj);
-    if (aj != a) continue;
-    const float g = p.g[j];
-    sb += g;
-    if (i < H) s = fmaf(g, p.h2[(size_t)j * H + i], s);
-  }
-  if (i < H) W3[(size_t)a * H + i] -= lr * s;
-  if (i == 0) b3[a] -= lr * sb;
+  for (int z = 0; z < n_ranges; ++z) s += P[(size_t)z * count + i];
+  Cm[i] -= lr * s;
 }
 
 }  // namespace
 
 size_t sgd_scratch_floats(int max_rows, int H) {
   const size_t rows = ((size_t)max_rows + SG_ROWS - 1) / SG_ROWS * SG_ROWS;
-  return 4 * rows * (size_t)H + rows + rows / SG_ROWS + 64;
+  // h1, h2, dh1, dh2, g [rows][<= 16 actions], Huber partials, partial gradient sums of the largest matrix
+  return 4 * rows * (size_t)H + rows * 16 + rows / SG_ROWS + 64 + (size_t)SG_SPLITS * H * (size_t)(H > 16 ? H : 16);
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }
 
 bool sgd_supported(int D, int H, int A) {
-  const size_t smem = ((size_t)D + 2 * (size_t)H + A) * SG_ROWS * sizeof(float);
-  return H >= 1 && D >= 1 && A >= 1 && smem <= 200 * 1024;
+  const size_t smem = (((size_t)D + 2 * (size_t)H + A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
+  return H >= 1 && D >= 1 && A >= 1 && A <= 16 && smem <= 200 * 1024;
 }
 
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s) {
   const int D = p.D, H = p.H, A = p.A;
   const int grid = sgd_partial_count(p.n);
-  const size_t smem_f = ((size_t)D + 2 * (size_t)H + A) * SG_ROWS * sizeof(float);
+  const size_t smem_f = (((size_t)D + 2 * (size_t)H + A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
   const size_t smem_b = (size_t)H * SG_ROWS * sizeof(float);
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(sgd_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f)) != cudaSuccess) return e;
@@ -255,12 +262,25 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s) {
   float* b1 = W1 + (size_t)H * D;
   float* W2 = b1 + H;
   float* b2 = W2 + (size_t)H * H;
-  // the backward pass has read W2 and W3; now the parameters may change
-  sgd_update_head_kernel<<<dim3((H + 127) / 128, A), 128, 0, s>>>(p, lr);
-  sgd_update_matrix_kernel<<<dim3((H + 31) / 32, (H + 31) / 32), 256, 0, s>>>(W2, H, H, p.dh2, H, p.h1, H, p.n, lr);
-  sgd_update_bias_kernel<<<(H + 127) / 128, 128, 0, s>>>(b2, H, p.dh2, H, p.n, lr);
-  sgd_update_matrix_kernel<<<dim3((D + 31) / 32, (H + 31) / 32), 256, 0, s>>>(W1, H, D, p.dh1, H, p.obs, D, p.n, lr);
-  sgd_update_bias_kernel<<<(H + 127) / 128, 128, 0, s>>>(b1, H, p.dh1, H, p.n, lr);
+  float* W3 = b2 + H;
+  float* b3 = W3 + (size_t)A * H;
+  // the backward pass has read W2 and W3; now the parameters may change.  Every update is the same product:
+  // C -= lr * (gradient rows)^T (input rows), the bias with a column of ones as input
+  int n_ranges = (p.n + 127) / 128;
+  if (n_ranges > SG_SPLITS) n_ranges = SG_SPLITS;
+  const int rows_per_range = ((p.n + n_ranges - 1) / n_ranges + 31) / 32 * 32;
+  n_ranges = (p.n + rows_per_range - 1) / rows_per_range;
+  auto upd = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
+    sgd_grad_partial_kernel<<<dim3((N + 31) / 32, (M + 31) / 32, n_ranges), 256, 0, s>>>(p.grad_partial, M, N, Am, lda, Bm, ldb, p.n,
+                                                                                       rows_per_range);
+    sgd_apply_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, p.grad_partial, M * N, n_ranges, lr);
+  };
+  upd(W3, A, H, p.g, A, p.h2, H);
+  upd(b3, A, 1, p.g, A, nullptr, 0);
+  upd(W2, H, H, p.dh2, H, p.h1, H);
+  upd(b2, H, 1, p.dh2, H, nullptr, 0);
+  upd(W1, H, D, p.dh1, H, p.obs, D);
+  upd(b1, H, 1, p.dh1, H, nullptr, 0);
   return cudaGetLastError();
 }
 
