@@ -235,6 +235,14 @@ int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float 
  * TJ_ERR_UNSUPPORTED for BF16 contexts, segment mode and the categorical policy. */
 int tj_sgd_step(tj_ctx *ctx, const tj_batch *batch, float lr, float *theta, const float *theta_target, float *loss_mean_out);
 
+/* The same gradient through Adam (the optimiser of Table 2; Kingma & Ba 2015), step counter t >= 1:
+ *   m <- beta1 m + (1 - beta1) g;  v <- beta2 v + (1 - beta2) g^2;
+ *   theta <- theta - lr * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+ * m, v: device FP32 moment blobs in the layout of theta, owned and zero-initialised by the caller, updated in place.
+ * Other arguments, limits and statuses as tj_sgd_step. */
+int tj_adam_step(tj_ctx *ctx, const tj_batch *batch, float lr, float beta1, float beta2, float eps, int64_t t, float *theta,
+                 const float *theta_target, float *m, float *v, float *loss_mean_out);
+
 /* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
  *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0;
  *   R_t = A_t + V_t.   rew [T][N], val [T+1][N], done [T][N] -> adv [T][N], ret [T][N].

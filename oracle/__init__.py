@@ -303,6 +303,27 @@ def sgd_step(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, gamma,
     return out, loss.value
 
 
+def adam_step(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, gamma, kappa, lr, beta1, beta2, eps, t, m, v):
+    """The gradient of sgd_step through Adam; returns (theta_new, m_new, v_new, loss)."""
+    arrs = [np.ascontiguousarray(a, np.float32) for a in (theta, theta_target, obs, rew, next_obs, m, v)]
+    theta, theta_target, obs, rew, next_obs, m, v = arrs
+    act = np.ascontiguousarray(act, np.int32)
+    done = np.ascontiguousarray(done, np.int32)
+    n = act.size
+    assert theta.size == blob_floats(D, H, A) == theta_target.size == m.size == v.size and obs.size == n * D
+    t_out, m_out, v_out = np.zeros_like(theta), np.zeros_like(theta), np.zeros_like(theta)
+    loss = C.c_double()
+    fn = lib().orc_adam_step
+    fn.restype = None
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                   C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int64,
+                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    fn(_p(theta), _p(theta_target), D, H, A, _p(obs), _p(act), _p(rew), _p(next_obs), _p(done), n, float(gamma),
+       float(kappa), float(lr), float(beta1), float(beta2), float(eps), int(t), _p(m), _p(v), _p(t_out), _p(m_out),
+       _p(v_out), C.byref(loss))
+    return t_out, m_out, v_out, loss.value
+
+
 def gae(rew, val, done, gamma, lam):
     rew = np.ascontiguousarray(rew, np.float32)
     val = np.ascontiguousarray(val, np.float32)

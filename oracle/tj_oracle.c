@@ -322,12 +322,13 @@ void orc_td_one(double q_sel, double q_next_max, double r, int done, double gamm
 /* n = 1 and theta_target = theta this is Algorithm 1's update line.  Everything in double from the FP32      */
 /* inputs; the new parameters are rounded to FP32 once, at the end.                                           */
 /* ===================================================================== */
-void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
-                  const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
-                  double kappa, double lr, float *theta_out, double *loss_mean) {
+/* grad[i] = dL/dtheta_i (double, caller-allocated, orc_blob_floats entries); returns the mean Huber loss */
+static double td_loss_gradient(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                               const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n,
+                               double gamma, double kappa, double *grad) {
   const size_t nW1 = (size_t)H * D, nW2 = (size_t)H * H, nW3 = (size_t)A * H;
   const size_t o_b1 = nW1, o_W2 = o_b1 + H, o_b2 = o_W2 + nW2, o_W3 = o_b2 + H, o_b3 = o_W3 + nW3, total = o_b3 + A;
-  double *grad = (double *)calloc(total, sizeof(double));
+  for (size_t i = 0; i < total; ++i) grad[i] = 0.0;
   double *h1 = (double *)malloc(sizeof(double) * H), *h2 = (double *)malloc(sizeof(double) * H);
   double *dh1 = (double *)malloc(sizeof(double) * H), *dh2 = (double *)malloc(sizeof(double) * H);
   double *qn = (double *)malloc(sizeof(double) * A);
@@ -386,9 +387,43 @@ void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, i
       for (int k = 0; k < D; ++k) grad[(size_t)i * D + k] += d * (double)x[k];
     }
   }
+  free(h1); free(h2); free(dh1); free(dh2); free(qn);
+  return loss / (double)n;
+}
+
+
+void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                  const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
+                  double kappa, double lr, float *theta_out, double *loss_mean) {
+  const size_t total = (size_t)orc_blob_floats(D, H, A, 0);
+  double *grad = (double *)malloc(total * sizeof(double));
+  const double loss = td_loss_gradient(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, n, gamma, kappa, grad);
   for (size_t i = 0; i < total; ++i) theta_out[i] = (float)((double)theta[i] - lr * grad[i]);
-  if (loss_mean) *loss_mean = loss / (double)n;
-  free(grad); free(h1); free(h2); free(dh1); free(dh2); free(qn);
+  if (loss_mean) *loss_mean = loss;
+  free(grad);
+}
+
+/* The same gradient fed to Adam (Kingma & Ba 2015; the optimiser of Table 2), step counter t >= 1:                   */
+/*   m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;  theta <- theta - lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps) */
+/* m and v are FP32 state blobs like theta (read from m, v; written to m_out, v_out), arithmetic in double.            */
+void orc_adam_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                   const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
+                   double kappa, double lr, double beta1, double beta2, double eps, int64_t t, const float *m, const float *v,
+                   float *theta_out, float *m_out, float *v_out, double *loss_mean) {
+  const size_t total = (size_t)orc_blob_floats(D, H, A, 0);
+  double *grad = (double *)malloc(total * sizeof(double));
+  const double loss = td_loss_gradient(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, n, gamma, kappa, grad);
+  const double c1 = 1.0 - pow(beta1, (double)t), c2 = 1.0 - pow(beta2, (double)t);
+  for (size_t i = 0; i < total; ++i) {
+    /* the moments are stored in FP32: the update uses the values as stored */
+    const float mf = (float)(beta1 * (double)m[i] + (1.0 - beta1) * grad[i]);
+    const float vf = (float)(beta2 * (double)v[i] + (1.0 - beta2) * grad[i] * grad[i]);
+    m_out[i] = mf;
+    v_out[i] = vf;
+    theta_out[i] = (float)((double)theta[i] - lr * ((double)mf / c1) / (sqrt((double)vf / c2) + eps));
+  }
+  if (loss_mean) *loss_mean = loss;
+  free(grad);
 }
 
 /* ===================================================================== */

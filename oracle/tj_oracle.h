@@ -116,6 +116,11 @@ void orc_td_one(double q_sel, double q_next_max, double r, int done, double gamm
 void orc_sgd_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
                   const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
                   double kappa, double lr, float *theta_out, double *loss_mean);
+/* the same gradient through Adam (Table 2's optimiser); t >= 1 counts the steps; m, v: FP32 moment blobs */
+void orc_adam_step(const float *theta, const float *theta_target, int D, int H, int A, const float *obs,
+                   const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
+                   double kappa, double lr, double beta1, double beta2, double eps, int64_t t, const float *m, const float *v,
+                   float *theta_out, float *m_out, float *v_out, double *loss_mean);
 void orc_gae(const float *rew, const float *val, const uint8_t *done, int T, int N, double gamma, double lambda,
              double *adv, double *ret);
 

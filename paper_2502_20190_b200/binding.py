@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
            "tj_last_error")
 
 
@@ -90,6 +90,7 @@ def load_library():
     L.tj_td_error_static.argtypes = [vp, vp, vp, vp, vp]
     L.tj_gae.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
     L.tj_sgd_step.argtypes = [vp, vp, f32, vp, vp, vp]
+    L.tj_adam_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, vp, vp, vp, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
@@ -154,6 +155,12 @@ def tj_td_error_static(h, batch: TjBatch, td_ptr: int, huber_ptr: int, loss_ptr:
 def tj_sgd_step(h, batch: TjBatch, lr: float, theta_ptr: int, theta_target_ptr: int, loss_ptr: int):
     """One learner update (Algorithm 1's update line as a minibatch semi-gradient step) on device blobs, in place."""
     return load_library().tj_sgd_step(h, C.byref(batch), lr, theta_ptr, theta_target_ptr, loss_ptr or None)
+
+
+def tj_adam_step(h, batch: TjBatch, lr, beta1, beta2, eps, t, theta_ptr, theta_target_ptr, m_ptr, v_ptr, loss_ptr):
+    """tj_sgd_step's gradient through Adam; m and v are device moment blobs updated in place."""
+    return load_library().tj_adam_step(h, C.byref(batch), lr, beta1, beta2, eps, t, theta_ptr, theta_target_ptr, m_ptr, v_ptr,
+                                       loss_ptr or None)
 
 
 def tj_gae(h, rew_ptr, val_ptr, done_ptr, T, N, gamma, lam, adv_ptr, ret_ptr):
@@ -331,6 +338,15 @@ class Context:
         assert theta.is_contiguous() and theta_target.is_contiguous() and theta.numel() == theta_target.numel()
         loss = torch.empty(1, dtype=torch.float32, device=self.device)
         self._check(tj_sgd_step(self.h, batch["c"], float(lr), theta.data_ptr(), theta_target.data_ptr(), loss.data_ptr()))
+        return loss
+
+    def adam_step(self, batch, lr, theta, theta_target, m, v, t, beta1=0.9, beta2=0.999, eps=1e-8):
+        torch = self.torch
+        for x in (theta, theta_target, m, v):
+            assert x.dtype == torch.float32 and x.is_contiguous() and x.numel() == theta.numel()
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        self._check(tj_adam_step(self.h, batch["c"], float(lr), float(beta1), float(beta2), float(eps), int(t), theta.data_ptr(),
+                                 theta_target.data_ptr(), m.data_ptr(), v.data_ptr(), loss.data_ptr()))
         return loss
 
     def gae(self, rew, val, done, gamma, lam, adv=None, ret=None):

@@ -541,8 +541,9 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
   return TJ_OK;
 }
 
-int tj_sgd_step(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, float* loss_mean_out) {
-  if (!x) return TJ_ERR_INVALID_ARG;
+namespace {
+int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, const tj::AdamParams* adam,
+                   float* loss_mean_out) {
   if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
   if (!theta || !theta_target) return fail(x, TJ_ERR_INVALID_ARG, "parameter blobs must not be null");
   if (theta == theta_target) return fail(x, TJ_ERR_INVALID_ARG, "theta and theta_target must be different buffers");
@@ -557,11 +558,32 @@ int tj_sgd_step(tj_ctx* x, const tj_batch* b, float lr, float* theta, const floa
   const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
   p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH; p.g = p.dh2 + RH; p.partial = p.g + rows * 16; p.grad_partial = p.partial + rows / 16 + 64;
   LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 15 : 14);
-  cudaError_t e = launch_sgd_step(p, lr, x->stream);
+  cudaError_t e = launch_sgd_step(p, lr, adam, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
   if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
     return cuda_fail(x, e, "learner update (loss reduction)");
   return TJ_OK;
+}
+}  // namespace
+
+int tj_sgd_step(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  return learner_update(x, b, lr, theta, theta_target, nullptr, loss_mean_out);
+}
+
+int tj_adam_step(tj_ctx* x, const tj_batch* b, float lr, float beta1, float beta2, float eps, int64_t t, float* theta,
+                 const float* theta_target, float* m, float* v, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!m || !v) return fail(x, TJ_ERR_INVALID_ARG, "moment blobs must not be null");
+  if (m == v || m == theta || v == theta) return fail(x, TJ_ERR_INVALID_ARG, "theta, m and v must be different buffers");
+  if (t < 1) return fail(x, TJ_ERR_INVALID_ARG, "the Adam step counter starts at 1");
+  if (!(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f && eps > 0.f))
+    return fail(x, TJ_ERR_INVALID_ARG, "Adam needs 0 <= beta1, beta2 < 1 and eps > 0");
+  tj::AdamParams a{};
+  a.m = m; a.v = v; a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
+  a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));
+  a.c2 = (float)(1.0 - std::pow((double)beta2, (double)t));
+  return learner_update(x, b, lr, theta, theta_target, &a, loss_mean_out);
 }
 
 int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, int32_t T, int32_t N, float gamma,

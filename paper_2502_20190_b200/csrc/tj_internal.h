@@ -109,6 +109,11 @@ struct SgdParams {
   float* grad_partial;         // scratch: per row range partial sums of one gradient matrix
 };
 
+struct AdamParams {
+  float *m, *v;               // moment blobs, same layout as theta
+  float beta1, beta2, eps, c1, c2;
+};
+
 struct SampleParams {
   int B, D, N, rec_words;
   uint2 seed;
@@ -186,7 +191,7 @@ int td_grid(int n);
 size_t sgd_scratch_floats(int max_rows, int H);
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);
-cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s);
+cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam /* nullable: plain SGD */, cudaStream_t s);
 int td_static_max_rows();
 cudaError_t launch_td_static(const TdParams& p, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,

@@ -233,6 +233,22 @@ __global__ void sgd_apply_kernel(float* __restrict__ Cm, const float* __restrict
   Cm[i] -= lr * s;
 }
 
+// the same gradient through Adam (Table 2's optimiser): m <- b1 m + (1-b1) g, v <- b2 v + (1-b2) g^2,
+// theta <- theta - lr (m / c1) / (sqrt(v / c2) + eps) with the bias corrections c1 = 1 - b1^t, c2 = 1 - b2^t from the host
+__global__ void sgd_apply_adam_kernel(float* __restrict__ Cm, float* __restrict__ m, float* __restrict__ v,
+                                      const float* __restrict__ P, int count, int n_ranges, float lr, float beta1, float beta2,
+                                      float eps, float c1, float c2) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float g = 0.f;
+  for (int z = 0; z < n_ranges; ++z) g += P[(size_t)z * count + i];
+  const float mi = fmaf(beta1, m[i], (1.f - beta1) * g);
+  const float vi = fmaf(beta2, v[i], (1.f - beta2) * g * g);
+  m[i] = mi;
+  v[i] = vi;
+  Cm[i] -= lr * (mi / c1) / (sqrtf(vi / c2) + eps);
+}
+
 }  // namespace
 
 size_t sgd_scratch_floats(int max_rows, int H) {
@@ -248,7 +264,7 @@ bool sgd_supported(int D, int H, int A) {
   return H >= 1 && D >= 1 && A >= 1 && A <= 16 && smem <= 200 * 1024;
 }
 
-cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s) {
+cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
   const int D = p.D, H = p.H, A = p.A;
   const int grid = sgd_partial_count(p.n);
   const size_t smem_f = (((size_t)D + 2 * (size_t)H + A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
@@ -273,7 +289,13 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, cudaStream_t s) {
   auto upd = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
     sgd_grad_partial_kernel<<<dim3((N + 31) / 32, (M + 31) / 32, n_ranges), 256, 0, s>>>(p.grad_partial, M, N, Am, lda, Bm, ldb, p.n,
                                                                                        rows_per_range);
-    sgd_apply_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, p.grad_partial, M * N, n_ranges, lr);
+    if (adam) {
+      const size_t off = (size_t)(C - p.theta);
+      sgd_apply_adam_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, adam->m + off, adam->v + off, p.grad_partial, M * N, n_ranges, lr,
+                                                                adam->beta1, adam->beta2, adam->eps, adam->c1, adam->c2);
+    } else {
+      sgd_apply_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, p.grad_partial, M * N, n_ranges, lr);
+    }
   };
   upd(W3, A, H, p.g, A, p.h2, H);
   upd(b3, A, 1, p.g, A, nullptr, 0);

@@ -63,8 +63,9 @@ def test_sgd_step_matches_oracle(env, kind, D, A, H, N, B):
     assert abs(float(loss.item()) - o_loss) <= 2 * RTOL_FP32 * (abs(o_loss) + 1e-3)
     dg = g_new.astype(np.float64) - theta.astype(np.float64)
     do = o_new.astype(np.float64) - theta.astype(np.float64)
-    # the FP32 rounding of theta_new itself (half an ulp of theta, on both sides) is part of the comparison floor
-    ulp = np.spacing(np.abs(theta).astype(np.float32)).astype(np.float64)
+    # the FP32 rounding of theta_new itself (half an ulp on each side, of a value that may sit one binade above theta) is
+    # part of the comparison floor
+    ulp = 2 * np.spacing(np.abs(theta).astype(np.float32)).astype(np.float64)
     for name, a, b in _groups(D, H, A):
         assert np.abs(do[a:b]).max() > 0, name                               # every group moves
         rms = np.sqrt(np.mean(do[a:b] ** 2))
@@ -109,3 +110,68 @@ def test_sgd_step_argument_checks(env):
     b2 = c2.alloc_batch(8)
     st = binding.tj_sgd_step(c2.h, b2["c"], 0.1, th.data_ptr(), tt.data_ptr(), 0)
     assert st == binding.TJ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (2, 16, 5, 200, 40, 333)])
+def test_adam_step_matches_oracle(env, kind, D, A, H, N, B):
+    """Adam on the same gradient.  Two regimes: (i) moments with history (t = 5, v0 > 0), where the update is smooth in the
+    gradient and the FP32 tolerance applies to every entry; (ii) the first step from zero moments, a sign step of size lr:
+    there an entry is compared only where the oracle's |g| exceeds 1e-3 of the group's rms (below that the FP32 summation
+    error of g can move the ratio g / (|g| + eps) by O(1)), and everywhere the step must stay within lr."""
+    torch, orc, binding = env
+    f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, epsilon=0.3, seed=778, replay_capacity=N * 16,
+                   minibatch=B, staleness_bound=20, warmup=N, target_sync_interval=1000, gamma=0.99, huber_delta=1.0,
+                   max_episode_steps=9)
+    ctx = binding.Context(**f)
+    theta_t, theta = blob_for(f, 1), blob_for(f, 2)
+    ctx.publish_weights(theta_t)
+    ctx.actor_step(6)
+    ctx.publish_weights(theta)
+    ctx.actor_step(6)
+    _, batch = ctx.replay_sample()
+    dev = ctx.device
+    bn = {k: batch[k].cpu().numpy() for k in ("obs", "act", "rew", "next_obs", "done")}
+    rng = np.random.default_rng(1)
+    # the oracle's gradient, for the scale of the moments and for the mask of regime (ii)
+    o_sgd, _ = orc.sgd_step(theta, theta_t, D, H, A, bn["obs"], bn["act"], bn["rew"], bn["next_obs"], bn["done"], 0.99, 1.0, 1.0)
+    g = theta.astype(np.float64) - o_sgd.astype(np.float64)
+    g_rms = float(np.sqrt(np.mean(g * g)))
+    lr, b1, b2, eps = 1e-3, 0.9, 0.999, 1e-8
+    ulp = 2 * np.spacing(np.abs(theta).astype(np.float32)).astype(np.float64)      # rounding of theta_new, both sides
+    # (i) with history
+    m0 = (rng.standard_normal(theta.size) * g_rms).astype(np.float32)
+    v0 = ((0.5 + rng.random(theta.size)) * g_rms ** 2).astype(np.float32)
+    th, tt = torch.from_numpy(theta.copy()).to(dev), torch.from_numpy(theta_t.copy()).to(dev)
+    m, v = torch.from_numpy(m0.copy()).to(dev), torch.from_numpy(v0.copy()).to(dev)
+    loss = ctx.adam_step(batch, lr, th, tt, m, v, 5, b1, b2, eps)
+    o_new, o_m, o_v, o_loss = orc.adam_step(theta, theta_t, D, H, A, bn["obs"], bn["act"], bn["rew"], bn["next_obs"], bn["done"],
+                                            0.99, 1.0, lr, b1, b2, eps, 5, m0, v0)
+    assert abs(float(loss.item()) - o_loss) <= 2 * RTOL_FP32 * (abs(o_loss) + 1e-3)
+    close(m.cpu().numpy(), o_m, RTOL_FP32, "m")
+    close(v.cpu().numpy(), o_v, RTOL_FP32, "v")
+    dg = th.cpu().numpy().astype(np.float64) - theta
+    do = o_new.astype(np.float64) - theta
+    for name, a, b in _groups(D, H, A):
+        rms = np.sqrt(np.mean(do[a:b] ** 2))
+        err = np.abs(dg[a:b] - do[a:b])
+        assert np.all(err <= RTOL_FP32 * np.abs(do[a:b]) + RTOL_FP32 * rms + ulp[a:b]), (name, err.max(), rms)
+    # (ii) first step from zero moments
+    th = torch.from_numpy(theta.copy()).to(dev)
+    m, v = torch.zeros_like(th), torch.zeros_like(th)
+    ctx.adam_step(batch, lr, th, tt, m, v, 1, b1, b2, eps)
+    z = np.zeros_like(theta)
+    o_new, o_m, o_v, _ = orc.adam_step(theta, theta_t, D, H, A, bn["obs"], bn["act"], bn["rew"], bn["next_obs"], bn["done"],
+                                       0.99, 1.0, lr, b1, b2, eps, 1, z, z)
+    dg = th.cpu().numpy().astype(np.float64) - theta
+    do = o_new.astype(np.float64) - theta
+    assert np.all(np.abs(dg) <= lr * (1 + 1e-4) + ulp)
+    n_cmp = 0
+    for name, a, b in _groups(D, H, A):
+        sure = np.abs(g[a:b]) > 1e-3 * np.sqrt(np.mean(g[a:b] ** 2))
+        n_cmp += int(sure.sum())
+        assert np.all(np.abs(dg[a:b] - do[a:b])[sure] <= 1e-4 * lr + ulp[a:b][sure]), name
+        dead = o_m[a:b] == 0                                                   # the gradient is exactly zero there
+        assert np.all(dg[a:b][dead] == 0) and np.all(do[a:b][dead] == 0)
+    assert n_cmp > 0.5 * np.count_nonzero(g)
+    close(m.cpu().numpy(), o_m, RTOL_FP32, "m after the first step")
+    assert ctx.stats()["device_error"] == 0

@@ -126,3 +126,56 @@ def test_update_is_a_batch_mean():
     n2, l2 = _step(theta, target, twice, 0.2)
     np.testing.assert_allclose(n1, n2, atol=1e-7)
     assert abs(l1 - l2) < 1e-12
+
+
+# ------------------------------------------------------------------------------------------------ Adam (Table 2)
+def _adam(theta, target, b, lr, b1, b2, eps, t, m, v):
+    return oracle.adam_step(theta, target, D, H, A, b["obs"], b["act"], b["rew"], b["next_obs"], b["done"], GAMMA, KAPPA, lr,
+                            b1, b2, eps, t, m, v)
+
+
+def _gradient(theta, target, b):
+    """the gradient the pinned SGD step applies (lr = 1 keeps the most digits)"""
+    new, _ = _step(theta, target, b, 1.0)
+    return theta.astype(np.float64) - new.astype(np.float64)
+
+
+def test_adam_first_step_has_the_closed_form():
+    """From m = v = 0 the bias-corrected moments are g and g^2: the first update is -lr * g / (|g| + eps)."""
+    rng = np.random.default_rng(21)
+    theta, target, b = _blob(rng), _blob(rng), _batch(rng, 7)
+    g = _gradient(theta, target, b)
+    z = np.zeros_like(theta)
+    lr, b1, b2, eps = 0.01, 0.9, 0.999, 1e-8
+    new, m, v, loss = _adam(theta, target, b, lr, b1, b2, eps, 1, z, z)
+    assert abs(loss - _loss(theta, target, b)) < 1e-12 * (1 + abs(loss))
+    big = np.abs(g) > 1e-4                                    # where the float32 storage of g, m and v does not blur the ratio
+    assert big.sum() > 50
+    d = new.astype(np.float64) - theta.astype(np.float64)
+    np.testing.assert_allclose(d[big], -lr * np.sign(g[big]), rtol=2e-3)          # |g| >> eps: a sign step of size lr
+    np.testing.assert_allclose(m[big], (1 - b1) * g[big], rtol=1e-3)
+    np.testing.assert_allclose(v[big], (1 - b2) * g[big] ** 2, rtol=2e-3)
+    assert np.all(d[g == 0] == 0)                             # untouched rows (other actions' head weights) do not move
+
+
+def test_adam_recurrence_and_limits():
+    rng = np.random.default_rng(22)
+    theta, target, b = _blob(rng), _blob(rng), _batch(rng, 5)
+    g = _gradient(theta, target, b)
+    m0 = (rng.standard_normal(theta.size) * 1e-2).astype(np.float32)
+    v0 = (rng.random(theta.size) * 1e-3).astype(np.float32)
+    lr, b1, b2, eps, t = 0.003, 0.8, 0.95, 1e-6, 4
+    new, m, v, _ = _adam(theta, target, b, lr, b1, b2, eps, t, m0, v0)
+    m_ref = b1 * m0.astype(np.float64) + (1 - b1) * g
+    v_ref = b2 * v0.astype(np.float64) + (1 - b2) * g * g
+    np.testing.assert_allclose(m, m_ref, rtol=1e-5, atol=1e-9)
+    np.testing.assert_allclose(v, v_ref, rtol=1e-5, atol=1e-12)
+    upd = -lr * (m_ref / (1 - b1 ** t)) / (np.sqrt(v_ref / (1 - b2 ** t)) + eps)
+    np.testing.assert_allclose(new.astype(np.float64) - theta, upd, rtol=1e-3, atol=3e-7)
+    # beta1 = beta2 = 0: no memory, every step is the first step's sign rule whatever m and v held
+    n0, _, _, _ = _adam(theta, target, b, lr, 0.0, 0.0, 1e-12, 9, m0, v0)
+    big = np.abs(g) > 1e-4
+    np.testing.assert_allclose((n0.astype(np.float64) - theta)[big], -lr * np.sign(g[big]), rtol=2e-3)
+    # lr = 0 moves nothing but still advances the moments
+    n1, m1, _, _ = _adam(theta, target, b, 0.0, b1, b2, eps, t, m0, v0)
+    assert np.array_equal(n1, theta) and not np.array_equal(m1, m0)
