@@ -175,3 +175,15 @@ def test_adam_step_matches_oracle(env, kind, D, A, H, N, B):
     assert n_cmp > 0.5 * np.count_nonzero(g)
     close(m.cpu().numpy(), o_m, RTOL_FP32, "m after the first step")
     assert ctx.stats()["device_error"] == 0
+
+
+def test_cartpole_dqn_learns_through_the_library(env):
+    """The whole path as one system: actor -> ring -> staleness-bounded sampler -> Adam update -> publish.  A random policy
+    keeps the pole up for about 10 steps; after 1.2 M env steps the 100-iteration window mean must have passed 60 (it
+    reaches ~150 with this seed) and no sampled transition may be staler than the bound."""
+    from paper_2502_20190_b200 import train_dqn
+    hist = train_dqn.train(staleness_bound=8, iters=1200, seed=1)
+    best = max(r["mean_return"] for r in hist if r["episodes"] > 0)
+    assert hist[0]["mean_return"] < 15
+    assert best > 60, [round(r["mean_return"], 1) for r in hist]
+    assert hist[-1]["max_sampled_staleness"] <= 8 and hist[-1]["updates"] > 4000
