@@ -324,6 +324,28 @@ def adam_step(theta, theta_target, D, H, A, obs, act, rew, next_obs, done, gamma
     return t_out, m_out, v_out, loss.value
 
 
+def ppo_step(theta, D, H, A, obs, act, logp_old, adv, ret, clip_eps, c_v, c_e, lr, beta1, beta2, eps, t, m, v):
+    """One PPO minibatch update (clipped surrogate + value loss - entropy bonus, Adam); returns
+    (theta_new, m_new, v_new, loss, stats[4])."""
+    arrs = [np.ascontiguousarray(a, np.float32) for a in (theta, obs, logp_old, adv, ret, m, v)]
+    theta, obs, logp_old, adv, ret, m, v = arrs
+    act = np.ascontiguousarray(act, np.int32)
+    n = act.size
+    assert theta.size == blob_floats(D, H, A, True) == m.size == v.size and obs.size == n * D
+    t_out, m_out, v_out = np.zeros_like(theta), np.zeros_like(theta), np.zeros_like(theta)
+    loss = C.c_double()
+    stats = np.zeros(4, np.float64)
+    fn = lib().orc_ppo_step
+    fn.restype = None
+    fn.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                   C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int64,
+                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    fn(_p(theta), D, H, A, _p(obs), _p(act), _p(logp_old), _p(adv), _p(ret), n, float(clip_eps), float(c_v), float(c_e),
+       float(lr), float(beta1), float(beta2), float(eps), int(t), _p(m), _p(v), _p(t_out), _p(m_out), _p(v_out),
+       C.byref(loss), _p(stats))
+    return t_out, m_out, v_out, loss.value, stats
+
+
 def gae(rew, val, done, gamma, lam):
     rew = np.ascontiguousarray(rew, np.float32)
     val = np.ascontiguousarray(val, np.float32)

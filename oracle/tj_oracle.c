@@ -427,6 +427,136 @@ void orc_adam_step(const float *theta, const float *theta_target, int D, int H, 
 }
 
 /* ===================================================================== */
+/* On-policy learner update: PPO's clipped surrogate (Schulman et al. 2017; the paper's on-policy algorithm,       */
+/* Sec. 4.1) on the shared-trunk network with a categorical policy head and a value head:                          */
+/*   p = softmax(logits), ratio = exp(log p[a] - logp_old),                                                         */
+/*   L = mean_j [ -min(ratio A, clip(ratio, 1-eps, 1+eps) A) + c_v/2 (V - R)^2 - c_e H(p) ]                          */
+/* then one Adam step on L.  Blob layout with the value head: [W1, b1, W2, b2, W3, b3, Wv, bv].                      */
+/* stats[0..3] = mean policy loss, mean value loss (without c_v), mean entropy, fraction of rows with the clip active */
+/* ===================================================================== */
+static double ppo_loss_gradient(const float *theta, int D, int H, int A, const float *obs, const int32_t *act,
+                                const float *logp_old, const float *adv, const float *ret, int n, double clip_eps, double c_v,
+                                double c_e, double *grad, double *stats) {
+  const size_t nW1 = (size_t)H * D, nW2 = (size_t)H * H, nW3 = (size_t)A * H;
+  const size_t o_b1 = nW1, o_W2 = o_b1 + H, o_b2 = o_W2 + nW2, o_W3 = o_b2 + H, o_b3 = o_W3 + nW3, o_Wv = o_b3 + A,
+               o_bv = o_Wv + H, total = o_bv + 1;
+  for (size_t i = 0; i < total; ++i) grad[i] = 0.0;
+  double *h1 = (double *)malloc(sizeof(double) * H), *h2 = (double *)malloc(sizeof(double) * H);
+  double *dh1 = (double *)malloc(sizeof(double) * H), *dh2 = (double *)malloc(sizeof(double) * H);
+  double *l = (double *)malloc(sizeof(double) * A), *pr = (double *)malloc(sizeof(double) * A),
+         *gl = (double *)malloc(sizeof(double) * A);
+  const float *W1 = theta, *b1 = theta + o_b1, *W2 = theta + o_W2, *b2 = theta + o_b2, *W3 = theta + o_W3, *b3 = theta + o_b3,
+              *Wv = theta + o_Wv, *bv = theta + o_bv;
+  double s_pi = 0.0, s_v = 0.0, s_h = 0.0, s_clip = 0.0;
+  for (int j = 0; j < n; ++j) {
+    const float *x = obs + (size_t)j * D;
+    int a = act[j];
+    if (a < 0) a = 0;
+    if (a >= A) a = A - 1;
+    for (int i = 0; i < H; ++i) {
+      double s = (double)b1[i];
+      for (int k = 0; k < D; ++k) s += (double)W1[(size_t)i * D + k] * (double)x[k];
+      h1[i] = s > 0.0 ? s : 0.0;
+    }
+    for (int i = 0; i < H; ++i) {
+      double s = (double)b2[i];
+      for (int k = 0; k < H; ++k) s += (double)W2[(size_t)i * H + k] * h1[k];
+      h2[i] = s > 0.0 ? s : 0.0;
+    }
+    double lmax = -1e300;
+    for (int i = 0; i < A; ++i) {
+      double s = (double)b3[i];
+      for (int k = 0; k < H; ++k) s += (double)W3[(size_t)i * H + k] * h2[k];
+      l[i] = s;
+      if (s > lmax) lmax = s;
+    }
+    double val = (double)bv[0];
+    for (int k = 0; k < H; ++k) val += (double)Wv[k] * h2[k];
+    double Z = 0.0;
+    for (int i = 0; i < A; ++i) Z += exp(l[i] - lmax);
+    const double logZ = lmax + log(Z);
+    double ent = 0.0;
+    for (int i = 0; i < A; ++i) {
+      pr[i] = exp(l[i] - logZ);
+      ent -= pr[i] * (l[i] - logZ);
+    }
+    const double logp = l[a] - logZ, ratio = exp(logp - (double)logp_old[j]), Aj = (double)adv[j];
+    const double rc = ratio < 1.0 - clip_eps ? 1.0 - clip_eps : (ratio > 1.0 + clip_eps ? 1.0 + clip_eps : ratio);
+    const double t1 = ratio * Aj, t2 = rc * Aj;
+    const int unclipped = t1 <= t2; /* the minimum is the unclipped term (also when both are equal) */
+    s_pi += -(unclipped ? t1 : t2);
+    s_clip += unclipped ? 0.0 : 1.0;
+    const double dv = val - (double)ret[j];
+    s_v += 0.5 * dv * dv;
+    s_h += ent;
+    /* gradients at the outputs, already divided by n */
+    const double g_logp = unclipped ? -Aj * ratio : 0.0;
+    for (int i = 0; i < A; ++i) {
+      const double dlogp = (i == a ? 1.0 : 0.0) - pr[i];
+      const double dent = -pr[i] * ((l[i] - logZ) + ent); /* dH/dl_i */
+      gl[i] = (g_logp * dlogp - c_e * dent) / (double)n;
+    }
+    const double gv = c_v * dv / (double)n;
+    /* heads */
+    for (int k = 0; k < H; ++k) dh2[k] = 0.0;
+    for (int i = 0; i < A; ++i) {
+      grad[o_b3 + i] += gl[i];
+      for (int k = 0; k < H; ++k) {
+        grad[o_W3 + (size_t)i * H + k] += gl[i] * h2[k];
+        dh2[k] += gl[i] * (double)W3[(size_t)i * H + k];
+      }
+    }
+    grad[o_bv] += gv;
+    for (int k = 0; k < H; ++k) {
+      grad[o_Wv + k] += gv * h2[k];
+      dh2[k] += gv * (double)Wv[k];
+      if (!(h2[k] > 0.0)) dh2[k] = 0.0;
+    }
+    /* layer 2 */
+    for (int k = 0; k < H; ++k) dh1[k] = 0.0;
+    for (int i = 0; i < H; ++i) {
+      if (dh2[i] == 0.0) continue;
+      grad[o_b2 + i] += dh2[i];
+      for (int k = 0; k < H; ++k) {
+        grad[o_W2 + (size_t)i * H + k] += dh2[i] * h1[k];
+        dh1[k] += dh2[i] * (double)W2[(size_t)i * H + k];
+      }
+    }
+    /* layer 1 */
+    for (int i = 0; i < H; ++i) {
+      const double d = h1[i] > 0.0 ? dh1[i] : 0.0;
+      if (d == 0.0) continue;
+      grad[o_b1 + i] += d;
+      for (int k = 0; k < D; ++k) grad[(size_t)i * D + k] += d * (double)x[k];
+    }
+  }
+  free(h1); free(h2); free(dh1); free(dh2); free(l); free(pr); free(gl);
+  if (stats) {
+    stats[0] = s_pi / n; stats[1] = s_v / n; stats[2] = s_h / n; stats[3] = s_clip / n;
+  }
+  return (s_pi + c_v * s_v - c_e * s_h) / (double)n;
+}
+
+void orc_ppo_step(const float *theta, int D, int H, int A, const float *obs, const int32_t *act, const float *logp_old,
+                  const float *adv, const float *ret, int n, double clip_eps, double c_v, double c_e, double lr, double beta1,
+                  double beta2, double eps, int64_t t, const float *m, const float *v, float *theta_out, float *m_out,
+                  float *v_out, double *loss, double *stats) {
+  const size_t total = (size_t)orc_blob_floats(D, H, A, 1);
+  double *grad = (double *)malloc(total * sizeof(double));
+  const double L = ppo_loss_gradient(theta, D, H, A, obs, act, logp_old, adv, ret, n, clip_eps, c_v, c_e, grad, stats);
+  const double c1 = 1.0 - pow(beta1, (double)t), c2 = 1.0 - pow(beta2, (double)t);
+  for (size_t i = 0; i < total; ++i) {
+    const float mf = (float)(beta1 * (double)m[i] + (1.0 - beta1) * grad[i]);
+    const float vf = (float)(beta2 * (double)v[i] + (1.0 - beta2) * grad[i] * grad[i]);
+    m_out[i] = mf;
+    v_out[i] = vf;
+    theta_out[i] = (float)((double)theta[i] - lr * ((double)mf / c1) / (sqrt((double)vf / c2) + eps));
+  }
+  if (loss) *loss = L;
+  free(grad);
+}
+
+/* ===================================================================== */
 /* GAE: delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;                      */
 /*      A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0; R_t = A_t + V_t */
 /* arrays are time-major: rew[T][N], val[T+1][N], done[T][N]              */

@@ -121,6 +121,12 @@ void orc_adam_step(const float *theta, const float *theta_target, int D, int H, 
                    const int32_t *act, const float *rew, const float *next_obs, const int32_t *done, int n, double gamma,
                    double kappa, double lr, double beta1, double beta2, double eps, int64_t t, const float *m, const float *v,
                    float *theta_out, float *m_out, float *v_out, double *loss_mean);
+/* PPO's clipped surrogate + value loss - entropy bonus on the shared-trunk network (blob with the value head), one Adam
+ * step; stats[4] = mean policy loss, mean value loss (0.5 (V-R)^2), mean entropy, clip fraction */
+void orc_ppo_step(const float *theta, int D, int H, int A, const float *obs, const int32_t *act, const float *logp_old,
+                  const float *adv, const float *ret, int n, double clip_eps, double c_v, double c_e, double lr, double beta1,
+                  double beta2, double eps, int64_t t, const float *m, const float *v, float *theta_out, float *m_out,
+                  float *v_out, double *loss, double *stats);
 void orc_gae(const float *rew, const float *val, const uint8_t *done, int T, int N, double gamma, double lambda,
              double *adv, double *ret);
 
