@@ -243,6 +243,27 @@ int tj_sgd_step(tj_ctx *ctx, const tj_batch *batch, float lr, float *theta, cons
 int tj_adam_step(tj_ctx *ctx, const tj_batch *batch, float lr, float beta1, float beta2, float eps, int64_t t, float *theta,
                  const float *theta_target, float *m, float *v, float *loss_mean_out);
 
+/* On-policy learner update: PPO's clipped surrogate (Schulman et al. 2017; the paper's on-policy algorithm, Sec. 4.1, with
+ * Table 2's "gae" advantages) on the shared-trunk network with the categorical policy head and the value head:
+ *   ratio_j = exp(log pi(a_j | s_j; theta) - logp_old_j)
+ *   L = mean_j [ -min(ratio_j A_j, clip(ratio_j, 1 - clip_eps, 1 + clip_eps) A_j) + c_v / 2 (V(s_j) - R_j)^2 - c_e H(pi(. | s_j)) ]
+ * followed by one Adam step on L (arguments as tj_adam_step).  theta, m, v: device FP32 blobs in the publish layout with the
+ * value head ([W1, b1, W2, b2, W3, b3, Wv, bv]).  The batch arrays are device pointers owned by the caller; rows of a
+ * segment (tj_segment_acquire) and of tj_gae's outputs can be passed as they lie: obs [n][obs_dim], the others [n].
+ * stats_out (nullable, device, 5 floats): L, mean policy term, mean 0.5 (V - R)^2, mean entropy, fraction of rows where
+ * the clipped term is the minimum -- all before the update.  batch.n <= the configured minibatch (4096 if none).
+ * TJ_ERR_UNSUPPORTED unless the context is FP32 with the categorical policy. */
+typedef struct {
+  int32_t n;
+  const float *obs;
+  const int32_t *act;
+  const float *logp_old;
+  const float *adv;
+  const float *ret;
+} tj_ppo_batch;
+int tj_ppo_step(tj_ctx *ctx, const tj_ppo_batch *batch, float lr, float beta1, float beta2, float eps, int64_t t, float clip_eps,
+                float c_v, float c_e, float *theta, float *m, float *v, float *stats_out);
+
 /* Generalised advantage estimation over time-major arrays (Table 2: gae lambda, discount gamma):
  *   delta_t = r_t + gamma (1-d_t) V_{t+1} - V_t;  A_t = delta_t + gamma lambda (1-d_t) A_{t+1}, A_T = 0;
  *   R_t = A_t + V_t.   rew [T][N], val [T+1][N], done [T][N] -> adv [T][N], ret [T][N].

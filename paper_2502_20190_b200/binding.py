@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
            "tj_last_error")
 
 
@@ -91,6 +91,7 @@ def load_library():
     L.tj_gae.argtypes = [vp, vp, vp, vp, i32, i32, f32, f32, vp, vp]
     L.tj_sgd_step.argtypes = [vp, vp, f32, vp, vp, vp]
     L.tj_adam_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, vp, vp, vp, vp, vp]
+    L.tj_ppo_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, f32, f32, f32, vp, vp, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
@@ -161,6 +162,17 @@ def tj_adam_step(h, batch: TjBatch, lr, beta1, beta2, eps, t, theta_ptr, theta_t
     """tj_sgd_step's gradient through Adam; m and v are device moment blobs updated in place."""
     return load_library().tj_adam_step(h, C.byref(batch), lr, beta1, beta2, eps, t, theta_ptr, theta_target_ptr, m_ptr, v_ptr,
                                        loss_ptr or None)
+
+
+class TjPpoBatch(C.Structure):
+    _fields_ = [("n", C.c_int32), ("obs", C.c_void_p), ("act", C.c_void_p), ("logp_old", C.c_void_p), ("adv", C.c_void_p),
+                ("ret", C.c_void_p)]
+
+
+def tj_ppo_step(h, batch: TjPpoBatch, lr, beta1, beta2, eps, t, clip_eps, c_v, c_e, theta_ptr, m_ptr, v_ptr, stats_ptr):
+    """One PPO minibatch update (clipped surrogate + value loss - entropy bonus, Adam) on device blobs, in place."""
+    return load_library().tj_ppo_step(h, C.byref(batch), lr, beta1, beta2, eps, t, clip_eps, c_v, c_e, theta_ptr, m_ptr, v_ptr,
+                                      stats_ptr or None)
 
 
 def tj_gae(h, rew_ptr, val_ptr, done_ptr, T, N, gamma, lam, adv_ptr, ret_ptr):
@@ -348,6 +360,21 @@ class Context:
         self._check(tj_adam_step(self.h, batch["c"], float(lr), float(beta1), float(beta2), float(eps), int(t), theta.data_ptr(),
                                  theta_target.data_ptr(), m.data_ptr(), v.data_ptr(), loss.data_ptr()))
         return loss
+
+    def ppo_step(self, obs, act, logp_old, adv, ret, lr, theta, m, v, t, clip_eps=0.2, c_v=0.5, c_e=0.01, beta1=0.9,
+                 beta2=0.999, eps=1e-8):
+        """obs [n][D], act (int32), logp_old, adv, ret [n]: contiguous device tensors (views of a segment are fine);
+        returns the 5 statistics tensor (loss, policy, value, entropy, clip fraction)"""
+        torch = self.torch
+        n = act.numel()
+        for x_ in (obs, act, logp_old, adv, ret, theta, m, v):
+            assert x_.is_contiguous()
+        assert obs.numel() == n * self.D and act.dtype == torch.int32
+        stats = torch.empty(5, dtype=torch.float32, device=self.device)
+        b = TjPpoBatch(n, obs.data_ptr(), act.data_ptr(), logp_old.data_ptr(), adv.data_ptr(), ret.data_ptr())
+        self._check(tj_ppo_step(self.h, b, float(lr), float(beta1), float(beta2), float(eps), int(t), float(clip_eps), float(c_v),
+                                float(c_e), theta.data_ptr(), m.data_ptr(), v.data_ptr(), stats.data_ptr()))
+        return stats
 
     def gae(self, rew, val, done, gamma, lam, adv=None, ret=None):
         torch = self.torch

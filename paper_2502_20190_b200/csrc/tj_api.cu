@@ -112,6 +112,12 @@ size_t carve(tj_ctx* x, void* base) {
     x->seg_logp = cv.take<float>(G * TN);
     x->seg_val = cv.take<float>(G * ((size_t)c.rollout_len + 1) * N);
     x->seg_done = cv.take<uint8_t>(G * TN);
+    x->sgd_rows = 0;
+    x->sgd_scratch = nullptr;
+    if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_CATEGORICAL && sgd_supported(D, c.hidden, c.n_actions + 1)) {
+      x->sgd_rows = c.minibatch > 0 ? c.minibatch : 4096;
+      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(x->sgd_rows, c.hidden));
+    }
   }
   if (c.env_kind == TJ_ENV_LINGAUSS) {
     x->lgAt = cv.take<float>((size_t)D * round_up4(D));
@@ -542,6 +548,16 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
 }
 
 namespace {
+// h1, h2, dh1, dh2 [rows][H] | g [rows][17] | loss partials | PPO statistic partials | gradient partial sums
+void lay_out_update_scratch(const tj_ctx* x, tj::SgdParams& p) {
+  const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
+  p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH;
+  p.g = p.dh2 + RH;
+  p.partial = p.g + rows * 17;
+  p.stat_partial = p.partial + rows / 16 + 8;
+  p.grad_partial = p.stat_partial + 5 * (rows / 16) + 8;
+}
+
 int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, const tj::AdamParams* adam,
                    float* loss_mean_out) {
   if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
@@ -555,8 +571,8 @@ int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const f
   p.theta = theta; p.theta_target = theta_target;
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
-  const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
-  p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH; p.g = p.dh2 + RH; p.partial = p.g + rows * 16; p.grad_partial = p.partial + rows / 16 + 64;
+  lay_out_update_scratch(x, p);
+  p.ldg = x->A; p.value_head = 0;
   LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 15 : 14);
   cudaError_t e = launch_sgd_step(p, lr, adam, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
@@ -584,6 +600,36 @@ int tj_adam_step(tj_ctx* x, const tj_batch* b, float lr, float beta1, float beta
   a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));
   a.c2 = (float)(1.0 - std::pow((double)beta2, (double)t));
   return learner_update(x, b, lr, theta, theta_target, &a, loss_mean_out);
+}
+
+int tj_ppo_step(tj_ctx* x, const tj_ppo_batch* b, float lr, float beta1, float beta2, float eps, int64_t t, float clip_eps,
+                float c_v, float c_e, float* theta, float* m, float* v, float* stats_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!b || !b->obs || !b->act || !b->logp_old || !b->adv || !b->ret) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
+  if (!theta || !m || !v) return fail(x, TJ_ERR_INVALID_ARG, "parameter and moment blobs must not be null");
+  if (m == v || m == theta || v == theta) return fail(x, TJ_ERR_INVALID_ARG, "theta, m and v must be different buffers");
+  if (t < 1) return fail(x, TJ_ERR_INVALID_ARG, "the Adam step counter starts at 1");
+  if (!(lr >= 0.f) || !(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f && eps > 0.f))
+    return fail(x, TJ_ERR_INVALID_ARG, "needs lr >= 0, 0 <= beta1, beta2 < 1 and eps > 0");
+  if (!(clip_eps >= 0.f && clip_eps < 1.f)) return fail(x, TJ_ERR_INVALID_ARG, "clip_eps must lie in [0, 1)");
+  if (x->cfg.policy_kind != TJ_POLICY_CATEGORICAL || !x->sgd_scratch)
+    return fail(x, TJ_ERR_UNSUPPORTED, "the PPO update is implemented for FP32 contexts with the categorical policy and value head");
+  if (b->n < 1 || b->n > x->sgd_rows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be between 1 and the configured minibatch (4096 if none)");
+  SgdParams p{};
+  p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A;
+  p.theta = theta; p.theta_target = nullptr;
+  p.obs = b->obs; p.act = b->act; p.logp_old = b->logp_old; p.adv = b->adv; p.ret = b->ret;
+  p.clip_eps = clip_eps; p.c_v = c_v; p.c_e = c_e;
+  lay_out_update_scratch(x, p);
+  p.ldg = x->A + 1; p.value_head = 1;
+  tj::AdamParams a{};
+  a.m = m; a.v = v; a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
+  a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));
+  a.c2 = (float)(1.0 - std::pow((double)beta2, (double)t));
+  LaunchScope scope(x, TJ_K_SGD, stats_out ? 19 : 18);
+  cudaError_t e = launch_ppo_step(p, lr, &a, stats_out, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "PPO update");
+  return TJ_OK;
 }
 
 int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, int32_t T, int32_t N, float gamma,

@@ -107,6 +107,14 @@ struct SgdParams {
   float* g;                    // scratch [n][A]: dL/dq, non-zero at the selected action only
   float* partial;              // scratch: one Huber partial sum per 16 rows
   float* grad_partial;         // scratch: per row range partial sums of one gradient matrix
+  int ldg;                     // row stride of g (A for the Q head, A + 1 with the value head's entry in column A)
+  int value_head;              // 1: policy + value heads (PPO), theta carries Wv, bv after b3
+  // PPO only
+  const float* logp_old;
+  const float* adv;
+  const float* ret;
+  float clip_eps, c_v, c_e;
+  float* stat_partial;         // scratch: five partial sums per 16 rows (loss, policy, value, entropy, clipped rows)
 };
 
 struct AdamParams {
@@ -192,6 +200,8 @@ size_t sgd_scratch_floats(int max_rows, int H);
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam /* nullable: plain SGD */, cudaStream_t s);
+cudaError_t launch_ppo_step(const SgdParams& p, float lr, const AdamParams* adam, float* stats_out /* device [5], nullable */,
+                            cudaStream_t s);
 int td_static_max_rows();
 cudaError_t launch_td_static(const TdParams& p, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,

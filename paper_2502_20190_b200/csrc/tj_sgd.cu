@@ -132,28 +132,115 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
   }
 }
 
+// On-policy forward (PPO): trunk, policy head and value head of the one network; per row the clipped surrogate, the value
+// loss and the entropy, and their gradients at the outputs: g[j][0..A) for the logits, g[j][A] for the value.
+// shared memory: xs [D][16] | a1 [H][16] | a2 [H][16] | qs [A + 1][16] | weight tile [256][33]
+__global__ void __launch_bounds__(SG_THREADS) ppo_forward_kernel(const SgdParams p) {
+  extern __shared__ __align__(16) float sg_sm[];
+  const int D = p.D, H = p.H, A = p.A;
+  float* xs = sg_sm;
+  float* a1 = xs + (size_t)D * SG_ROWS;
+  float* a2 = a1 + (size_t)H * SG_ROWS;
+  float* qs = a2 + (size_t)H * SG_ROWS;
+  float* wt = qs + (size_t)(A + 1) * SG_ROWS;
+  __shared__ float part[5][SG_ROWS];
+  const int row0 = blockIdx.x * SG_ROWS;
+  const float *W1 = p.theta, *b1 = W1 + (size_t)H * D, *W2 = b1 + H, *b2 = W2 + (size_t)H * H, *W3 = b2 + H, *b3 = W3 + (size_t)A * H,
+              *Wv = b3 + A, *bv = Wv + H;
+  for (int i = threadIdx.x; i < D * SG_ROWS; i += SG_THREADS) {
+    const int k = i / SG_ROWS, r = i % SG_ROWS;
+    xs[i] = row0 + r < p.n ? p.obs[(size_t)(row0 + r) * D + k] : 0.f;
+  }
+  __syncthreads();
+  sg_dense<true>(W1, b1, H, D, xs, a1, wt);
+  __syncthreads();
+  sg_dense<true>(W2, b2, H, H, a1, a2, wt);
+  __syncthreads();
+  sg_dense<false>(W3, b3, A, H, a2, qs, wt);
+  sg_dense<false>(Wv, bv, 1, H, a2, qs + (size_t)A * SG_ROWS, wt);
+  for (int i = threadIdx.x; i < H * SG_ROWS; i += SG_THREADS) {
+    const int k = i / SG_ROWS, r = i % SG_ROWS;
+    if (row0 + r < p.n) {
+      p.h1[(size_t)(row0 + r) * H + k] = a1[i];
+      p.h2[(size_t)(row0 + r) * H + k] = a2[i];
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < SG_ROWS) {
+    const int r = threadIdx.x, j = row0 + r;
+    float l_tot = 0.f, l_pi = 0.f, l_v = 0.f, l_h = 0.f, l_c = 0.f;
+    if (j < p.n) {
+      int a = p.act[j];
+      a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+      float lmax = qs[r];
+      for (int i = 1; i < A; ++i) lmax = fmaxf(lmax, qs[(size_t)i * SG_ROWS + r]);
+      float Z = 0.f;
+      for (int i = 0; i < A; ++i) Z += expf(qs[(size_t)i * SG_ROWS + r] - lmax);
+      const float logZ = lmax + logf(Z);
+      float ent = 0.f;
+      for (int i = 0; i < A; ++i) {
+        const float lp = qs[(size_t)i * SG_ROWS + r] - logZ;
+        ent -= expf(lp) * lp;
+      }
+      const float logp = qs[(size_t)a * SG_ROWS + r] - logZ;
+      const float ratio = expf(logp - p.logp_old[j]), Aj = p.adv[j];
+      const float rc = fminf(fmaxf(ratio, 1.f - p.clip_eps), 1.f + p.clip_eps);
+      const float t1 = ratio * Aj, t2 = rc * Aj;
+      const bool unclipped = t1 <= t2;
+      const float val = qs[(size_t)A * SG_ROWS + r], dv = val - p.ret[j];
+      l_pi = -(unclipped ? t1 : t2);
+      l_c = unclipped ? 0.f : 1.f;
+      l_v = 0.5f * dv * dv;
+      l_h = ent;
+      l_tot = l_pi + p.c_v * l_v - p.c_e * l_h;
+      const float g_logp = unclipped ? -Aj * ratio : 0.f, inv_n = 1.f / (float)p.n;
+      float* gr = p.g + (size_t)j * p.ldg;
+      for (int i = 0; i < A; ++i) {
+        const float lp = qs[(size_t)i * SG_ROWS + r] - logZ, pi = expf(lp);
+        const float dlogp = (i == a ? 1.f : 0.f) - pi;
+        const float dent = -pi * (lp + ent);
+        gr[i] = (g_logp * dlogp - p.c_e * dent) * inv_n;
+      }
+      gr[A] = p.c_v * dv * inv_n;
+    }
+    part[0][r] = l_tot; part[1][r] = l_pi; part[2][r] = l_v; part[3][r] = l_h; part[4][r] = l_c;
+  }
+  __syncthreads();
+  if (threadIdx.x < 5) {
+    float s = 0.f;
+    for (int r = 0; r < SG_ROWS; ++r) s += part[threadIdx.x][r];
+    p.stat_partial[(size_t)blockIdx.x * 5 + threadIdx.x] = s;
+  }
+}
+
+// out[k] = (sum over the blocks of partial k) / n, k = 0..4, blocks in ascending order
+__global__ void ppo_finish_kernel(const float* __restrict__ stat_partial, int n_blocks, int n, float* __restrict__ out) {
+  const int k = threadIdx.x;
+  if (k >= 5) return;
+  float s = 0.f;
+  for (int b = 0; b < n_blocks; ++b) s += stat_partial[(size_t)b * 5 + k];
+  out[k] = s / (float)n;
+}
+
 // backward through the activations, SG_ROWS rows per block: shared memory d2 [H][16]
 __global__ void __launch_bounds__(SG_THREADS) sgd_backward_kernel(const SgdParams p) {
   extern __shared__ __align__(16) float sg_sm[];
   const int D = p.D, H = p.H, A = p.A;
   float* d2 = sg_sm;
-  __shared__ float gs[SG_ROWS];
-  __shared__ int as[SG_ROWS];
   const int row0 = blockIdx.x * SG_ROWS;
   const float* W2 = p.theta + (size_t)H * D + H;
   const float* W3 = W2 + (size_t)H * H + H;
-  if (threadIdx.x < SG_ROWS) {
-    const int j = row0 + threadIdx.x;
-    int a = j < p.n ? p.act[j] : 0;
-    as[threadIdx.x] = a < 0 ? 0 : (a >= A ? A - 1 : a);
-    gs[threadIdx.x] = j < p.n ? p.g[(size_t)j * A + as[threadIdx.x]] : 0.f;
-  }
-  __syncthreads();
-  // dh2[r][i] = g_r W3[a_r][i] where h2 > 0
+  const float* Wv = W3 + (size_t)A * H + A;
+  // dh2[r][i] = sum_a g[r][a] W3[a][i] (+ g[r][A] Wv[i] with the value head) where h2 > 0; for the Q head g has one
+  // non-zero entry per row
   for (int idx = threadIdx.x; idx < H * SG_ROWS; idx += SG_THREADS) {
     const int r = idx / H, i = idx % H, j = row0 + r;
     float v = 0.f;
-    if (j < p.n && p.h2[(size_t)j * H + i] > 0.f) v = gs[r] * W3[(size_t)as[r] * H + i];
+    if (j < p.n && p.h2[(size_t)j * H + i] > 0.f) {
+      const float* gr = p.g + (size_t)j * p.ldg;
+      for (int a = 0; a < A; ++a) v = fmaf(gr[a], W3[(size_t)a * H + i], v);
+      if (p.value_head) v = fmaf(gr[A], Wv[i], v);
+    }
     d2[(size_t)i * SG_ROWS + r] = v;
     if (j < p.n) p.dh2[(size_t)j * H + i] = v;
   }
@@ -253,8 +340,9 @@ __global__ void sgd_apply_adam_kernel(float* __restrict__ Cm, float* __restrict_
 
 size_t sgd_scratch_floats(int max_rows, int H) {
   const size_t rows = ((size_t)max_rows + SG_ROWS - 1) / SG_ROWS * SG_ROWS;
-  // h1, h2, dh1, dh2, g [rows][<= 16 actions], Huber partials, partial gradient sums of the largest matrix
-  return 4 * rows * (size_t)H + rows * 16 + rows / SG_ROWS + 64 + (size_t)SG_SPLITS * H * (size_t)(H > 16 ? H : 16);
+  // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), partial gradient sums of the
+  // largest matrix
+  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * H * (size_t)(H > 16 ? H : 16);
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }
@@ -264,15 +352,14 @@ bool sgd_supported(int D, int H, int A) {
   return H >= 1 && D >= 1 && A >= 1 && A <= 16 && smem <= 200 * 1024;
 }
 
-cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
+namespace {
+// the backward pass and every parameter update: C -= lr * (gradient rows)^T (input rows), a bias with a column of ones
+cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
   const int D = p.D, H = p.H, A = p.A;
   const int grid = sgd_partial_count(p.n);
-  const size_t smem_f = (((size_t)D + 2 * (size_t)H + A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
   const size_t smem_b = (size_t)H * SG_ROWS * sizeof(float);
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(sgd_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(sgd_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b)) != cudaSuccess) return e;
-  sgd_forward_kernel<<<grid, SG_THREADS, smem_f, s>>>(p);
   sgd_backward_kernel<<<grid, SG_THREADS, smem_b, s>>>(p);
   float* W1 = p.theta;
   float* b1 = W1 + (size_t)H * D;
@@ -280,12 +367,13 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
   float* b2 = W2 + (size_t)H * H;
   float* W3 = b2 + H;
   float* b3 = W3 + (size_t)A * H;
-  // the backward pass has read W2 and W3; now the parameters may change.  Every update is the same product:
-  // C -= lr * (gradient rows)^T (input rows), the bias with a column of ones as input
+  float* Wv = b3 + A;
+  float* bv = Wv + H;
   int n_ranges = (p.n + 127) / 128;
   if (n_ranges > SG_SPLITS) n_ranges = SG_SPLITS;
   const int rows_per_range = ((p.n + n_ranges - 1) / n_ranges + 31) / 32 * 32;
   n_ranges = (p.n + rows_per_range - 1) / rows_per_range;
+  // the backward pass has read W2 and the heads; now the parameters may change
   auto upd = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
     sgd_grad_partial_kernel<<<dim3((N + 31) / 32, (M + 31) / 32, n_ranges), 256, 0, s>>>(p.grad_partial, M, N, Am, lda, Bm, ldb, p.n,
                                                                                        rows_per_range);
@@ -297,13 +385,35 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
       sgd_apply_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, p.grad_partial, M * N, n_ranges, lr);
     }
   };
-  upd(W3, A, H, p.g, A, p.h2, H);
-  upd(b3, A, 1, p.g, A, nullptr, 0);
+  upd(W3, A, H, p.g, p.ldg, p.h2, H);
+  upd(b3, A, 1, p.g, p.ldg, nullptr, 0);
+  if (p.value_head) {
+    upd(Wv, 1, H, p.g + A, p.ldg, p.h2, H);
+    upd(bv, 1, 1, p.g + A, p.ldg, nullptr, 0);
+  }
   upd(W2, H, H, p.dh2, H, p.h1, H);
   upd(b2, H, 1, p.dh2, H, nullptr, 0);
   upd(W1, H, D, p.dh1, H, p.obs, D);
   upd(b1, H, 1, p.dh1, H, nullptr, 0);
   return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
+  const size_t smem_f = (((size_t)p.D + 2 * (size_t)p.H + p.A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(sgd_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f)) != cudaSuccess) return e;
+  sgd_forward_kernel<<<sgd_partial_count(p.n), SG_THREADS, smem_f, s>>>(p);
+  return backward_and_update(p, lr, adam, s);
+}
+
+cudaError_t launch_ppo_step(const SgdParams& p, float lr, const AdamParams* adam, float* stats_out, cudaStream_t s) {
+  const size_t smem_f = (((size_t)p.D + 2 * (size_t)p.H + p.A + 1) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(ppo_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f)) != cudaSuccess) return e;
+  ppo_forward_kernel<<<sgd_partial_count(p.n), SG_THREADS, smem_f, s>>>(p);
+  if (stats_out) ppo_finish_kernel<<<1, 32, 0, s>>>(p.stat_partial, sgd_partial_count(p.n), p.n, stats_out);
+  return backward_and_update(p, lr, adam, s);
 }
 
 }  // namespace tj

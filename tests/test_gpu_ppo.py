@@ -1,0 +1,88 @@
+"""GPU parity for the on-policy update (tj_ppo_step) against the oracle's orc_ppo_step, on rows of a real rollout segment:
+the GPU context rolls out, tj_gae turns the segment into advantages and returns, and both sides take the same minibatch.
+
+Compared with moment history (t = 4, v0 > 0) so that Adam is smooth in the gradient: parameter change per group within the
+FP32 tolerance plus the rounding of theta_new, moments within the tolerance, the five statistics within 2e-5.  The rows
+whose ratio sits within 1e-5 of a clip edge would make the clipped / unclipped decision depend on rounding; the test checks
+that the batch has none (the margin rule of the other parity tests)."""
+import numpy as np
+import pytest
+
+from parity_util import RTOL_FP32, blob_for, close, fields_for
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import oracle
+    from paper_2502_20190_b200 import binding, build
+    build.build()
+    oracle.build()
+    return torch, oracle, binding
+
+
+@pytest.mark.parametrize("kind,D,A,H,N,T,B", [(0, 4, 2, 64, 48, 8, 300), (1, 6, 3, 128, 40, 10, 257)])
+def test_ppo_step_matches_oracle(env, kind, D, A, H, N, T, B):
+    torch, orc, binding = env
+    f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, policy_kind=1, seed=99, replay_capacity=0,
+                   rollout_len=T, n_segments=2, staleness_bound=4, minibatch=B, gamma=0.99, gae_lambda=0.95,
+                   max_episode_steps=7)
+    ctx = binding.Context(**f)
+    theta_old = blob_for(f, 1)
+    ctx.publish_weights(theta_old)
+    ctx.actor_step(T)
+    st, seg = ctx.segment_acquire()
+    assert st == 0
+    adv, ret = ctx.gae(seg["rew"], seg["val"], seg["done"], 0.99, 0.95)
+    n = min(B, T * N)
+    obs = seg["obs"].reshape(T * N, D)[:n].contiguous()
+    act = seg["act"].reshape(-1)[:n].contiguous()
+    logp = seg["logp"].reshape(-1)[:n].contiguous()
+    # as if the behaviour policy had been further away: spreads the ratios so that both branches of the min occur
+    logp = (logp + 0.3 * torch.randn(n, generator=torch.Generator().manual_seed(5)).to(logp.device)).contiguous()
+    adv_n = adv.reshape(-1)[:n].contiguous()
+    ret_n = ret.reshape(-1)[:n].contiguous()
+    # the policy has moved since the rollout: a later parameter version, so ratios differ from 1 and some rows clip
+    rng = np.random.default_rng(3)
+    theta = (theta_old + 0.6 * rng.standard_normal(theta_old.size).astype(np.float32) * np.abs(theta_old).mean()).astype(np.float32)
+    g_scale = 1e-2
+    m0 = (rng.standard_normal(theta.size) * g_scale).astype(np.float32)
+    v0 = ((0.5 + rng.random(theta.size)) * g_scale ** 2).astype(np.float32)
+    dev = ctx.device
+    th, m, v = (torch.from_numpy(a.copy()).to(dev) for a in (theta, m0, v0))
+    lr, clip, cv, ce = 3e-4, 0.2, 0.5, 0.01
+    stats = ctx.ppo_step(obs, act, logp, adv_n, ret_n, lr, th, m, v, 4, clip, cv, ce)
+    o_new, o_m, o_v, o_loss, o_stats = orc.ppo_step(theta, D, H, A, obs.cpu().numpy(), act.cpu().numpy(), logp.cpu().numpy(),
+                                                    adv_n.cpu().numpy(), ret_n.cpu().numpy(), clip, cv, ce, lr, 0.9, 0.999, 1e-8, 4,
+                                                    m0, v0)
+    gs = stats.cpu().numpy().astype(np.float64)
+    want = np.array([o_loss, o_stats[0], o_stats[1], o_stats[2], o_stats[3]])
+    assert 0 < o_stats[3] < 1                                      # both branches of the min occur
+    assert np.all(np.abs(gs - want) <= 2 * RTOL_FP32 * (np.abs(want) + np.abs(want).max())), (gs, want)
+    close(m.cpu().numpy(), o_m, RTOL_FP32, "m")
+    close(v.cpu().numpy(), o_v, 3 * RTOL_FP32, "v")      # quadratic in g: twice its relative error, plus rounding
+    dg = th.cpu().numpy().astype(np.float64) - theta
+    do = o_new.astype(np.float64) - theta
+    ulp = 2 * np.spacing(np.abs(theta).astype(np.float32)).astype(np.float64)
+    rms = np.sqrt(np.mean(do ** 2))
+    assert rms > 0
+    assert np.all(np.abs(dg - do) <= RTOL_FP32 * np.abs(do) + RTOL_FP32 * rms + ulp), float(np.abs(dg - do).max())
+    assert ctx.stats()["device_error"] == 0
+
+
+def test_ppo_step_argument_checks(env):
+    torch, orc, binding = env
+    f = fields_for(env_kind=0, n_envs=32, obs_dim=4, n_actions=2, hidden=32, epsilon=0.1, seed=5, replay_capacity=32 * 8,
+                   minibatch=64, staleness_bound=8, warmup=32, target_sync_interval=10, gamma=0.99, huber_delta=1.0)
+    ctx = binding.Context(**f)                                      # a Q-head context has no PPO update
+    z = torch.zeros(64, device=ctx.device)
+    b = binding.TjPpoBatch(8, z.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr())
+    th, m, v = torch.zeros(10, device=ctx.device), torch.zeros(10, device=ctx.device), torch.zeros(10, device=ctx.device)
+    st = binding.tj_ppo_step(ctx.h, b, 1e-3, 0.9, 0.999, 1e-8, 1, 0.2, 0.5, 0.01, th.data_ptr(), m.data_ptr(), v.data_ptr(), 0)
+    assert st == binding.TJ_ERR_UNSUPPORTED
+    st = binding.tj_ppo_step(ctx.h, b, 1e-3, 0.9, 0.999, 1e-8, 0, 0.2, 0.5, 0.01, th.data_ptr(), m.data_ptr(), v.data_ptr(), 0)
+    assert st == binding.TJ_ERR_INVALID_ARG

@@ -148,7 +148,7 @@ def test_adam_step_matches_oracle(env, kind, D, A, H, N, B):
                                             0.99, 1.0, lr, b1, b2, eps, 5, m0, v0)
     assert abs(float(loss.item()) - o_loss) <= 2 * RTOL_FP32 * (abs(o_loss) + 1e-3)
     close(m.cpu().numpy(), o_m, RTOL_FP32, "m")
-    close(v.cpu().numpy(), o_v, RTOL_FP32, "v")
+    close(v.cpu().numpy(), o_v, 3 * RTOL_FP32, "v")      # quadratic in g: twice its relative error, plus rounding
     dg = th.cpu().numpy().astype(np.float64) - theta
     do = o_new.astype(np.float64) - theta
     for name, a, b in _groups(D, H, A):
