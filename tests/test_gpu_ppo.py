@@ -86,3 +86,14 @@ def test_ppo_step_argument_checks(env):
     assert st == binding.TJ_ERR_UNSUPPORTED
     st = binding.tj_ppo_step(ctx.h, b, 1e-3, 0.9, 0.999, 1e-8, 0, 0.2, 0.5, 0.01, th.data_ptr(), m.data_ptr(), v.data_ptr(), 0)
     assert st == binding.TJ_ERR_INVALID_ARG
+
+
+def test_cartpole_ppo_learns_and_respects_the_segment_staleness_bound(env):
+    """The on-policy path as one system: rollout segments -> acquire -> GAE -> PPO minibatches -> publish.  With the consumed
+    segment two versions behind (lag 2) the policy must still pass a mean return of 300 within 2.6 M env steps (it needs
+    1.5-1.8 M), every consumed segment must be at most `lag` versions old and none may be dropped."""
+    from paper_2502_20190_b200 import train_ppo
+    hist = train_ppo.train(lag=2, iters=80, seed=1)
+    assert hist[0]["mean_return"] < 40
+    assert train_ppo.env_steps_to(hist, 300) is not None, [round(r["mean_return"]) for r in hist]
+    assert max(r["segment_lag"] for r in hist) == 2 and hist[-1]["dropped_stale"] == 0
