@@ -2,13 +2,15 @@
 // network, action selection, z = A s, env epilogue, record and reset in one persistent kernel whose roles overlap.
 //
 // A thread block owns 128 rows (envs) per tile, one row per TMEM lane, and walks tiles persistently.  Roles:
-//   warp 0, one lane    producer: streams 16 KB operand chunks (weights, env matrix parts) from L2 into a 4-slot ring
+//   warp 0, one lane    producer: streams operand chunks (32 KB of weights, 16 KB of the env matrix) from L2 into a ring of
+//                       two 32 KB slots
 //   warp 1, one lane    MMA issuer (tcgen05.mma, M = 128, N = 128 per hidden block)
-//   warps 4-11          network warps (two threads per row): state row -> BF16 (layer-1 operand) and TF32 high/low parts
-//                       (operand of z = A s), the record's observation; per 128-neuron block of a hidden layer:
-//                       accumulator -> bias, ReLU, BF16 -> next layer's operand; z -> the record's next_obs field, as scratch
-//   warps 12-19         env warps (two threads per row): take the head outputs out of TMEM, select the action, read z back
-//                       and finish the step (tanh, Philox noise, reward, done, record, reset or new state, counters)
+//   warps 4-11          network warps (two threads per row): state rows -> BF16 (layer-1 operand); per 128-neuron block of a
+//                       hidden layer:
+//                       accumulator -> bias, ReLU, BF16 -> next layer's operand; z -> a scratch tile in global memory
+//   warps 12-19         env warps: the TF32 parts of the next tile's state rows and the record's observation; take the head
+//                       outputs out of TMEM, select the action, read z back and finish the step (tanh, Philox noise, reward,
+//                       done, record, reset or new state, counters), eight rows x four 16-byte pieces per warp instruction
 // The env warps work on tile i while the network warps and the tensor pipe are already on tile i + 1.
 //
 // Per tile the tensor pipe runs ten accumulator blocks that alternate between two 128-column accumulators:
@@ -45,12 +47,12 @@ constexpr int PA_MAX_GRID = 192;           // thread blocks the z scratch is siz
 struct PaSmem {
   uint64_t full[PA_STAGES], empty[PA_STAGES];
   uint64_t x_ready;        // network -> MMA: X holds the tile's BF16 rows
-  uint64_t u_ready;        // network -> MMA: U holds the tile's TF32 high / low parts
+  uint64_t u_ready;        // env -> MMA: U holds the tile's TF32 high / low parts
   uint64_t acc_full[2];    // MMA -> network: an accumulator block is complete
   uint64_t acc_empty[2];   // network -> MMA: it has been drained (and its result stored)
   uint64_t head_full;      // MMA -> env and network: head outputs complete; U may be rewritten
   uint64_t env_taken;      // env -> MMA: head outputs are in registers
-  uint64_t z_stored;       // network -> env: z of the tile is in the records
+  uint64_t z_stored;       // network -> env: z of the tile is in the scratch tile
   uint64_t act_ready;      // env: the rows' actions are in shared memory
   int act[2][PA_M];        // by tile parity
   uint32_t tmem_base;
@@ -73,7 +75,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
   // Thread blocks walk the neuron blocks of a layer in rotated order, so that at any moment they stream different
   // parts of the weights from L2 (the arithmetic per neuron is unchanged)
   const int rot = (int)(blockIdx.x % (unsigned)n_hb);
-  const int n_kc2 = H / PA_KC;           // 64-wide K chunks of layer 2 (layer 1 has two)
+  const int n_kc2 = H / PA_KC;           // K chunks of a layer-2 block (a layer-1 block has PA_D / PA_KC)
 
   if (tid == 0) {
     for (int s = 0; s < PA_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
@@ -106,8 +108,8 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------------- producer
-      // order per tile (the order the MMA issuer consumes): layer 1 (2 chunks per block), env matrix (4 high, 4 low),
-      // layer 2 (H/64 chunks per block), head
+      // order per tile (the order the MMA issuer consumes): layer 1 (one chunk per block), env matrix (4 high, 4 low),
+      // layer 2 (H/128 chunks per block), head
       uint32_t it = 0;
       const uint32_t head_bytes = (uint32_t)PA_N3 * H * 2;
       const int n1 = n_hb * (PA_D / PA_KC), n2 = n_hb * n_kc2;
@@ -145,7 +147,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       };
       for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tiles) {
         if (!tc_wait(&ctl->x_ready, tiles & 1, abort_flag)) goto done;
-        // layer 1: per 128-neuron block two chunks (128 x 64); A operand = X in shared memory
+        // layer 1: per 128-neuron block PA_D / PA_KC chunks; A operand = X in shared memory
         for (int b = 0; b < n_hb; ++b) {
           const int u = b;
           if (!acquire(u)) goto done;
@@ -191,7 +193,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           }
           umma_commit((u & 1) ? &ctl->acc_full[1] : &ctl->acc_full[0]);
         }
-        // layer 2: per block H/64 chunks; A operand = h1 in tensor memory (8 columns per K = 16); the drain of the last
+        // layer 2: per block H / PA_KC chunks; A operand = h1 in tensor memory (8 columns per K = 16); the drain of the last
         // layer-1 block (awaited by the first block here) completes h1
         for (int b = 0; b < n_hb; ++b) {
           const int u = n_hb + 1 + b;
