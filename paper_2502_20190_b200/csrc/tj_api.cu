@@ -102,7 +102,7 @@ size_t carve(tj_ctx* x, void* base) {
     x->sgd_scratch = nullptr;
     if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_EPS_GREEDY && sgd_supported(D, c.hidden, c.n_actions)) {
       x->sgd_rows = c.minibatch;
-      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(c.minibatch, c.hidden));
+      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(c.minibatch, D, c.hidden));
     }
   } else {
     const size_t TN = (size_t)c.rollout_len * N, G = c.n_segments;
@@ -116,7 +116,7 @@ size_t carve(tj_ctx* x, void* base) {
     x->sgd_scratch = nullptr;
     if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_CATEGORICAL && sgd_supported(D, c.hidden, c.n_actions + 1)) {
       x->sgd_rows = c.minibatch > 0 ? c.minibatch : 4096;
-      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(x->sgd_rows, c.hidden));
+      x->sgd_scratch = cv.take<float>(sgd_scratch_floats(x->sgd_rows, D, c.hidden));
     }
   }
   if (c.env_kind == TJ_ENV_LINGAUSS) {

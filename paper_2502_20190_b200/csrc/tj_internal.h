@@ -196,7 +196,7 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
 cudaError_t launch_td(const TdParams& p, cudaStream_t s);
 int td_grid(int n);
-size_t sgd_scratch_floats(int max_rows, int H);
+size_t sgd_scratch_floats(int max_rows, int D, int H);   // the largest gradient matrix is H x max(H, D)
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam /* nullable: plain SGD */, cudaStream_t s);

@@ -338,11 +338,11 @@ __global__ void sgd_apply_adam_kernel(float* __restrict__ Cm, float* __restrict_
 
 }  // namespace
 
-size_t sgd_scratch_floats(int max_rows, int H) {
+size_t sgd_scratch_floats(int max_rows, int D, int H) {
   const size_t rows = ((size_t)max_rows + SG_ROWS - 1) / SG_ROWS * SG_ROWS;
   // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), partial gradient sums of the
   // largest matrix
-  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * H * (size_t)(H > 16 ? H : 16);
+  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * H * (size_t)(H > D ? (H > 17 ? H : 17) : (D > 17 ? D : 17));
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }

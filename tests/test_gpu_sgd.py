@@ -34,7 +34,7 @@ def _groups(D, H, A):
     return [(names[i], int(offs[i]), int(offs[i + 1])) for i in range(6)]
 
 
-@pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (1, 6, 3, 96, 50, 333), (2, 16, 5, 200, 40, 77),
+@pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (1, 6, 3, 96, 50, 333), (2, 16, 5, 200, 40, 77), (2, 48, 4, 32, 40, 100),
                                             (0, 4, 2, 256, 128, 1024)])
 def test_sgd_step_matches_oracle(env, kind, D, A, H, N, B):
     torch, orc, binding = env
