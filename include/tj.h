@@ -13,7 +13,9 @@
  *   learner (Sec. 3.1, learner loop; Sec. 3.3 and Eq. 2-3 for staleness control):
  *           staleness-bounded minibatch sampling, gather, online/target forward,
  *           TD target and Huber error (Algorithm 1, TD-error line); GAE for the
- *           on-policy case (Table 2: gae 0.95, gamma 0.99)
+ *           on-policy case (Table 2: gae 0.95, gamma 0.99); the parameter update
+ *           (Algorithm 1, update line) as an FP32 SGD / Adam step on that loss, and
+ *           PPO's clipped surrogate for the on-policy case (Sec. 4.1)
  *   weights (dependency I relaxed): the learner publishes a new parameter version,
  *           the actor picks up the newest one at its next call.
  *
