@@ -1,0 +1,56 @@
+"""Production / consumption balance on one GPU (Sec. 3.3, Eq. 2-3 of the paper, read for a time-shared device).
+
+The paper fixes the share of consumed to produced samples, P = B_s / N_s' (Eq. 2 with N_s' the samples produced per
+consumed batch), and splits M cores between learners and actors so that the training and production throughputs meet
+(Eq. 3: max min(TR_L, TR_A) s.t. N_c / N_s' = P, M_L + M_A = M, TR_L ~ TR_A).  On one GPU the resource that is split is
+time: with R_A env steps per second while only the actor runs and R_L samples per second while only the learner runs, a
+fraction f of the time on the actor produces f R_A and the rest consumes (1 - f) R_L.  The constraint
+(1 - f) R_L = P f R_A gives f = R_L / (R_L + P R_A): both sides then run exactly as fast as the ratio allows, which is
+the balanced point (more actor time would only produce samples that are never consumed, Table 1's L2A16 / L2A24 rows).
+Host arithmetic only; nothing here touches the GPU."""
+from __future__ import annotations
+
+import math
+
+
+def actor_steps_per_learner_step(P: float, minibatch: int, n_envs: int) -> int:
+    """How many env steps of all n_envs the actor takes per learner step so that consumed / produced = P:
+    minibatch / (k * n_envs) = P, k rounded to the nearest positive integer."""
+    if P <= 0 or minibatch <= 0 or n_envs <= 0:
+        raise ValueError("P, minibatch and n_envs must be positive")
+    return max(1, int(round(minibatch / (P * n_envs))))
+
+
+def realised_ratio(k: int, minibatch: int, n_envs: int) -> float:
+    """consumed / produced with k actor steps per learner step"""
+    return minibatch / (k * n_envs)
+
+
+def time_share(R_A: float, R_L: float, P: float) -> dict:
+    """The balanced split of device time.  R_A: env steps/s of the actor alone, R_L: samples/s of the learner alone,
+    P: consumed per produced sample.  Returns the actor's time fraction and the two throughputs at that point."""
+    if R_A <= 0 or R_L <= 0 or P <= 0:
+        raise ValueError("rates and P must be positive")
+    f = R_L / (R_L + P * R_A)
+    return dict(actor_fraction=f, produced_per_s=f * R_A, consumed_per_s=(1.0 - f) * R_L)
+
+
+def rates_from_stats(stats: dict, produced: int, consumed: int) -> tuple:
+    """(R_A, R_L) from a context's per-kernel-class times (tj_set_profiling on): classes 0-2 are the actor's kernels,
+    3-4 and 7 the learner's (sample + gather, TD error, update)."""
+    ms = stats["kernel_ms"]
+    t_a = (ms[0] + ms[1] + ms[2]) * 1e-3
+    t_l = (ms[3] + ms[4] + ms[7]) * 1e-3
+    if t_a <= 0 or t_l <= 0:
+        raise ValueError("no timed launches: call tj_set_profiling(1) before the steps")
+    return produced / t_a, consumed / t_l
+
+
+def starved_fraction(staleness_bound: int, publishes_per_block: float) -> float:
+    """Share of sample calls that find nothing eligible when every produced block (one actor step of all envs) is
+    followed by `publishes_per_block` version bumps and only versions within `staleness_bound` may be consumed: a block
+    written at version v is eligible for calls at versions v .. v + S, i.e. for S + 1 of the publishes_per_block calls
+    that follow it before the next block arrives (the consumer-ahead-of-producer case of Sec. 3.3)."""
+    if publishes_per_block <= 0:
+        raise ValueError("publishes_per_block must be positive")
+    return max(0.0, 1.0 - (staleness_bound + 1) / publishes_per_block)
