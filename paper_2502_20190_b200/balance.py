@@ -21,9 +21,22 @@ def actor_steps_per_learner_step(P: float, minibatch: int, n_envs: int) -> int:
     return max(1, int(round(minibatch / (P * n_envs))))
 
 
-def realised_ratio(k: int, minibatch: int, n_envs: int) -> float:
-    """consumed / produced with k actor steps per learner step"""
-    return minibatch / (k * n_envs)
+def realised_ratio(k: int, minibatch: int, n_envs: int, updates: int = 1) -> float:
+    """consumed / produced with k actor steps per `updates` learner steps"""
+    return updates * minibatch / (k * n_envs)
+
+
+def schedule(P: float, minibatch: int, n_envs: int) -> tuple:
+    """(k, u): k actor steps of all n_envs, then u learner steps, so that u * minibatch / (k * n_envs) is as close to P as
+    whole numbers allow with one of the two equal to 1 (the cadence that keeps the consumed samples freshest: the learner
+    never waits for more than one block when it consumes faster than one minibatch per block, and never runs more than
+    its share ahead otherwise)."""
+    if P <= 0 or minibatch <= 0 or n_envs <= 0:
+        raise ValueError("P, minibatch and n_envs must be positive")
+    per_block = P * n_envs / minibatch            # learner steps per actor step at ratio P
+    if per_block >= 1.0:
+        return 1, max(1, int(round(per_block)))
+    return max(1, int(round(1.0 / per_block))), 1
 
 
 def time_share(R_A: float, R_L: float, P: float) -> dict:
@@ -37,10 +50,10 @@ def time_share(R_A: float, R_L: float, P: float) -> dict:
 
 def rates_from_stats(stats: dict, produced: int, consumed: int) -> tuple:
     """(R_A, R_L) from a context's per-kernel-class times (tj_set_profiling on): classes 0-2 are the actor's kernels,
-    3-4 and 7 the learner's (sample + gather, TD error, update)."""
+    3-5 and 7 the learner's (sample + gather, TD error, the publish that hands each new version over, update)."""
     ms = stats["kernel_ms"]
     t_a = (ms[0] + ms[1] + ms[2]) * 1e-3
-    t_l = (ms[3] + ms[4] + ms[7]) * 1e-3
+    t_l = (ms[3] + ms[4] + ms[5] + ms[7]) * 1e-3
     if t_a <= 0 or t_l <= 0:
         raise ValueError("no timed launches: call tj_set_profiling(1) before the steps")
     return produced / t_a, consumed / t_l

@@ -10,16 +10,20 @@ from __future__ import annotations
 
 import argparse
 import json
+import time
 
 import numpy as np
 
-from . import binding, synth
+from . import balance, binding, synth
 
 
 def train(staleness_bound=8, iters=1500, n_envs=1024, hidden=64, minibatch=1024, updates_per_iter=4, lr=5e-4,
-          target_every=200, epsilon=0.1, seed=1, report_every=100, device=0):
-    """Runs `iters` iterations of (one env step of every env, `updates_per_iter` learner steps, each followed by a
-    publish).  Returns a list of dicts: iteration, env steps, mean return of the episodes finished since the last report."""
+          target_every=200, epsilon=0.1, seed=1, report_every=100, device=0, actor_steps_per_iter=1, rates_out=None):
+    """Runs `iters` iterations of (`actor_steps_per_iter` env steps of every env, `updates_per_iter` learner steps, each
+    followed by a publish).  Returns a list of dicts: iteration, env steps, mean return of the episodes finished since the
+    last report.  With `rates_out` (a dict) the per-kernel times are recorded and the dict receives the actor's and the
+    learner's stand-alone rates (Eq. 3's TR_A, TR_L: env steps and consumed samples per second of their own kernel time),
+    the balanced time split for the realised ratio and the throughput that split predicts."""
     import torch
     torch.cuda.set_device(device)
     f = synth.config_fields({}, env_kind=synth.ENV_CARTPOLE, n_envs=n_envs, obs_dim=4, n_actions=2, hidden=hidden,
@@ -32,9 +36,13 @@ def train(staleness_bound=8, iters=1500, n_envs=1024, hidden=64, minibatch=1024,
     m, v = torch.zeros_like(theta), torch.zeros_like(theta)
     batch = ctx.alloc_batch()
     ctx.publish_weights(theta)
+    if rates_out is not None:
+        ctx.set_profiling(1)
     hist, t_adam, last_eps, last_ret, starved = [], 0, 0, 0.0, 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
     for it in range(1, iters + 1):
-        ctx.actor_step(1)
+        ctx.actor_step(actor_steps_per_iter)
         for _ in range(updates_per_iter):
             st, _ = ctx.replay_sample(batch=batch, allow=(0, binding.TJ_ERR_WARMUP, binding.TJ_ERR_STARVED))
             if st != 0:
@@ -50,8 +58,16 @@ def train(staleness_bound=8, iters=1500, n_envs=1024, hidden=64, minibatch=1024,
             n_ep = s["episodes_finished"] - last_eps
             mean_ret = (s["return_sum"] - last_ret) / n_ep if n_ep else float("nan")
             last_eps, last_ret = s["episodes_finished"], s["return_sum"]
-            hist.append(dict(iter=it, env_steps=it * n_envs, updates=t_adam, episodes=int(n_ep), mean_return=float(mean_ret),
+            hist.append(dict(iter=it, env_steps=it * n_envs * actor_steps_per_iter, updates=t_adam, episodes=int(n_ep), mean_return=float(mean_ret),
                              max_sampled_staleness=int(s["max_sampled_staleness"]), starved=starved))
+    torch.cuda.synchronize()
+    loop_s = time.perf_counter() - t0
+    if rates_out is not None:
+        produced, consumed = iters * actor_steps_per_iter * n_envs, t_adam * minibatch
+        R_A, R_L = balance.rates_from_stats(ctx.stats(), produced, consumed)
+        P = consumed / produced
+        rates_out.update(R_A=R_A, R_L=R_L, P=P, loop_s=loop_s, loop_produced_per_s=produced / loop_s,
+                         kernel_s=sum(ctx.stats()["kernel_ms"]) * 1e-3, **balance.time_share(R_A, R_L, P))
     return hist
 
 
@@ -62,11 +78,16 @@ def main():
     ap.add_argument("--envs", type=int, default=1024)
     ap.add_argument("--hidden", type=int, default=64)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--ratio", type=float, default=None,
+                    help="consumed : produced samples (Eq. 2's P); sets the actor / learner cadence through balance.schedule")
     a = ap.parse_args()
+    k, u = (1, 4) if a.ratio is None else balance.schedule(a.ratio, 1024, a.envs)
     for S in a.staleness:
-        h = train(staleness_bound=S, iters=a.iters, n_envs=a.envs, hidden=a.hidden, seed=a.seed)
-        print(json.dumps(dict(staleness_bound=S, curve=[(r["env_steps"], round(r["mean_return"], 1)) for r in h],
-                              final=h[-1])))
+        rates = {}
+        h = train(staleness_bound=S, iters=a.iters, n_envs=a.envs, hidden=a.hidden, seed=a.seed, actor_steps_per_iter=k,
+                  updates_per_iter=u, rates_out=rates)
+        print(json.dumps(dict(staleness_bound=S, actor_steps_per_iter=k, updates_per_iter=u, balance=rates,
+                              curve=[(r["env_steps"], round(r["mean_return"], 1)) for r in h], final=h[-1])))
 
 
 if __name__ == "__main__":

@@ -26,6 +26,19 @@ def test_ratio_and_time_share_closed_forms():
         balance.time_share(0, 1, 1)
 
 
+def test_schedule_realises_the_ratio_with_whole_steps():
+    for P, B, N in [(1 / 16, 1024, 4096), (4.0, 1024, 1024), (1.0, 4096, 1024), (1 / 8, 512, 512), (1.0, 1024, 1024)]:
+        k, u = balance.schedule(P, B, N)
+        assert min(k, u) == 1
+        assert balance.realised_ratio(k, B, N, u) == pytest.approx(P)
+    # not representable exactly: the nearest whole cadence
+    k, u = balance.schedule(0.3, 1024, 1024)
+    assert (k, u) == (3, 1) and balance.realised_ratio(k, 1024, 1024, u) == pytest.approx(1 / 3)
+    assert balance.schedule(2.4, 1024, 1024) == (1, 2)
+    with pytest.raises(ValueError):
+        balance.schedule(0, 1, 1)
+
+
 @pytest.mark.parametrize("S,publishes", [(0, 4), (1, 4), (3, 4), (1, 2), (2, 8)])
 def test_starved_share_matches_the_oracle_sampler(S, publishes):
     """One actor step (one block), then `publishes` rounds of sample + publish, repeated: the oracle's sampler starves in

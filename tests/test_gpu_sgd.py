@@ -187,3 +187,22 @@ def test_cartpole_dqn_learns_through_the_library(env):
     assert hist[0]["mean_return"] < 15
     assert best > 60, [round(r["mean_return"], 1) for r in hist]
     assert hist[-1]["max_sampled_staleness"] <= 8 and hist[-1]["updates"] > 4000
+
+
+@pytest.mark.gpu
+def test_measured_rates_give_the_balanced_split():
+    """Eq. 2-3 from measured rates: the loop at consumed : produced = 1 : 8 reports stand-alone actor and learner rates,
+    and the balanced time split built from them predicts a throughput the measured loop cannot exceed (kernel time is part
+    of the loop's wall time) and is not far below."""
+    from paper_2502_20190_b200 import balance, train_dqn
+    k, u = balance.schedule(0.125, 1024, 1024)
+    assert (k, u) == (8, 1)
+    rates = {}
+    h = train_dqn.train(staleness_bound=8, iters=200, actor_steps_per_iter=k, updates_per_iter=u, rates_out=rates)
+    assert h[-1]["env_steps"] == 200 * 8 * 1024 and h[-1]["updates"] > 0
+    assert rates["P"] == pytest.approx(h[-1]["updates"] * 1024 / h[-1]["env_steps"])
+    assert rates["R_A"] > 0 and rates["R_L"] > 0 and 0 < rates["actor_fraction"] < 1
+    assert rates["consumed_per_s"] == pytest.approx(rates["P"] * rates["produced_per_s"])
+    assert rates["kernel_s"] <= rates["loop_s"]
+    assert rates["loop_produced_per_s"] <= rates["produced_per_s"] * 1.001
+    assert rates["loop_produced_per_s"] >= 0.2 * rates["produced_per_s"]
