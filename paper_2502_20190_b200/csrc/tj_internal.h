@@ -106,7 +106,7 @@ struct SgdParams {
   float *h1, *h2, *dh1, *dh2;  // scratch [n][H] each
   float* g;                    // scratch [n][A]: dL/dq, non-zero at the selected action only
   float* partial;              // scratch: one Huber partial sum per 16 rows
-  float* grad_partial;         // scratch: per row range partial sums of one gradient matrix
+  float* grad_partial;         // scratch: per row range one partial gradient laid out like the parameter blob
   int ldg;                     // row stride of g (A for the Q head, A + 1 with the value head's entry in column A)
   int value_head;              // 1: policy + value heads (PPO), theta carries Wv, bv after b3
   // PPO only
@@ -196,7 +196,7 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
 cudaError_t launch_td(const TdParams& p, cudaStream_t s);
 int td_grid(int n);
-size_t sgd_scratch_floats(int max_rows, int D, int H);   // the largest gradient matrix is H x max(H, D)
+size_t sgd_scratch_floats(int max_rows, int D, int H);   // activations, deltas and 32 partial gradients of the blob
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam /* nullable: plain SGD */, cudaStream_t s);

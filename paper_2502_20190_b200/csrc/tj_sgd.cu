@@ -272,17 +272,35 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_backward_kernel(const SgdParam
 
 constexpr int SG_SPLITS = 32;     // at most this many row ranges per gradient product (partial sums go through scratch)
 
-// P[z][m][n] = sum over the rows j of range z of A[j][m] * Bm[j][n]   (A n_rows x M with row stride lda; Bm n_rows x N,
-// stride ldb; Bm == nullptr stands for a column of ones, N = 1: a bias gradient).  32 x 32 tile per block, 256 threads,
-// each 2 x 2; rows in ascending order.  The row ranges (blockIdx.z) make the reduction over the minibatch parallel; the
-// second kernel adds the partial sums in range order, so the result does not depend on the launch.
-__global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, int M, int N, const float* __restrict__ Am,
-                                                               int lda, const float* __restrict__ Bm, int ldb, int n_rows,
+// One gradient product of the update: C (M x N, at float offset `off` of the parameter blob) gets (Am rows)^T (Bm rows),
+// a bias (Bm == nullptr) a column of ones.  Tiles of all products are numbered in one list: tile_begin is this product's
+// first tile.
+struct GradProduct {
+  const float* Am;
+  const float* Bm;
+  int off, M, N, lda, ldb, tile_begin;
+};
+struct GradProducts {
+  GradProduct g[8];
+  int n, n_tiles;
+};
+
+// Every gradient product of one update in a single launch: thread block (tile, range) sums, over its range of minibatch
+// rows, one 32 x 32 tile of one product and writes it to P[range][off + m * N + n] -- a partial gradient laid out like the
+// parameter blob itself, `count` floats per range.  No atomics: the apply kernel adds the ranges in order.
+__global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, const GradProducts gp, int count, int n_rows,
                                                                int rows_per_range) {
   __shared__ float As[32][33], Bs[32][33];
-  const int m0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  int q = 0;
+  while (q + 1 < gp.n && (int)blockIdx.x >= gp.g[q + 1].tile_begin) ++q;
+  const GradProduct& d = gp.g[q];
+  const int M = d.M, N = d.N, lda = d.lda, ldb = d.ldb;
+  const float* __restrict__ Am = d.Am;
+  const float* __restrict__ Bm = d.Bm;
+  const int tiles_n = (N + 31) / 32, t = blockIdx.x - d.tile_begin;
+  const int m0 = (t / tiles_n) * 32, n0 = (t % tiles_n) * 32;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const int j_begin = blockIdx.z * rows_per_range;
+  const int j_begin = blockIdx.y * rows_per_range;
   const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
   float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
   for (int j0 = j_begin; j0 < j_end; j0 += 32) {
@@ -307,7 +325,7 @@ __global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict
 #pragma unroll
     for (int v = 0; v < 2; ++v) {
       const int m = m0 + ty + 16 * u, n = n0 + tx + 16 * v;
-      if (m < M && n < N) P[((size_t)blockIdx.z * M + m) * N + n] = acc[u][v];
+      if (m < M && n < N) P[(size_t)blockIdx.y * count + d.off + (size_t)m * N + n] = acc[u][v];
     }
 }
 
@@ -340,9 +358,10 @@ __global__ void sgd_apply_adam_kernel(float* __restrict__ Cm, float* __restrict_
 
 size_t sgd_scratch_floats(int max_rows, int D, int H) {
   const size_t rows = ((size_t)max_rows + SG_ROWS - 1) / SG_ROWS * SG_ROWS;
-  // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), partial gradient sums of the
-  // largest matrix
-  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * H * (size_t)(H > D ? (H > 17 ? H : 17) : (D > 17 ? D : 17));
+  // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), and per row range one partial
+  // gradient of the whole parameter blob (at most 16 actions and a value head)
+  const size_t blob = (size_t)H * D + H + (size_t)H * H + H + 17 * (size_t)H + 17;
+  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * blob;
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }
@@ -373,28 +392,38 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
   if (n_ranges > SG_SPLITS) n_ranges = SG_SPLITS;
   const int rows_per_range = ((p.n + n_ranges - 1) / n_ranges + 31) / 32 * 32;
   n_ranges = (p.n + rows_per_range - 1) / rows_per_range;
-  // the backward pass has read W2 and the heads; now the parameters may change
-  auto upd = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
-    sgd_grad_partial_kernel<<<dim3((N + 31) / 32, (M + 31) / 32, n_ranges), 256, 0, s>>>(p.grad_partial, M, N, Am, lda, Bm, ldb, p.n,
-                                                                                       rows_per_range);
-    if (adam) {
-      const size_t off = (size_t)(C - p.theta);
-      sgd_apply_adam_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, adam->m + off, adam->v + off, p.grad_partial, M * N, n_ranges, lr,
-                                                                adam->beta1, adam->beta2, adam->eps, adam->c1, adam->c2);
-    } else {
-      sgd_apply_kernel<<<(M * N + 255) / 256, 256, 0, s>>>(C, p.grad_partial, M * N, n_ranges, lr);
-    }
+  // the backward pass has read W2 and the heads; now the parameters may change: all products in one launch, then one
+  // pass over the whole blob
+  GradProducts gp{};
+  auto add = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
+    GradProduct& d = gp.g[gp.n++];
+    d.Am = Am;
+    d.Bm = Bm;
+    d.off = (int)(C - p.theta);
+    d.M = M;
+    d.N = N;
+    d.lda = lda;
+    d.ldb = ldb;
+    d.tile_begin = gp.n_tiles;
+    gp.n_tiles += ((M + 31) / 32) * ((N + 31) / 32);
   };
-  upd(W3, A, H, p.g, p.ldg, p.h2, H);
-  upd(b3, A, 1, p.g, p.ldg, nullptr, 0);
+  add(W1, H, D, p.dh1, H, p.obs, D);
+  add(b1, H, 1, p.dh1, H, nullptr, 0);
+  add(W2, H, H, p.dh2, H, p.h1, H);
+  add(b2, H, 1, p.dh2, H, nullptr, 0);
+  add(W3, A, H, p.g, p.ldg, p.h2, H);
+  add(b3, A, 1, p.g, p.ldg, nullptr, 0);
   if (p.value_head) {
-    upd(Wv, 1, H, p.g + A, p.ldg, p.h2, H);
-    upd(bv, 1, 1, p.g + A, p.ldg, nullptr, 0);
+    add(Wv, 1, H, p.g + A, p.ldg, p.h2, H);
+    add(bv, 1, 1, p.g + A, p.ldg, nullptr, 0);
   }
-  upd(W2, H, H, p.dh2, H, p.h1, H);
-  upd(b2, H, 1, p.dh2, H, nullptr, 0);
-  upd(W1, H, D, p.dh1, H, p.obs, D);
-  upd(b1, H, 1, p.dh1, H, nullptr, 0);
+  const int count = (int)((p.value_head ? bv + 1 : b3 + A) - p.theta);
+  sgd_grad_partial_kernel<<<dim3(gp.n_tiles, n_ranges), 256, 0, s>>>(p.grad_partial, gp, count, p.n, rows_per_range);
+  if (adam)
+    sgd_apply_adam_kernel<<<(count + 255) / 256, 256, 0, s>>>(p.theta, adam->m, adam->v, p.grad_partial, count, n_ranges, lr, adam->beta1,
+                                                              adam->beta2, adam->eps, adam->c1, adam->c2);
+  else
+    sgd_apply_kernel<<<(count + 255) / 256, 256, 0, s>>>(p.theta, p.grad_partial, count, n_ranges, lr);
   return cudaGetLastError();
 }
 }  // namespace
