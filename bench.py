@@ -156,8 +156,8 @@ class Runner:
         self.version = 0
         self.learner_ok = 0
         # --with-update: the learner also takes a gradient step (tj_sgd_step) and the published parameters are the ones it
-        # trains, instead of the pre-drawn pool (FP32 replay workloads only)
-        self.with_update = bool(with_update) and self.w["replay_capacity"] > 0 and self.w["weight_dtype"] == synth.W_FP32
+        # trains, instead of the pre-drawn pool (replay workloads only; FP32 master parameters in BF16 workloads too)
+        self.with_update = bool(with_update) and self.w["replay_capacity"] > 0
         if self.with_update:
             self.theta = self.dev_blobs[0].clone()
             self.theta_target = self.dev_blobs[0].clone()

@@ -234,7 +234,9 @@ int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float 
  * theta (in/out) and theta_target: device FP32 blobs in the tj_publish_weights layout, distinct buffers, owned by the
  * caller; nothing in the context changes -- publish theta afterwards to hand it to the actor.  batch.n <= the configured
  * minibatch.  loss_mean_out (nullable, device): the loss before the update.  FP32 arithmetic, every sum in a fixed order.
- * TJ_ERR_UNSUPPORTED for BF16 contexts, segment mode and the categorical policy. */
+ * In a BF16 context theta is the FP32 master copy: the update and its loss are FP32 all the same, the rounding to BF16
+ * happens at tj_publish_weights (so this loss differs from tj_td_error's, which uses the published BF16 copy, by that
+ * rounding).  TJ_ERR_UNSUPPORTED for segment mode and the categorical policy. */
 int tj_sgd_step(tj_ctx *ctx, const tj_batch *batch, float lr, float *theta, const float *theta_target, float *loss_mean_out);
 
 /* The same gradient through Adam (the optimiser of Table 2; Kingma & Ba 2015), step counter t >= 1:
@@ -254,7 +256,8 @@ int tj_adam_step(tj_ctx *ctx, const tj_batch *batch, float lr, float beta1, floa
  * segment (tj_segment_acquire) and of tj_gae's outputs can be passed as they lie: obs [n][obs_dim], the others [n].
  * stats_out (nullable, device, 5 floats): L, mean policy term, mean 0.5 (V - R)^2, mean entropy, fraction of rows where
  * the clipped term is the minimum -- all before the update.  batch.n <= the configured minibatch (4096 if none).
- * TJ_ERR_UNSUPPORTED unless the context is FP32 with the categorical policy. */
+ * BF16 contexts: theta is the FP32 master copy, as for tj_sgd_step.
+ * TJ_ERR_UNSUPPORTED unless the context is in segment mode with the categorical policy. */
 typedef struct {
   int32_t n;
   const float *obs;

@@ -100,7 +100,7 @@ size_t carve(tj_ctx* x, void* base) {
     x->elig_count = cv.take<int>(1);
     x->sgd_rows = 0;
     x->sgd_scratch = nullptr;
-    if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_EPS_GREEDY && sgd_supported(D, c.hidden, c.n_actions)) {
+    if (c.policy_kind == TJ_POLICY_EPS_GREEDY && sgd_supported(D, c.hidden, c.n_actions)) {
       x->sgd_rows = c.minibatch;
       x->sgd_scratch = cv.take<float>(sgd_scratch_floats(c.minibatch, D, c.hidden));
     }
@@ -114,7 +114,7 @@ size_t carve(tj_ctx* x, void* base) {
     x->seg_done = cv.take<uint8_t>(G * TN);
     x->sgd_rows = 0;
     x->sgd_scratch = nullptr;
-    if (c.weight_dtype == TJ_W_FP32 && c.policy_kind == TJ_POLICY_CATEGORICAL && sgd_supported(D, c.hidden, c.n_actions + 1)) {
+    if (c.policy_kind == TJ_POLICY_CATEGORICAL && sgd_supported(D, c.hidden, c.n_actions + 1)) {
       x->sgd_rows = c.minibatch > 0 ? c.minibatch : 4096;
       x->sgd_scratch = cv.take<float>(sgd_scratch_floats(x->sgd_rows, D, c.hidden));
     }
@@ -564,7 +564,8 @@ int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const f
   if (!theta || !theta_target) return fail(x, TJ_ERR_INVALID_ARG, "parameter blobs must not be null");
   if (theta == theta_target) return fail(x, TJ_ERR_INVALID_ARG, "theta and theta_target must be different buffers");
   if (!(lr >= 0.f)) return fail(x, TJ_ERR_INVALID_ARG, "lr must not be negative");
-  if (!x->sgd_scratch) return fail(x, TJ_ERR_UNSUPPORTED, "the learner update is implemented for FP32 replay contexts with the Q head");
+  if (!x->sgd_scratch || x->cfg.policy_kind != TJ_POLICY_EPS_GREEDY || x->cfg.replay_capacity <= 0)
+    return fail(x, TJ_ERR_UNSUPPORTED, "the learner update is implemented for replay contexts with the Q head");
   if (b->n < 1 || b->n > x->sgd_rows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be between 1 and the configured minibatch");
   SgdParams p{};
   p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A;
@@ -613,7 +614,7 @@ int tj_ppo_step(tj_ctx* x, const tj_ppo_batch* b, float lr, float beta1, float b
     return fail(x, TJ_ERR_INVALID_ARG, "needs lr >= 0, 0 <= beta1, beta2 < 1 and eps > 0");
   if (!(clip_eps >= 0.f && clip_eps < 1.f)) return fail(x, TJ_ERR_INVALID_ARG, "clip_eps must lie in [0, 1)");
   if (x->cfg.policy_kind != TJ_POLICY_CATEGORICAL || !x->sgd_scratch)
-    return fail(x, TJ_ERR_UNSUPPORTED, "the PPO update is implemented for FP32 contexts with the categorical policy and value head");
+    return fail(x, TJ_ERR_UNSUPPORTED, "the PPO update is implemented for segment contexts with the categorical policy and value head");
   if (b->n < 1 || b->n > x->sgd_rows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be between 1 and the configured minibatch (4096 if none)");
   SgdParams p{};
   p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A;

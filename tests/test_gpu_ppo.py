@@ -25,12 +25,13 @@ def env():
     return torch, oracle, binding
 
 
-@pytest.mark.parametrize("kind,D,A,H,N,T,B", [(0, 4, 2, 64, 48, 8, 300), (1, 6, 3, 128, 40, 10, 257)])
-def test_ppo_step_matches_oracle(env, kind, D, A, H, N, T, B):
+@pytest.mark.parametrize("kind,D,A,H,N,T,B,wdt", [(0, 4, 2, 64, 48, 8, 300, 0), (1, 6, 3, 128, 40, 10, 257, 0),
+                                                  (0, 4, 2, 64, 48, 8, 200, 1)])       # last: BF16 context, FP32 master blob
+def test_ppo_step_matches_oracle(env, kind, D, A, H, N, T, B, wdt):
     torch, orc, binding = env
     f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, policy_kind=1, seed=99, replay_capacity=0,
                    rollout_len=T, n_segments=2, staleness_bound=4, minibatch=B, gamma=0.99, gae_lambda=0.95,
-                   max_episode_steps=7)
+                   max_episode_steps=7, weight_dtype=wdt)
     ctx = binding.Context(**f)
     theta_old = blob_for(f, 1)
     ctx.publish_weights(theta_old)

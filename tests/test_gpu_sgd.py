@@ -37,10 +37,21 @@ def _groups(D, H, A):
 @pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (1, 6, 3, 96, 50, 333), (2, 16, 5, 200, 40, 77), (2, 48, 4, 32, 40, 100),
                                             (0, 4, 2, 256, 128, 1024)])
 def test_sgd_step_matches_oracle(env, kind, D, A, H, N, B):
+    _check_sgd_step(env, kind, D, A, H, N, B, 0)
+
+
+@pytest.mark.parametrize("kind,D,A,H,N,B", [(2, 32, 4, 64, 128, 300), (2, 128, 7, 128, 256, 500)])
+def test_sgd_step_in_a_bf16_context_updates_the_fp32_master_copy(env, kind, D, A, H, N, B):
+    """A BF16 context (the second shape runs the pipelined tensor-core actor) rounds the parameters at publish only: the
+    update itself is the FP32 one, on the caller's FP32 blob, and matches the same oracle step."""
+    _check_sgd_step(env, kind, D, A, H, N, B, 1)
+
+
+def _check_sgd_step(env, kind, D, A, H, N, B, weight_dtype):
     torch, orc, binding = env
     f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, epsilon=0.3, seed=777, replay_capacity=N * 16,
                    minibatch=B, staleness_bound=20, warmup=N, target_sync_interval=1000, gamma=0.99, huber_delta=1.0,
-                   max_episode_steps=9)
+                   max_episode_steps=9, weight_dtype=weight_dtype)
     ctx = binding.Context(**f)
     theta_t = blob_for(f, 1)            # the first publish also becomes the target
     theta = blob_for(f, 2)
@@ -102,13 +113,11 @@ def test_sgd_step_argument_checks(env):
     before = th.clone()
     ctx.sgd_step(batch, 0.0, th, tt)
     assert torch.equal(before, th)
-    # a BF16 context refuses the call
-    f2 = fields_for(env_kind=2, n_envs=128, obs_dim=32, n_actions=4, hidden=64, epsilon=0.1, seed=5, replay_capacity=128 * 4,
-                    minibatch=64, staleness_bound=8, warmup=128, target_sync_interval=10, gamma=0.99, huber_delta=1.0,
-                    weight_dtype=1)
+    # a segment-mode context (categorical policy) has no Q-learning update
+    f2 = fields_for(env_kind=0, n_envs=32, obs_dim=4, n_actions=2, hidden=32, policy_kind=1, seed=5, replay_capacity=0,
+                    rollout_len=4, n_segments=2, staleness_bound=1, minibatch=64)
     c2 = binding.Context(**f2)
-    b2 = c2.alloc_batch(8)
-    st = binding.tj_sgd_step(c2.h, b2["c"], 0.1, th.data_ptr(), tt.data_ptr(), 0)
+    st = binding.tj_sgd_step(c2.h, batch["c"], 0.1, th.data_ptr(), tt.data_ptr(), 0)
     assert st == binding.TJ_ERR_UNSUPPORTED
 
 
