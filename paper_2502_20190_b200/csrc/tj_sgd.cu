@@ -132,6 +132,143 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// Wide networks and large minibatches: the layers as tiled FP32 matrix products (a weight element is reused for 128 rows
+// instead of 16).  C[m][n] = epi(sum_k A[m][k] Bop[k][n]): A row-major M x K.  B_KN false: B is N x K row-major (a weight
+// matrix as the forward pass uses it, Bop = B^T); true: B is K x N row-major (the same matrix in the backward pass).
+// 128 x 64 tile per block, 16 k per step, each thread 8 x 4; k ascending, one accumulator per output: a fixed order.
+constexpr int GM_BM = 128, GM_BN = 64, GM_BK = 16, GM_THREADS = 256;
+enum { GM_BIAS_RELU = 0, GM_BIAS = 1, GM_MASK = 2 };   // relu(acc + bias[n]) | acc + bias[n] | acc where mask[m][n] > 0, else 0
+
+template <bool B_KN, int EPI>
+__global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+                                                             float* __restrict__ C, int ldc, int M, int N, int K,
+                                                             const float* __restrict__ bias, const float* __restrict__ mask, int ldm) {
+  __shared__ __align__(16) float As[GM_BK][GM_BM + 4];
+  __shared__ __align__(16) float Bs[GM_BK][GM_BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * GM_BM, n0 = blockIdx.x * GM_BN;
+  const bool vecA = (lda & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0;
+  const bool vecB = (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0;
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  // four consecutive k of one row (of A, or of an N x K B): a 16-byte load where the row allows it
+  auto load_k4 = [](const float* base, int ld, int row, int n_rows, int k, int K, bool vec) -> float4 {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row < n_rows && k < K) {
+      const float* src = base + (size_t)row * ld + k;
+      if (vec && k + 3 < K) {
+        v = __ldg(reinterpret_cast<const float4*>(src));
+      } else {
+        v.x = __ldg(src);
+        if (k + 1 < K) v.y = __ldg(src + 1);
+        if (k + 2 < K) v.z = __ldg(src + 2);
+        if (k + 3 < K) v.w = __ldg(src + 3);
+      }
+    }
+    return v;
+  };
+  for (int k0 = 0; k0 < K; k0 += GM_BK) {
+#pragma unroll
+    for (int i = tid; i < GM_BM * 4; i += GM_THREADS) {
+      const int r = i >> 2, kq = (i & 3) * 4;
+      const float4 v = load_k4(A, lda, m0 + r, M, k0 + kq, K, vecA);
+      As[kq][r] = v.x; As[kq + 1][r] = v.y; As[kq + 2][r] = v.z; As[kq + 3][r] = v.w;
+    }
+    if (!B_KN) {
+      const int r = tid >> 2, kq = (tid & 3) * 4;
+      const float4 v = load_k4(B, ldb, n0 + r, N, k0 + kq, K, vecB);
+      Bs[kq][r] = v.x; Bs[kq + 1][r] = v.y; Bs[kq + 2][r] = v.z; Bs[kq + 3][r] = v.w;
+    } else {
+      const int kk = tid >> 4, nq = (tid & 15) * 4, k = k0 + kk, n = n0 + nq;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (k < K && n < N) {
+        const float* src = B + (size_t)k * ldb + n;
+        if (vecB && n + 3 < N) {
+          v = __ldg(reinterpret_cast<const float4*>(src));
+        } else {
+          v.x = __ldg(src);
+          if (n + 1 < N) v.y = __ldg(src + 1);
+          if (n + 2 < N) v.z = __ldg(src + 2);
+          if (n + 3 < N) v.w = __ldg(src + 3);
+        }
+      }
+      *reinterpret_cast<float4*>(&Bs[kk][nq]) = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < GM_BK; ++kk) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][ty * 8 + 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int m = m0 + ty * 8 + i;
+    if (m >= M) break;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= N) break;
+      float v = acc[i][j];
+      if (EPI == GM_BIAS_RELU) v = fmaxf(v + __ldg(bias + n), 0.f);
+      else if (EPI == GM_BIAS) v = v + __ldg(bias + n);
+      else v = __ldg(mask + (size_t)m * ldm + n) > 0.f ? v : 0.f;
+      C[(size_t)m * ldc + n] = v;
+    }
+  }
+}
+
+template <bool B_KN, int EPI>
+void sg_gemm(const float* A, int lda, const float* B, int ldb, float* C, int ldc, int M, int N, int K, const float* bias,
+             const float* mask, int ldm, cudaStream_t s) {
+  sg_gemm_kernel<B_KN, EPI><<<dim3((N + GM_BN - 1) / GM_BN, (M + GM_BM - 1) / GM_BM), GM_THREADS, 0, s>>>(A, lda, B, ldb, C, ldc, M, N, K,
+                                                                                                     bias, mask, ldm);
+}
+
+// TD error, Huber loss and its gradient at the outputs from the two networks' Q values: q (in) and g (out) share p.g
+// ([n][A]: a row is read, then overwritten by its own thread), qt [n][A]; loss partials per SG_ROWS rows as in the
+// fused forward kernel
+__global__ void __launch_bounds__(32) sgd_loss_kernel(const SgdParams p, const float* __restrict__ qt) {
+  __shared__ float hub[SG_ROWS];
+  const int r = threadIdx.x, j = blockIdx.x * SG_ROWS + r, A = p.A;
+  if (r < SG_ROWS) {
+    float h = 0.f;
+    if (j < p.n) {
+      int a = p.act[j];
+      a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+      float* gr = p.g + (size_t)j * A;
+      const float qsel = gr[a];
+      const float* tr = qt + (size_t)j * A;
+      float qmax = tr[0];
+      for (int i = 1; i < A; ++i) qmax = fmaxf(qmax, tr[i]);
+      const float y = p.rew[j] + p.gamma * (p.done[j] ? 0.f : 1.f) * qmax;
+      const float delta = y - qsel, ad = fabsf(delta);
+      h = ad <= p.kappa ? 0.5f * delta * delta : p.kappa * (ad - 0.5f * p.kappa);
+      const float gj = -fminf(fmaxf(delta, -p.kappa), p.kappa) / (float)p.n;
+      for (int i = 0; i < A; ++i) gr[i] = i == a ? gj : 0.f;
+    }
+    hub[r] = h;
+  }
+  __syncwarp();
+  if (r == 0) {
+    float s = 0.f;
+    for (int i = 0; i < SG_ROWS; ++i) s += hub[i];
+    p.partial[blockIdx.x] = s;
+  }
+}
+
 // On-policy forward (PPO): trunk, policy head and value head of the one network; per row the clipped surrogate, the value
 // loss and the entropy, and their gradients at the outputs: g[j][0..A) for the logits, g[j][A] for the value.
 // shared memory: xs [D][16] | a1 [H][16] | a2 [H][16] | qs [A + 1][16] | weight tile [256][33]
@@ -285,46 +422,79 @@ struct GradProducts {
   int n, n_tiles;
 };
 
+constexpr int GP_TILE = 64, GP_ROWS = 16;   // tile of a gradient product; minibatch rows staged per step
+
 // Every gradient product of one update in a single launch: thread block (tile, range) sums, over its range of minibatch
-// rows, one 32 x 32 tile of one product and writes it to P[range][off + m * N + n] -- a partial gradient laid out like the
+// rows, one 64 x 64 tile of one product and writes it to P[range][off + m * N + n] -- a partial gradient laid out like the
 // parameter blob itself, `count` floats per range.  No atomics: the apply kernel adds the ranges in order.
 __global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, const GradProducts gp, int count, int n_rows,
                                                                int rows_per_range) {
-  __shared__ float As[32][33], Bs[32][33];
+  __shared__ __align__(16) float As[GP_ROWS][GP_TILE + 4], Bs[GP_ROWS][GP_TILE + 4];
   int q = 0;
   while (q + 1 < gp.n && (int)blockIdx.x >= gp.g[q + 1].tile_begin) ++q;
   const GradProduct& d = gp.g[q];
   const int M = d.M, N = d.N, lda = d.lda, ldb = d.ldb;
   const float* __restrict__ Am = d.Am;
   const float* __restrict__ Bm = d.Bm;
-  const int tiles_n = (N + 31) / 32, t = blockIdx.x - d.tile_begin;
-  const int m0 = (t / tiles_n) * 32, n0 = (t % tiles_n) * 32;
+  const int tiles_n = (N + GP_TILE - 1) / GP_TILE, t = blockIdx.x - d.tile_begin;
+  const int m0 = (t / tiles_n) * GP_TILE, n0 = (t % tiles_n) * GP_TILE;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int j_begin = blockIdx.y * rows_per_range;
   const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
-  float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-  for (int j0 = j_begin; j0 < j_end; j0 += 32) {
-    for (int i = threadIdx.x; i < 32 * 32; i += 256) {
-      const int jj = i >> 5, c = i & 31, j = j0 + jj;
-      As[jj][c] = (j < j_end && m0 + c < M) ? Am[(size_t)j * lda + m0 + c] : 0.f;
-      Bs[jj][c] = (j < j_end && n0 + c < N) ? (Bm ? Bm[(size_t)j * ldb + n0 + c] : 1.f) : 0.f;
+  const bool vecA = (lda & 3) == 0 && (reinterpret_cast<uintptr_t>(Am) & 15) == 0;
+  const bool vecB = Bm && (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(Bm) & 15) == 0;
+  // four consecutive columns of row j (zero beyond the row range or the matrix): a 16-byte load where the row allows it
+  auto load_c4 = [](const float* base, int ld, int j, int j_end, int c, int C, bool vec) -> float4 {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (j < j_end && c < C) {
+      const float* src = base + (size_t)j * ld + c;
+      if (vec && c + 3 < C) {
+        v = *reinterpret_cast<const float4*>(src);
+      } else {
+        v.x = src[0];
+        if (c + 1 < C) v.y = src[1];
+        if (c + 2 < C) v.z = src[2];
+        if (c + 3 < C) v.w = src[3];
+      }
+    }
+    return v;
+  };
+  float acc[4][4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u)
+#pragma unroll
+    for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
+  for (int j0 = j_begin; j0 < j_end; j0 += GP_ROWS) {
+    {
+      const int jj = threadIdx.x >> 4, c = (threadIdx.x & 15) * 4, j = j0 + jj;
+      *reinterpret_cast<float4*>(&As[jj][c]) = load_c4(Am, lda, j, j_end, m0 + c, M, vecA);
+      float4 bvv;
+      if (Bm) {
+        bvv = load_c4(Bm, ldb, j, j_end, n0 + c, N, vecB);
+      } else {
+        const float one = j < j_end ? 1.f : 0.f;
+        bvv = make_float4(n0 + c < N ? one : 0.f, n0 + c + 1 < N ? one : 0.f, n0 + c + 2 < N ? one : 0.f, n0 + c + 3 < N ? one : 0.f);
+      }
+      *reinterpret_cast<float4*>(&Bs[jj][c]) = bvv;
     }
     __syncthreads();
-#pragma unroll 8
-    for (int jj = 0; jj < 32; ++jj) {
-      const float a0 = As[jj][ty], a1 = As[jj][ty + 16], b0 = Bs[jj][tx], b1 = Bs[jj][tx + 16];
-      acc[0][0] = fmaf(a0, b0, acc[0][0]);
-      acc[0][1] = fmaf(a0, b1, acc[0][1]);
-      acc[1][0] = fmaf(a1, b0, acc[1][0]);
-      acc[1][1] = fmaf(a1, b1, acc[1][1]);
+#pragma unroll
+    for (int jj = 0; jj < GP_ROWS; ++jj) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[jj][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[jj][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(av[u], bv[v], acc[u][v]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int u = 0; u < 2; ++u)
+  for (int u = 0; u < 4; ++u)
 #pragma unroll
-    for (int v = 0; v < 2; ++v) {
-      const int m = m0 + ty + 16 * u, n = n0 + tx + 16 * v;
+    for (int v = 0; v < 4; ++v) {
+      const int m = m0 + ty * 4 + u, n = n0 + tx * 4 + v;
       if (m < M && n < N) P[(size_t)blockIdx.y * count + d.off + (size_t)m * N + n] = acc[u][v];
     }
 }
@@ -372,14 +542,25 @@ bool sgd_supported(int D, int H, int A) {
 }
 
 namespace {
+// the tiled path pays off once a layer is a real matrix product; below that the fused per-16-rows kernels launch less
+bool use_tiled(const SgdParams& p) { return !p.value_head && p.H >= 128 && p.n >= 512; }
+
 // the backward pass and every parameter update: C -= lr * (gradient rows)^T (input rows), a bias with a column of ones
 cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
   const int D = p.D, H = p.H, A = p.A;
   const int grid = sgd_partial_count(p.n);
   const size_t smem_b = (size_t)H * SG_ROWS * sizeof(float);
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(sgd_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b)) != cudaSuccess) return e;
-  sgd_backward_kernel<<<grid, SG_THREADS, smem_b, s>>>(p);
+  if (use_tiled(p)) {
+    // dh2 = (g W3) where h2 > 0; dh1 = (dh2 W2) where h1 > 0
+    const float* W2t = p.theta + (size_t)H * D + H;
+    const float* W3t = W2t + (size_t)H * H + H;
+    sg_gemm<true, GM_MASK>(p.g, p.ldg, W3t, H, p.dh2, H, p.n, H, A, nullptr, p.h2, H, s);
+    sg_gemm<true, GM_MASK>(p.dh2, H, W2t, H, p.dh1, H, p.n, H, H, nullptr, p.h1, H, s);
+  } else {
+    if ((e = cudaFuncSetAttribute(sgd_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b)) != cudaSuccess) return e;
+    sgd_backward_kernel<<<grid, SG_THREADS, smem_b, s>>>(p);
+  }
   float* W1 = p.theta;
   float* b1 = W1 + (size_t)H * D;
   float* W2 = b1 + H;
@@ -405,7 +586,7 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     d.lda = lda;
     d.ldb = ldb;
     d.tile_begin = gp.n_tiles;
-    gp.n_tiles += ((M + 31) / 32) * ((N + 31) / 32);
+    gp.n_tiles += ((M + GP_TILE - 1) / GP_TILE) * ((N + GP_TILE - 1) / GP_TILE);
   };
   add(W1, H, D, p.dh1, H, p.obs, D);
   add(b1, H, 1, p.dh1, H, nullptr, 0);
@@ -429,6 +610,22 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
 }  // namespace
 
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
+  if (use_tiled(p)) {
+    const int n = p.n, D = p.D, H = p.H, A = p.A;
+    const float *W1 = p.theta, *b1 = W1 + (size_t)H * D, *W2 = b1 + H, *b2 = W2 + (size_t)H * H, *W3 = b2 + H, *b3 = W3 + (size_t)A * H;
+    const float *T1 = p.theta_target, *tb1 = T1 + (size_t)H * D, *T2 = tb1 + H, *tb2 = T2 + (size_t)H * H, *T3 = tb2 + H,
+                *tb3 = T3 + (size_t)A * H;
+    // online network: h1, h2 kept, Q values into g; target network: its activations borrow dh1 / dh2 (free until the
+    // backward pass), its Q values then take dh1's place
+    sg_gemm<false, GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+    sgd_loss_kernel<<<sgd_partial_count(n), 32, 0, s>>>(p, p.dh1);
+    return backward_and_update(p, lr, adam, s);
+  }
   const size_t smem_f = (((size_t)p.D + 2 * (size_t)p.H + p.A) * SG_ROWS + (size_t)SG_THREADS * (SG_KT + 1)) * sizeof(float);
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(sgd_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f)) != cudaSuccess) return e;

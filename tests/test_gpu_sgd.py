@@ -34,8 +34,11 @@ def _groups(D, H, A):
     return [(names[i], int(offs[i]), int(offs[i + 1])) for i in range(6)]
 
 
+# the last four run the tiled matrix-product kernels (hidden >= 128 and >= 512 rows): hidden and row counts that are not
+# multiples of the 64 x 128 tile, an obs_dim that rules out 16-byte loads, an action count above one k-step's quarter
 @pytest.mark.parametrize("kind,D,A,H,N,B", [(0, 4, 2, 64, 64, 256), (1, 6, 3, 96, 50, 333), (2, 16, 5, 200, 40, 77), (2, 48, 4, 32, 40, 100),
-                                            (0, 4, 2, 256, 128, 1024)])
+                                            (0, 4, 2, 256, 128, 1024), (2, 16, 5, 200, 64, 600), (1, 6, 3, 136, 64, 700),
+                                            (2, 20, 9, 130, 64, 513)])
 def test_sgd_step_matches_oracle(env, kind, D, A, H, N, B):
     _check_sgd_step(env, kind, D, A, H, N, B, 0)
 
