@@ -136,23 +136,25 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
 // Wide networks and large minibatches: the layers as tiled FP32 matrix products (a weight element is reused for 128 rows
 // instead of 16).  C[m][n] = epi(sum_k A[m][k] Bop[k][n]): A row-major M x K.  B_KN false: B is N x K row-major (a weight
 // matrix as the forward pass uses it, Bop = B^T); true: B is K x N row-major (the same matrix in the backward pass).
-// 128 x 64 tile per block, 16 k per step, each thread 8 x 4; k ascending, one accumulator per output: a fixed order.
+// 128 x 64 tile per block (32 x 64 for the heads, whose few outputs would leave most SMs idle with tall tiles), 16 k per
+// step, each thread 8 x 4 (2 x 4); k ascending, one accumulator per output: a fixed order.
 constexpr int GM_BM = 128, GM_BN = 64, GM_BK = 16, GM_THREADS = 256;
 enum { GM_BIAS_RELU = 0, GM_BIAS = 1, GM_MASK = 2 };   // relu(acc + bias[n]) | acc + bias[n] | acc where mask[m][n] > 0, else 0
 
-template <bool B_KN, int EPI>
+template <bool B_KN, int EPI, int BM>
 __global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
                                                              float* __restrict__ C, int ldc, int M, int N, int K,
                                                              const float* __restrict__ bias, const float* __restrict__ mask, int ldm) {
-  __shared__ __align__(16) float As[GM_BK][GM_BM + 4];
+  __shared__ __align__(16) float As[GM_BK][BM + 4];
   __shared__ __align__(16) float Bs[GM_BK][GM_BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int m0 = blockIdx.y * GM_BM, n0 = blockIdx.x * GM_BN;
+  constexpr int RM = BM / 16;   // rows per thread
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * GM_BN;
   const bool vecA = (lda & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0;
   const bool vecB = (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0;
-  float acc[8][4];
+  float acc[RM][4];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < RM; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
   // four consecutive k of one row (of A, or of an N x K B): a 16-byte load where the row allows it
@@ -171,51 +173,73 @@ __global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __rest
     }
     return v;
   };
-  for (int k0 = 0; k0 < K; k0 += GM_BK) {
+  // the next k-step's operands travel from global memory to registers while this one is multiplied
+  constexpr int NA = (BM * 4 + GM_THREADS - 1) / GM_THREADS;
+  float4 ra[NA], rb;
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int i = tid; i < GM_BM * 4; i += GM_THREADS) {
-      const int r = i >> 2, kq = (i & 3) * 4;
-      const float4 v = load_k4(A, lda, m0 + r, M, k0 + kq, K, vecA);
-      As[kq][r] = v.x; As[kq + 1][r] = v.y; As[kq + 2][r] = v.z; As[kq + 3][r] = v.w;
+    for (int u = 0; u < NA; ++u) {
+      const int i = tid + u * GM_THREADS;
+      if (i < BM * 4) ra[u] = load_k4(A, lda, m0 + (i >> 2), M, k0 + (i & 3) * 4, K, vecA);
     }
     if (!B_KN) {
-      const int r = tid >> 2, kq = (tid & 3) * 4;
-      const float4 v = load_k4(B, ldb, n0 + r, N, k0 + kq, K, vecB);
-      Bs[kq][r] = v.x; Bs[kq + 1][r] = v.y; Bs[kq + 2][r] = v.z; Bs[kq + 3][r] = v.w;
+      rb = load_k4(B, ldb, n0 + (tid >> 2), N, k0 + (tid & 3) * 4, K, vecB);
     } else {
-      const int kk = tid >> 4, nq = (tid & 15) * 4, k = k0 + kk, n = n0 + nq;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int k = k0 + (tid >> 4), n = n0 + (tid & 15) * 4;
+      rb = make_float4(0.f, 0.f, 0.f, 0.f);
       if (k < K && n < N) {
         const float* src = B + (size_t)k * ldb + n;
         if (vecB && n + 3 < N) {
-          v = __ldg(reinterpret_cast<const float4*>(src));
+          rb = __ldg(reinterpret_cast<const float4*>(src));
         } else {
-          v.x = __ldg(src);
-          if (n + 1 < N) v.y = __ldg(src + 1);
-          if (n + 2 < N) v.z = __ldg(src + 2);
-          if (n + 3 < N) v.w = __ldg(src + 3);
+          rb.x = __ldg(src);
+          if (n + 1 < N) rb.y = __ldg(src + 1);
+          if (n + 2 < N) rb.z = __ldg(src + 2);
+          if (n + 3 < N) rb.w = __ldg(src + 3);
         }
       }
-      *reinterpret_cast<float4*>(&Bs[kk][nq]) = v;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < K; k0 += GM_BK) {
+#pragma unroll
+    for (int u = 0; u < NA; ++u) {
+      const int i = tid + u * GM_THREADS, r = i >> 2, kq = (i & 3) * 4;
+      if (i >= BM * 4) break;
+      As[kq][r] = ra[u].x; As[kq + 1][r] = ra[u].y; As[kq + 2][r] = ra[u].z; As[kq + 3][r] = ra[u].w;
+    }
+    if (!B_KN) {
+      const int r = tid >> 2, kq = (tid & 3) * 4;
+      Bs[kq][r] = rb.x; Bs[kq + 1][r] = rb.y; Bs[kq + 2][r] = rb.z; Bs[kq + 3][r] = rb.w;
+    } else {
+      *reinterpret_cast<float4*>(&Bs[tid >> 4][(tid & 15) * 4]) = rb;
     }
     __syncthreads();
+    if (k0 + GM_BK < K) fetch(k0 + GM_BK);
 #pragma unroll
     for (int kk = 0; kk < GM_BK; ++kk) {
-      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
-      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][ty * 8 + 4]);
+      float av[RM];
+      if constexpr (RM == 8) {
+        const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
+        const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][ty * 8 + 4]);
+        av[0] = a0.x; av[1] = a0.y; av[2] = a0.z; av[3] = a0.w;
+        av[RM - 4] = a1.x; av[RM - 3] = a1.y; av[RM - 2] = a1.z; av[RM - 1] = a1.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < RM; ++i) av[i] = As[kk][ty * RM + i];
+      }
       const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
       const float bv[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < RM; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int m = m0 + ty * 8 + i;
+  for (int i = 0; i < RM; ++i) {
+    const int m = m0 + ty * RM + i;
     if (m >= M) break;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -230,10 +254,10 @@ __global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __rest
   }
 }
 
-template <bool B_KN, int EPI>
+template <bool B_KN, int EPI, int BM = GM_BM>
 void sg_gemm(const float* A, int lda, const float* B, int ldb, float* C, int ldc, int M, int N, int K, const float* bias,
              const float* mask, int ldm, cudaStream_t s) {
-  sg_gemm_kernel<B_KN, EPI><<<dim3((N + GM_BN - 1) / GM_BN, (M + GM_BM - 1) / GM_BM), GM_THREADS, 0, s>>>(A, lda, B, ldb, C, ldc, M, N, K,
+  sg_gemm_kernel<B_KN, EPI, BM><<<dim3((N + GM_BN - 1) / GM_BN, (M + BM - 1) / BM), GM_THREADS, 0, s>>>(A, lda, B, ldb, C, ldc, M, N, K,
                                                                                                      bias, mask, ldm);
 }
 
@@ -619,10 +643,10 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
     // backward pass), its Q values then take dh1's place
     sg_gemm<false, GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, s);
     sg_gemm<false, GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, s);
-    sg_gemm<false, GM_BIAS>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
     sg_gemm<false, GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, s);
     sg_gemm<false, GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, s);
-    sg_gemm<false, GM_BIAS>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+    sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
     sgd_loss_kernel<<<sgd_partial_count(n), 32, 0, s>>>(p, p.dh1);
     return backward_and_update(p, lr, adam, s);
   }
