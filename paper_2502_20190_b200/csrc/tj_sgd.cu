@@ -488,20 +488,25 @@ __global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict
   for (int u = 0; u < 4; ++u)
 #pragma unroll
     for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
-  for (int j0 = j_begin; j0 < j_end; j0 += GP_ROWS) {
-    {
-      const int jj = threadIdx.x >> 4, c = (threadIdx.x & 15) * 4, j = j0 + jj;
-      *reinterpret_cast<float4*>(&As[jj][c]) = load_c4(Am, lda, j, j_end, m0 + c, M, vecA);
-      float4 bvv;
-      if (Bm) {
-        bvv = load_c4(Bm, ldb, j, j_end, n0 + c, N, vecB);
-      } else {
-        const float one = j < j_end ? 1.f : 0.f;
-        bvv = make_float4(n0 + c < N ? one : 0.f, n0 + c + 1 < N ? one : 0.f, n0 + c + 2 < N ? one : 0.f, n0 + c + 3 < N ? one : 0.f);
-      }
-      *reinterpret_cast<float4*>(&Bs[jj][c]) = bvv;
+  // the next rows travel from global memory to registers while these are multiplied
+  const int l_jj = threadIdx.x >> 4, l_c = (threadIdx.x & 15) * 4;
+  float4 ra, rb;
+  auto fetch = [&](int j0) {
+    const int j = j0 + l_jj;
+    ra = load_c4(Am, lda, j, j_end, m0 + l_c, M, vecA);
+    if (Bm) {
+      rb = load_c4(Bm, ldb, j, j_end, n0 + l_c, N, vecB);
+    } else {
+      const float one = j < j_end ? 1.f : 0.f;
+      rb = make_float4(n0 + l_c < N ? one : 0.f, n0 + l_c + 1 < N ? one : 0.f, n0 + l_c + 2 < N ? one : 0.f, n0 + l_c + 3 < N ? one : 0.f);
     }
+  };
+  if (j_begin < j_end) fetch(j_begin);
+  for (int j0 = j_begin; j0 < j_end; j0 += GP_ROWS) {
+    *reinterpret_cast<float4*>(&As[l_jj][l_c]) = ra;
+    *reinterpret_cast<float4*>(&Bs[l_jj][l_c]) = rb;
     __syncthreads();
+    if (j0 + GP_ROWS < j_end) fetch(j0 + GP_ROWS);
 #pragma unroll
     for (int jj = 0; jj < GP_ROWS; ++jj) {
       const float4 a = *reinterpret_cast<const float4*>(&As[jj][ty * 4]);
