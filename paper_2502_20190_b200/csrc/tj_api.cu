@@ -574,6 +574,7 @@ int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const f
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
   lay_out_update_scratch(x, p);
   p.ldg = x->A; p.value_head = 0;
+  p.error = &x->dstats->error;
   LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 15 : 14);
   cudaError_t e = launch_sgd_step(p, lr, adam, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
@@ -623,6 +624,7 @@ int tj_ppo_step(tj_ctx* x, const tj_ppo_batch* b, float lr, float beta1, float b
   p.clip_eps = clip_eps; p.c_v = c_v; p.c_e = c_e;
   lay_out_update_scratch(x, p);
   p.ldg = x->A + 1; p.value_head = 1;
+  p.error = &x->dstats->error;
   tj::AdamParams a{};
   a.m = m; a.v = v; a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
   a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));

@@ -115,6 +115,7 @@ struct SgdParams {
   const float* ret;
   float clip_eps, c_v, c_e;
   float* stat_partial;         // scratch: five partial sums per 16 rows (loss, policy, value, entropy, clipped rows)
+  unsigned long long* error;   // device error word of the context (a bounded wait that ran out)
 };
 
 struct AdamParams {

@@ -7,6 +7,7 @@
 //   update    W3[a] -= lr sum_j g_j h2_j, W2 -= lr dh2^T h1, W1 -= lr dh1^T x, biases likewise
 // Every sum runs in a fixed order (rows ascending), so a step is reproducible bit for bit.
 #include "tj_internal.h"
+#include "tj_tc.cuh"
 
 namespace tj {
 
@@ -259,6 +260,187 @@ void sg_gemm(const float* A, int lda, const float* B, int ldb, float* C, int ldc
              const float* mask, int ldm, cudaStream_t s) {
   sg_gemm_kernel<B_KN, EPI, BM><<<dim3((N + GM_BN - 1) / GM_BN, (M + BM - 1) / BM), GM_THREADS, 0, s>>>(A, lda, B, ldb, C, ldc, M, N, K,
                                                                                                      bias, mask, ldm);
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// The same product on the tensor cores, FP32-faithful: every operand is split into a TF32 high part (the top 19 bits) and
+// the remainder, and C accumulates A_hi B_hi + A_lo B_hi + A_hi B_lo in FP32 (the dropped A_lo B_lo term is 2^-22 of the
+// product).  A: M x K row-major, B: N x K row-major (a weight matrix as the forward pass uses it), K a multiple of 4, rows
+// 16-byte aligned.  One 128 x 128 tile per block, accumulator in tensor memory (128 columns); per step of 16 k the
+// threads split the step's operands into one of two shared-memory stages (K-major core matrices of 8 rows x 16 bytes)
+// while the tensor core works on the other, and the step after that is already on its way from global memory.  65 KB of
+// shared memory: two blocks per SM cover each other's waits.
+constexpr int TG_M = 128, TG_N = 128, TG_K = 16, TG_THREADS = 256, TG_PF = 3;
+constexpr int TG_OPER_BYTES = TG_M * TG_K * 4;            // one operand part of one stage: 8 KB
+constexpr int TG_STAGE_BYTES = 4 * TG_OPER_BYTES;         // A_hi | A_lo | B_hi | B_lo
+constexpr int TG_SMEM_BYTES = 2 * TG_STAGE_BYTES + 1024;  // + alignment slack
+
+template <int EPI>
+__global__ void __launch_bounds__(TG_THREADS, 2) sg_gemm_tc_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B,
+                                                                   int ldb, float* __restrict__ C, int ldc, int M, int N, int K,
+                                                                   const float* __restrict__ bias, const float* __restrict__ mask,
+                                                                   int ldm, unsigned long long* __restrict__ error) {
+  extern __shared__ uint8_t tg_raw[];
+  uint8_t* stage0 = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tg_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) uint64_t done[2];
+  __shared__ uint32_t tmem_base;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.y * TG_M, n0 = blockIdx.x * TG_N;
+  if (tid == 0) {
+    mbar_init(&done[0], 1);
+    mbar_init(&done[1], 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base)), "r"(128u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base;
+
+  // loader mapping: a warp instruction covers eight rows x four 16-byte pieces (64 contiguous bytes per row); warp w
+  // owns rows 16 w .. 16 w + 15 of both operands' tiles, a thread two pieces of each
+  static_assert(TG_K == 16, "the loader maps four 16-byte pieces to a row");
+  const int r8 = lane >> 2, kq = lane & 3;
+  // TG_PF register sets: the operands of the next TG_PF steps are in flight from global memory at any time
+  float4 ra[TG_PF][2], rb[TG_PF][2];
+  auto fetch = [&](int k0, float4 (&fa)[2], float4 (&fb)[2]) {
+    const int k = k0 + kq * 4;
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      const int rr = warp * 16 + g * 8 + r8;
+      fa[g] = (m0 + rr < M && k < K) ? __ldg(reinterpret_cast<const float4*>(A + (size_t)(m0 + rr) * lda + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      fb[g] = (n0 + rr < N && k < K) ? __ldg(reinterpret_cast<const float4*>(B + (size_t)(n0 + rr) * ldb + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto split_store = [](uint8_t* hi_dst, uint8_t* lo_dst, const float4 v) {
+    float4 hi, lo;
+    hi.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); lo.x = v.x - hi.x;
+    hi.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); lo.y = v.y - hi.y;
+    hi.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); lo.z = v.z - hi.z;
+    hi.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); lo.w = v.w - hi.w;
+    *reinterpret_cast<float4*>(hi_dst) = hi;
+    *reinterpret_cast<float4*>(lo_dst) = lo;
+  };
+  const int nk = (K + TG_K - 1) / TG_K;
+  const uint32_t idesc = make_idesc_tf32(TG_N);
+  constexpr uint32_t SBO = (TG_K / 4) * 128u;     // eight rows further: one row group of K/4 core matrices
+  bool ok = true;
+  // one step: registers -> split -> stage i & 1, the tensor core's products on it, the load of step i + TG_PF.  Returns
+  // false (for every thread alike) when a wait ran out.
+  auto step = [&](int i, float4 (&fa)[2], float4 (&fb)[2]) -> bool {
+    const int s = i & 1;
+    uint8_t* st = stage0 + (size_t)s * TG_STAGE_BYTES;
+    // the tensor core must be done with this stage (its use two steps ago).  One warp polls the barrier, the others
+    // sleep at the block barrier: polls from every warp would take shared-memory cycles from the tensor core, whose
+    // TF32 operand reads (8 KB per instruction) already need most of them
+    if (i >= 2) {
+      if (warp == 1) ok = tc_wait_elect(&done[s], (uint32_t)(((i >> 1) - 1) & 1), &abort_flag);
+      if (__syncthreads_or(!ok)) return false;
+    }
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      const int rr = warp * 16 + g * 8 + r8;
+      const size_t off = (size_t)(rr >> 3) * SBO + (size_t)(rr & 7) * 16 + (size_t)kq * 128;
+      split_store(st + off, st + TG_OPER_BYTES + off, fa[g]);
+      split_store(st + 2 * TG_OPER_BYTES + off, st + 3 * TG_OPER_BYTES + off, fb[g]);
+    }
+    fence_async_smem();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t a_hi = smem_addr(st), a_lo = a_hi + TG_OPER_BYTES, b_hi = a_hi + 2 * TG_OPER_BYTES, b_lo = a_hi + 3 * TG_OPER_BYTES;
+#pragma unroll
+      for (int j = 0; j < TG_K / 8; ++j) {
+        const uint32_t o = (uint32_t)j * 256u;
+        umma_tf32(tmem, make_desc(a_hi + o, 128u, SBO), make_desc(b_hi + o, 128u, SBO), idesc, (i | j) != 0);
+        umma_tf32(tmem, make_desc(a_lo + o, 128u, SBO), make_desc(b_hi + o, 128u, SBO), idesc, true);
+        umma_tf32(tmem, make_desc(a_hi + o, 128u, SBO), make_desc(b_lo + o, 128u, SBO), idesc, true);
+      }
+      umma_commit(&done[s]);
+    }
+    if (i + TG_PF < nk) fetch((i + TG_PF) * TG_K, fa, fb);
+    return true;
+  };
+#pragma unroll
+  for (int pf = 0; pf < TG_PF; ++pf)
+    if (pf < nk) fetch(pf * TG_K, ra[pf], rb[pf]);
+  bool running = true;
+  for (int i = 0; i < nk && running; i += TG_PF) {
+#pragma unroll
+    for (int pf = 0; pf < TG_PF; ++pf)
+      if (running && i + pf < nk) running = step(i + pf, ra[pf], rb[pf]);
+  }
+  // every product is complete once the last commit has arrived (a commit covers all earlier ones of its thread)
+  if (running && warp == 1) ok = tc_wait_elect(&done[(nk - 1) & 1], (uint32_t)(((nk - 1) >> 1) & 1), &abort_flag);
+  ok = !__syncthreads_or(!ok || !running);
+  if (ok) {
+    tc_fence_after();
+    const int q = warp & 3, hsel = warp >> 2;      // TMEM lane quarter of this warp, column half
+    const int m = m0 + q * 32 + lane;
+    const uint32_t t_acc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(hsel * 64);
+    uint32_t v[64];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) tmem_ld16(t_acc + (uint32_t)(g * 16), v + 16 * g);
+    tmem_ld_wait();
+    if (m < M) {
+      const bool vec = (ldc & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0;
+#pragma unroll
+      for (int c4 = 0; c4 < 16; ++c4) {
+        const int n = n0 + hsel * 64 + c4 * 4;
+        if (n >= N) break;
+        float o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float x = __uint_as_float(v[c4 * 4 + j]);
+          if (n + j < N) {
+            if (EPI == GM_BIAS_RELU) x = fmaxf(x + __ldg(bias + n + j), 0.f);
+            else if (EPI == GM_BIAS) x = x + __ldg(bias + n + j);
+            else x = __ldg(mask + (size_t)m * ldm + n + j) > 0.f ? x : 0.f;
+          }
+          o[j] = x;
+        }
+        float* dst = C + (size_t)m * ldc + n;
+        if (vec && n + 3 < N) {
+          *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (n + j < N) dst[j] = o[j];
+        }
+      }
+    }
+  } else if (tid == 0) {
+    atomicExch(error, 3ull);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128u) : "memory");
+}
+
+// shapes the tensor-core product takes: 16-byte rows on both operands and enough work to fill 128 x 128 tiles
+static bool tc_gemm_ok(const float* A, int lda, const float* B, int ldb, int M, int N, int K) {
+  return (K & 3) == 0 && (lda & 3) == 0 && (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0 &&
+         (reinterpret_cast<uintptr_t>(B) & 15) == 0 && K >= 32 && N >= 64 && M >= 512;
+}
+
+// forward-layout product (B is N x K): tensor cores where the shape allows, the FMA tiles otherwise
+template <int EPI>
+cudaError_t sg_layer(const float* A, int lda, const float* B, int ldb, float* C, int ldc, int M, int N, int K, const float* bias,
+                     const float* mask, int ldm, unsigned long long* error, cudaStream_t s) {
+  if (tc_gemm_ok(A, lda, B, ldb, M, N, K)) {
+    cudaError_t e = cudaFuncSetAttribute(sg_gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    sg_gemm_tc_kernel<EPI><<<dim3((N + TG_N - 1) / TG_N, (M + TG_M - 1) / TG_M), TG_THREADS, TG_SMEM_BYTES, s>>>(A, lda, B, ldb, C, ldc, M, N, K,
+                                                                                                         bias, mask, ldm, error);
+  } else {
+    sg_gemm<false, EPI>(A, lda, B, ldb, C, ldc, M, N, K, bias, mask, ldm, s);
+  }
+  return cudaGetLastError();
 }
 
 // TD error, Huber loss and its gradient at the outputs from the two networks' Q values: q (in) and g (out) share p.g
@@ -646,11 +828,12 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
                 *tb3 = T3 + (size_t)A * H;
     // online network: h1, h2 kept, Q values into g; target network: its activations borrow dh1 / dh2 (free until the
     // backward pass), its Q values then take dh1's place
-    sg_gemm<false, GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, s);
-    sg_gemm<false, GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, s);
+    cudaError_t e;
+    if ((e = sg_layer<GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+    if ((e = sg_layer<GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
     sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
-    sg_gemm<false, GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, s);
-    sg_gemm<false, GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, s);
+    if ((e = sg_layer<GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+    if ((e = sg_layer<GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
     sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
     sgd_loss_kernel<<<sgd_partial_count(n), 32, 0, s>>>(p, p.dh1);
     return backward_and_update(p, lr, adam, s);
