@@ -233,7 +233,9 @@ int tj_td_error_static(tj_ctx *ctx, const tj_batch *batch, float *td_out, float 
  * With huber_delta = inf, one row and theta_target = theta this is Algorithm 1's update line.
  * theta (in/out) and theta_target: device FP32 blobs in the tj_publish_weights layout, distinct buffers, owned by the
  * caller; nothing in the context changes -- publish theta afterwards to hand it to the actor.  batch.n <= the configured
- * minibatch.  loss_mean_out (nullable, device): the loss before the update.  FP32 arithmetic, every sum in a fixed order.
+ * minibatch.  loss_mean_out (nullable, device): the loss before the update.  FP32 arithmetic, every sum in a fixed order;
+ * hidden-layer products with at least 96 tiles of 128 x 128 outputs (e.g. 8,192 rows x 512 units) run on the tensor cores
+ * as three TF32 products of high / low operand parts with FP32 accumulation: up to 3 * 2^-22 per product instead of 2^-24.
  * In a BF16 context theta is the FP32 master copy: the update and its loss are FP32 all the same, the rounding to BF16
  * happens at tj_publish_weights (so this loss differs from tj_td_error's, which uses the published BF16 copy, by that
  * rounding).  TJ_ERR_UNSUPPORTED for segment mode and the categorical policy. */

@@ -548,14 +548,16 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
 }
 
 namespace {
-// h1, h2, dh1, dh2 [rows][H] | g [rows][17] | loss partials | PPO statistic partials | gradient partial sums
+// h1, h2, dh1, dh2 [rows][H] | g [rows][17] | loss partials | PPO statistic partials | W2^T [H][H] | gradient partial sums
 void lay_out_update_scratch(const tj_ctx* x, tj::SgdParams& p) {
   const size_t rows = ((size_t)x->sgd_rows + 15) / 16 * 16, RH = rows * (size_t)x->H;
   p.h1 = x->sgd_scratch; p.h2 = p.h1 + RH; p.dh1 = p.h2 + RH; p.dh2 = p.dh1 + RH;
   p.g = p.dh2 + RH;
   p.partial = p.g + rows * 17;
   p.stat_partial = p.partial + rows / 16 + 8;
-  p.grad_partial = p.stat_partial + 5 * (rows / 16) + 8;
+  p.w2t = p.stat_partial + 5 * (rows / 16) + 8;
+  p.w2t += (4 - ((reinterpret_cast<uintptr_t>(p.w2t) / sizeof(float)) & 3)) & 3;   // 16-byte rows for the vector loads
+  p.grad_partial = p.w2t + (size_t)x->H * x->H;
 }
 
 int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, const tj::AdamParams* adam,

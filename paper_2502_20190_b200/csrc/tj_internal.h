@@ -107,6 +107,7 @@ struct SgdParams {
   float* g;                    // scratch [n][A]: dL/dq, non-zero at the selected action only
   float* partial;              // scratch: one Huber partial sum per 16 rows
   float* grad_partial;         // scratch: per row range one partial gradient laid out like the parameter blob
+  float* w2t;                  // scratch [H][H]: W2 transposed, the backward pass's operand on the tensor-core path
   int ldg;                     // row stride of g (A for the Q head, A + 1 with the value head's entry in column A)
   int value_head;              // 1: policy + value heads (PPO), theta carries Wv, bv after b3
   // PPO only

@@ -422,10 +422,23 @@ __global__ void __launch_bounds__(TG_THREADS, 2) sg_gemm_tc_kernel(const float* 
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128u) : "memory");
 }
 
-// shapes the tensor-core product takes: 16-byte rows on both operands and enough work to fill 128 x 128 tiles
+// dst[c][r] = src[r][c] for an n x n matrix (32 x 32 tiles through shared memory, both sides coalesced)
+__global__ void __launch_bounds__(256) sg_transpose_kernel(const float* __restrict__ src, float* __restrict__ dst, int n) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32, tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8)
+    if (r0 + i < n && c0 + tx < n) tile[i][tx] = src[(size_t)(r0 + i) * n + c0 + tx];
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8)
+    if (c0 + i < n && r0 + tx < n) dst[(size_t)(c0 + i) * n + r0 + tx] = tile[tx][i];
+}
+
+// shapes the tensor-core product takes: 16-byte rows on both operands and enough 128 x 128 tiles to occupy most SMs (with
+// fewer, the 128 x 64 FMA tiles spread the work over more blocks and finish sooner)
 static bool tc_gemm_ok(const float* A, int lda, const float* B, int ldb, int M, int N, int K) {
+  const long long tiles = (long long)((M + TG_M - 1) / TG_M) * ((N + TG_N - 1) / TG_N);
   return (K & 3) == 0 && (lda & 3) == 0 && (ldb & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0 &&
-         (reinterpret_cast<uintptr_t>(B) & 15) == 0 && K >= 32 && N >= 64 && M >= 512;
+         (reinterpret_cast<uintptr_t>(B) & 15) == 0 && K >= 32 && tiles >= 96;
 }
 
 // forward-layout product (B is N x K): tensor cores where the shape allows, the FMA tiles otherwise
@@ -740,9 +753,9 @@ __global__ void sgd_apply_adam_kernel(float* __restrict__ Cm, float* __restrict_
 size_t sgd_scratch_floats(int max_rows, int D, int H) {
   const size_t rows = ((size_t)max_rows + SG_ROWS - 1) / SG_ROWS * SG_ROWS;
   // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), and per row range one partial
-  // gradient of the whole parameter blob (at most 16 actions and a value head)
+  // gradient of the whole parameter blob (at most 16 actions and a value head); W2 transposed
   const size_t blob = (size_t)H * D + H + (size_t)H * H + H + 17 * (size_t)H + 17;
-  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)SG_SPLITS * blob;
+  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)H * H + (size_t)SG_SPLITS * blob;
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }
@@ -764,10 +777,16 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
   cudaError_t e;
   if (use_tiled(p)) {
     // dh2 = (g W3) where h2 > 0; dh1 = (dh2 W2) where h1 > 0
-    const float* W2t = p.theta + (size_t)H * D + H;
-    const float* W3t = W2t + (size_t)H * H + H;
-    sg_gemm<true, GM_MASK>(p.g, p.ldg, W3t, H, p.dh2, H, p.n, H, A, nullptr, p.h2, H, s);
-    sg_gemm<true, GM_MASK>(p.dh2, H, W2t, H, p.dh1, H, p.n, H, H, nullptr, p.h1, H, s);
+    const float* W2m = p.theta + (size_t)H * D + H;
+    const float* W3m = W2m + (size_t)H * H + H;
+    sg_gemm<true, GM_MASK>(p.g, p.ldg, W3m, H, p.dh2, H, p.n, H, A, nullptr, p.h2, H, s);
+    if (tc_gemm_ok(p.dh2, H, p.w2t, H, p.n, H, H)) {
+      // the tensor-core product wants both operands K-major: dh1 = dh2 (W2^T)^T with W2^T written out first
+      sg_transpose_kernel<<<dim3((H + 31) / 32, (H + 31) / 32), 256, 0, s>>>(W2m, p.w2t, H);
+      if ((e = sg_layer<GM_MASK>(p.dh2, H, p.w2t, H, p.dh1, H, p.n, H, H, nullptr, p.h1, H, p.error, s)) != cudaSuccess) return e;
+    } else {
+      sg_gemm<true, GM_MASK>(p.dh2, H, W2m, H, p.dh1, H, p.n, H, H, nullptr, p.h1, H, s);
+    }
   } else {
     if ((e = cudaFuncSetAttribute(sgd_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_b)) != cudaSuccess) return e;
     sgd_backward_kernel<<<grid, SG_THREADS, smem_b, s>>>(p);

@@ -50,7 +50,19 @@ def test_sgd_step_in_a_bf16_context_updates_the_fp32_master_copy(env, kind, D, A
     _check_sgd_step(env, kind, D, A, H, N, B, 1)
 
 
-def _check_sgd_step(env, kind, D, A, H, N, B, weight_dtype):
+RTOL_TF32X3 = 1e-4
+
+
+def test_sgd_step_on_the_tensor_core_path_matches_oracle(env):
+    """25 x 4 tiles of 128 x 128 (3,100 rows, hidden 500: ragged both ways) are enough for the hidden layers and dh1 to run
+    as 3 x TF32 tensor-core products.  Their tolerance: an operand enters as a TF32 high part plus a remainder that the
+    tensor core again reads with 11 significant bits, so each product carries up to 2 * 2^-22 from the two truncated
+    remainders plus 2^-22 from the dropped low x low term, 3 * 2^-22 = 7e-7 against FP32's 2^-24 = 6e-8 per operation:
+    twelve times the FP32 tolerance, rounded down to 1e-4."""
+    _check_sgd_step(env, 2, 16, 5, 500, 512, 3100, 0, rtol=RTOL_TF32X3)
+
+
+def _check_sgd_step(env, kind, D, A, H, N, B, weight_dtype, rtol=RTOL_FP32):
     torch, orc, binding = env
     f = fields_for(env_kind=kind, n_envs=N, obs_dim=D, n_actions=A, hidden=H, epsilon=0.3, seed=777, replay_capacity=N * 16,
                    minibatch=B, staleness_bound=20, warmup=N, target_sync_interval=1000, gamma=0.99, huber_delta=1.0,
@@ -84,7 +96,7 @@ def _check_sgd_step(env, kind, D, A, H, N, B, weight_dtype):
         assert np.abs(do[a:b]).max() > 0, name                               # every group moves
         rms = np.sqrt(np.mean(do[a:b] ** 2))
         err = np.abs(dg[a:b] - do[a:b])
-        bound = RTOL_FP32 * np.abs(do[a:b]) + RTOL_FP32 * rms + ulp[a:b]
+        bound = rtol * np.abs(do[a:b]) + rtol * rms + ulp[a:b]
         assert np.all(err <= bound), "%s: worst %.3e over bound %.3e" % (name, err.max(), bound[np.argmax(err - bound)])
     # a second step from the updated parameters stays on the oracle's trajectory
     loss2 = ctx.sgd_step(batch, lr, th, tt)
