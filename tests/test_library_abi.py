@@ -35,7 +35,11 @@ def test_config_struct_matches_and_workspace_sizes(lib):
         C_, N, D = w["replay_capacity"], w["n_envs"], w["obs_dim"]
         if C_:
             assert nbytes >= C_ * (2 * D + 4) * 4
-            assert nbytes < C_ * (2 * D + 4) * 4 + N * max(D, 4) * 4 + 64 * 2**20
+            # beside the ring and the env state: the learner update's scratch (four activation / delta arrays of
+            # minibatch x hidden, 32 partial gradients of the parameter blob, W2 transposed) and 64 MiB for the rest
+            B, H = w["minibatch"], w["hidden"]
+            update = (4 * B * H + 32 * (H * (D + H + 19) + 17) + H * H + 24 * B) * 4
+            assert nbytes < C_ * (2 * D + 4) * 4 + N * max(D, 4) * 4 + update + 64 * 2**20
     # the largest workload's ring is 16M records of 1040 bytes
     assert nbytes > 17.4e9
 
