@@ -256,16 +256,26 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
   }
 }
 
-// fixed-order sum of the per-block partial losses: one warp fetches 32 partials at a time (one coalesced load instead of
-// 32 dependent ones), lane 0 adds them in index order -- the same sum, term by term, as a single thread walking the array
+// fixed-order sum of the per-block partial losses: one warp fetches 16 x 32 partials with independent coalesced loads
+// (a single thread walking the array pays one memory latency per element, a warp fetching one chunk per iteration one per
+// chunk), then lane 0 adds them in index order -- the same sum, term by term
 __global__ void td_finish_kernel(const float* __restrict__ partial, int n_partial, int n, float* __restrict__ loss_out) {
   if (blockIdx.x != 0 || threadIdx.x >= 32) return;
   const int lane = threadIdx.x;
   float sum = 0.f;
-  for (int i0 = 0; i0 < n_partial; i0 += 32) {
-    const float mine = i0 + lane < n_partial ? partial[i0 + lane] : 0.f;
-    const int cnt = n_partial - i0 < 32 ? n_partial - i0 : 32;
-    for (int l = 0; l < cnt; ++l) sum += __shfl_sync(0xffffffffu, mine, l);
+  for (int base = 0; base < n_partial; base += 16 * 32) {
+    float mine[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const int i = base + c * 32 + lane;
+      mine[c] = i < n_partial ? partial[i] : 0.f;
+    }
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const int left = n_partial - (base + c * 32);
+      const int cnt = left < 0 ? 0 : (left < 32 ? left : 32);
+      for (int l = 0; l < cnt; ++l) sum += __shfl_sync(0xffffffffu, mine[c], l);
+    }
   }
   if (lane == 0) *loss_out = sum / (float)n;
 }
