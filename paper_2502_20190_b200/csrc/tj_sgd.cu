@@ -641,22 +641,18 @@ struct GradProducts {
   int n, n_tiles;
 };
 
-constexpr int GP_TILE = 64, GP_ROWS = 16;   // tile of a gradient product; minibatch rows staged per step
+constexpr int GP_TILE = 64, GP_ROWS = 16;   // columns of a gradient tile; minibatch rows staged per step
 
-// Every gradient product of one update in a single launch: thread block (tile, range) sums, over its range of minibatch
-// rows, one 64 x 64 tile of one product and writes it to P[range][off + m * N + n] -- a partial gradient laid out like the
-// parameter blob itself, `count` floats per range.  No atomics: the apply kernel adds the ranges in order.
-__global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, const GradProducts gp, int count, int n_rows,
-                                                               int rows_per_range) {
-  __shared__ __align__(16) float As[GP_ROWS][GP_TILE + 4], Bs[GP_ROWS][GP_TILE + 4];
-  int q = 0;
-  while (q + 1 < gp.n && (int)blockIdx.x >= gp.g[q + 1].tile_begin) ++q;
-  const GradProduct& d = gp.g[q];
+// One tile (TM x 64, TM = 64 or 128: each thread TM / 16 x 4) of one gradient product over one range of minibatch rows
+template <int TM>
+__device__ __forceinline__ void grad_tile(float* __restrict__ P, const GradProduct& d, int t, int count, int n_rows, int rows_per_range,
+                                          float (*As)[128 + 4], float (*Bs)[GP_TILE + 4]) {
+  constexpr int RM = TM / 16, NA = TM / 64;
   const int M = d.M, N = d.N, lda = d.lda, ldb = d.ldb;
   const float* __restrict__ Am = d.Am;
   const float* __restrict__ Bm = d.Bm;
-  const int tiles_n = (N + GP_TILE - 1) / GP_TILE, t = blockIdx.x - d.tile_begin;
-  const int m0 = (t / tiles_n) * GP_TILE, n0 = (t % tiles_n) * GP_TILE;
+  const int tiles_n = (N + GP_TILE - 1) / GP_TILE;
+  const int m0 = (t / tiles_n) * TM, n0 = (t % tiles_n) * GP_TILE;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   const int j_begin = blockIdx.y * rows_per_range;
   const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
@@ -678,17 +674,18 @@ __global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict
     }
     return v;
   };
-  float acc[4][4];
+  float acc[RM][4];
 #pragma unroll
-  for (int u = 0; u < 4; ++u)
+  for (int u = 0; u < RM; ++u)
 #pragma unroll
     for (int v = 0; v < 4; ++v) acc[u][v] = 0.f;
   // the next rows travel from global memory to registers while these are multiplied
   const int l_jj = threadIdx.x >> 4, l_c = (threadIdx.x & 15) * 4;
-  float4 ra, rb;
+  float4 ra[NA], rb;
   auto fetch = [&](int j0) {
     const int j = j0 + l_jj;
-    ra = load_c4(Am, lda, j, j_end, m0 + l_c, M, vecA);
+#pragma unroll
+    for (int h = 0; h < NA; ++h) ra[h] = load_c4(Am, lda, j, j_end, m0 + h * 64 + l_c, M, vecA);
     if (Bm) {
       rb = load_c4(Bm, ldb, j, j_end, n0 + l_c, N, vecB);
     } else {
@@ -698,29 +695,50 @@ __global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict
   };
   if (j_begin < j_end) fetch(j_begin);
   for (int j0 = j_begin; j0 < j_end; j0 += GP_ROWS) {
-    *reinterpret_cast<float4*>(&As[l_jj][l_c]) = ra;
+#pragma unroll
+    for (int h = 0; h < NA; ++h) *reinterpret_cast<float4*>(&As[l_jj][h * 64 + l_c]) = ra[h];
     *reinterpret_cast<float4*>(&Bs[l_jj][l_c]) = rb;
     __syncthreads();
     if (j0 + GP_ROWS < j_end) fetch(j0 + GP_ROWS);
 #pragma unroll
     for (int jj = 0; jj < GP_ROWS; ++jj) {
-      const float4 a = *reinterpret_cast<const float4*>(&As[jj][ty * 4]);
-      const float4 b = *reinterpret_cast<const float4*>(&Bs[jj][tx * 4]);
-      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+      float av[RM];
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
+      for (int h = 0; h < RM / 4; ++h) {
+        const float4 a = *reinterpret_cast<const float4*>(&As[jj][ty * RM + h * 4]);
+        av[h * 4] = a.x; av[h * 4 + 1] = a.y; av[h * 4 + 2] = a.z; av[h * 4 + 3] = a.w;
+      }
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[jj][tx * 4]);
+      const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int u = 0; u < RM; ++u)
 #pragma unroll
         for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(av[u], bv[v], acc[u][v]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int u = 0; u < 4; ++u)
+  for (int u = 0; u < RM; ++u)
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
-      const int m = m0 + ty * 4 + u, n = n0 + tx * 4 + v;
+      const int m = m0 + ty * RM + u, n = n0 + tx * 4 + v;
       if (m < M && n < N) P[(size_t)blockIdx.y * count + d.off + (size_t)m * N + n] = acc[u][v];
     }
+}
+
+// Every gradient product of one update in a single launch: thread block (tile, range) sums, over its range of minibatch
+// rows, one tile of one product (128 x 64 where the product has at least 128 rows, else 64 x 64) and writes it to
+// P[range][off + m * N + n] -- a partial gradient laid out like the parameter blob itself, `count` floats per range.
+// No atomics: the apply kernel adds the ranges in order.
+__global__ void __launch_bounds__(256) sgd_grad_partial_kernel(float* __restrict__ P, const GradProducts gp, int count, int n_rows,
+                                                               int rows_per_range) {
+  __shared__ __align__(16) float As[GP_ROWS][128 + 4], Bs[GP_ROWS][GP_TILE + 4];
+  int q = 0;
+  while (q + 1 < gp.n && (int)blockIdx.x >= gp.g[q + 1].tile_begin) ++q;
+  const GradProduct& d = gp.g[q];
+  const int t = blockIdx.x - d.tile_begin;
+  if (d.M >= 128) grad_tile<128>(P, d, t, count, n_rows, rows_per_range, As, Bs);
+  else grad_tile<64>(P, d, t, count, n_rows, rows_per_range, As, Bs);
 }
 
 // C[i] -= lr * (P[0][i] + P[1][i] + ...), the partial sums added in range order
@@ -816,7 +834,8 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     d.lda = lda;
     d.ldb = ldb;
     d.tile_begin = gp.n_tiles;
-    gp.n_tiles += ((M + GP_TILE - 1) / GP_TILE) * ((N + GP_TILE - 1) / GP_TILE);
+    const int tm = M >= 128 ? 128 : 64;   // as the kernel picks it
+    gp.n_tiles += ((M + tm - 1) / tm) * ((N + GP_TILE - 1) / GP_TILE);
   };
   add(W1, H, D, p.dh1, H, p.obs, D);
   add(b1, H, 1, p.dh1, H, nullptr, 0);
