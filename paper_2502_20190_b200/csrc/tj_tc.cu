@@ -263,9 +263,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) mlp_bf16_tc_kernel(const TcMlpP
               uint32_t o[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                const float f0 = fmaxf(__uint_as_float(v[16 * hh + 2 * j]) + b[cc + 2 * j], 0.f);
-                const float f1 = fmaxf(__uint_as_float(v[16 * hh + 2 * j + 1]) + b[cc + 2 * j + 1], 0.f);
-                o[j] = pack_bf16x2(f0, f1);
+                const float f0 = __uint_as_float(v[16 * hh + 2 * j]) + b[cc + 2 * j];
+                const float f1 = __uint_as_float(v[16 * hh + 2 * j + 1]) + b[cc + 2 * j + 1];
+                o[j] = pack_bf16x2_relu(f0, f1);
               }
               *reinterpret_cast<uint4*>(dst + (size_t)(cc / 8) * 128) = make_uint4(o[0], o[1], o[2], o[3]);
               *reinterpret_cast<uint4*>(dst + (size_t)(cc / 8 + 1) * 128) = make_uint4(o[4], o[5], o[6], o[7]);

@@ -312,12 +312,12 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
             const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + c0 + hh * 32 + 4 * j4));
-            const float f0 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 0]) + bb.x, 0.f);
-            const float f1 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 1]) + bb.y, 0.f);
-            const float f2 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 2]) + bb.z, 0.f);
-            const float f3 = fmaxf(__uint_as_float(v[hh * 32 + 4 * j4 + 3]) + bb.w, 0.f);
-            o[2 * j4] = pack_bf16x2(f0, f1);
-            o[2 * j4 + 1] = pack_bf16x2(f2, f3);
+            const float f0 = __uint_as_float(v[hh * 32 + 4 * j4 + 0]) + bb.x;
+            const float f1 = __uint_as_float(v[hh * 32 + 4 * j4 + 1]) + bb.y;
+            const float f2 = __uint_as_float(v[hh * 32 + 4 * j4 + 2]) + bb.z;
+            const float f3 = __uint_as_float(v[hh * 32 + 4 * j4 + 3]) + bb.w;
+            o[2 * j4] = pack_bf16x2_relu(f0, f1);
+            o[2 * j4 + 1] = pack_bf16x2_relu(f2, f3);
           }
           if (layer == 0) {
             tmem_st16(t_lane + PA_COL_HB + (uint32_t)((c0 + hh * 32) / 2), o);
