@@ -29,7 +29,7 @@ from paper_2502_20190_b200 import synth  # noqa: E402
 
 SM_COUNT, FMA_LANES_PER_SM = 148, 128
 # dram__bytes (read + write) per env-step of the pipelined tensor-core actor launch, from one ncu capture of the kernel as
-# it stands (113,664 envs: 1.318 TB/s over 188.9 us = 249.0 MB per launch); traffic grows with the number of envs.  Set to
+# it stands (113,664 envs: 1.320 TB/s over 188.6 us = 249.0 MB per launch); traffic grows with the number of envs.  Set to
 # None when the kernel changes.  See profiles/cfg5_pipelined_tensor_core_actor.md.
 NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": 2190.7}
 L2_FLUSH_BYTES = 256 << 20
