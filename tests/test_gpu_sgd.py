@@ -229,4 +229,4 @@ def test_measured_rates_give_the_balanced_split():
     assert rates["consumed_per_s"] == pytest.approx(rates["P"] * rates["produced_per_s"])
     assert rates["kernel_s"] <= rates["loop_s"]
     assert rates["loop_produced_per_s"] <= rates["produced_per_s"] * 1.001
-    assert rates["loop_produced_per_s"] >= 0.1 * rates["produced_per_s"]       # host time between launches stays a minor part
+    assert rates["loop_produced_per_s"] >= 0.1 * rates["produced_per_s"]       # loose: first launches of a kernel are slow and 200 iterations are short
