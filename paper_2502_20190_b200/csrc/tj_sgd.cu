@@ -265,11 +265,11 @@ void sg_gemm(const float* A, int lda, const float* B, int ldb, float* C, int ldc
 // ---------------------------------------------------------------------------------------------------------------------
 // The same product on the tensor cores, FP32-faithful: every operand is split into a TF32 high part (the top 19 bits) and
 // the remainder, and C accumulates A_hi B_hi + A_lo B_hi + A_hi B_lo in FP32 (the dropped A_lo B_lo term is 2^-22 of the
-// product).  A: M x K row-major, B: N x K row-major (a weight matrix as the forward pass uses it), K a multiple of 4, rows
+// product, and the tensor core reads each remainder with 11 significant bits: another 2^-22 each).  A: M x K row-major, B: N x K row-major (a weight matrix as the forward pass uses it), K a multiple of 4, rows
 // 16-byte aligned.  One 128 x 128 tile per block, accumulator in tensor memory (128 columns); per step of 16 k the
 // threads split the step's operands into one of two shared-memory stages (K-major core matrices of 8 rows x 16 bytes)
-// while the tensor core works on the other, and the step after that is already on its way from global memory.  65 KB of
-// shared memory: two blocks per SM cover each other's waits.
+// while the tensor core works on the other, and the operands of the following TG_PF steps are on their way from global
+// memory to registers.  65 KB of shared memory: two blocks per SM cover each other's waits.
 constexpr int TG_M = 128, TG_N = 128, TG_K = 16, TG_THREADS = 256, TG_PF = 3;
 constexpr int TG_OPER_BYTES = TG_M * TG_K * 4;            // one operand part of one stage: 8 KB
 constexpr int TG_STAGE_BYTES = 4 * TG_OPER_BYTES;         // A_hi | A_lo | B_hi | B_lo
