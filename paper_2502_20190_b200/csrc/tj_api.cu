@@ -577,7 +577,7 @@ int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const f
   lay_out_update_scratch(x, p);
   p.ldg = x->A; p.value_head = 0;
   p.error = &x->dstats->error;
-  LaunchScope scope(x, TJ_K_SGD, loss_mean_out ? 15 : 14);
+  LaunchScope scope(x, TJ_K_SGD, tj::sgd_step_launches(p) + (loss_mean_out ? 1 : 0));
   cudaError_t e = launch_sgd_step(p, lr, adam, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
   if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
@@ -631,7 +631,7 @@ int tj_ppo_step(tj_ctx* x, const tj_ppo_batch* b, float lr, float beta1, float b
   a.m = m; a.v = v; a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
   a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));
   a.c2 = (float)(1.0 - std::pow((double)beta2, (double)t));
-  LaunchScope scope(x, TJ_K_SGD, stats_out ? 19 : 18);
+  LaunchScope scope(x, TJ_K_SGD, tj::ppo_step_launches(p, stats_out != nullptr));
   cudaError_t e = launch_ppo_step(p, lr, &a, stats_out, x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "PPO update");
   return TJ_OK;

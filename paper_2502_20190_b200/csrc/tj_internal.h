@@ -202,6 +202,8 @@ size_t sgd_scratch_floats(int max_rows, int D, int H);   // activations, deltas 
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam /* nullable: plain SGD */, cudaStream_t s);
+int sgd_step_launches(const SgdParams& p);   // kernels one launch_sgd_step call launches (the path depends on the shape)
+int ppo_step_launches(const SgdParams& p, bool with_stats);
 cudaError_t launch_ppo_step(const SgdParams& p, float lr, const AdamParams* adam, float* stats_out /* device [5], nullable */,
                             cudaStream_t s);
 int td_static_max_rows();

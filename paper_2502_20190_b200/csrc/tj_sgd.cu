@@ -858,6 +858,17 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
 }
 }  // namespace
 
+// launches of the backward pass and the update: dh2 and dh1 (with W2's transpose on the tensor-core path) or the fused
+// backward kernel, the grouped gradient products, the apply pass
+static int backward_launches(const SgdParams& p) {
+  if (!use_tiled(p)) return 3;
+  return (tc_gemm_ok(p.dh2, p.H, p.w2t, p.H, p.n, p.H, p.H) ? 3 : 2) + 2;
+}
+
+int sgd_step_launches(const SgdParams& p) { return (use_tiled(p) ? 7 : 1) + backward_launches(p); }
+
+int ppo_step_launches(const SgdParams& p, bool with_stats) { return 1 + (with_stats ? 1 : 0) + backward_launches(p); }
+
 cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
   if (use_tiled(p)) {
     const int n = p.n, D = p.D, H = p.H, A = p.A;
