@@ -336,3 +336,182 @@ def test_gae_on_an_acquired_segment(orc):
         R = seg["rew"][t] + 0.99 * nd * ((1 - 0.95) * seg["val"][t + 1] + 0.95 * R_next)
         assert np.allclose(ret[t], R, atol=1e-9)
         R_next = R
+
+
+# ------------------------------------------------------------------ the other two environments
+# The building blocks used below (stream words, normals, uniforms, the env steps, the MLP, the selection rule) each have
+# their own pins; these tests pin how the state machine puts them together for the linear-Gaussian and the Acrobot
+# environments: which Philox stream, block, env and step index feeds what, the reset range, what the record holds.
+def _mk_lingauss(orc, D, **kw):
+    A, B = synth.lingauss_matrices(4321, D, 5)
+    base = dict(env_kind=orc.ENV_LINGAUSS, n_envs=3, obs_dim=D, n_actions=5, hidden=8, epsilon=0.25, seed=4321,
+                replay_capacity=12, minibatch=4, staleness_bound=2, warmup=0, gamma=0.99, huber_delta=1.0, lg_A=A, lg_B=B)
+    base.update(kw)
+    return orc.Oracle(**base), base["lg_A"], base["lg_B"]
+
+
+def _bf16_weights(orc, blob, D, H, A):
+    """The blob with its three weight matrices rounded to bfloat16 (biases untouched)."""
+    out = blob.copy()
+    spans = [(0, H * D), (H * D + H, H * D + H + H * H), (H * D + H + H * H + H, H * D + H + H * H + H + A * H)]
+    for lo, hi in spans:
+        out[lo:hi] = [orc.bf16_round(x) for x in blob[lo:hi]]
+    return out
+
+
+@pytest.mark.parametrize("D,done_norm,bf16", [(8, 1.9, False), (128, 7.2, False), (8, 1.9, True)])
+def test_lingauss_actor_step_is_the_composition_of_its_blocks(orc, D, done_norm, bf16):
+    o, A, B = _mk_lingauss(orc, D, lg_done_norm=done_norm, max_episode_steps=6,
+                           weight_dtype=orc.W_BF16 if bf16 else orc.W_FP32)
+    blob = _blob(o, 1)
+    o.publish(blob)
+    used = _bf16_weights(orc, blob, D, 8, 5) if bf16 else blob
+    thr = orc.explore_threshold(0.25)
+    # initial states: RESET words of block b, env e at the all-ones step, U(-0.1, 0.1), components 4b .. 4b+3
+    state = np.zeros((3, D), np.float32)
+    for e in range(3):
+        for b in range(D // 4):
+            w = orc.stream_words(4321, orc.STREAM_RESET, b, e, 2**64 - 1)
+            state[e, 4 * b:4 * b + 4] = [_uniform(orc, x, -0.1, 0.2) for x in w]
+    assert np.array_equal(o.state, state) and np.all(np.abs(state) < 0.1) and np.abs(state).max() > 0.05
+    ep = np.zeros(3, np.int32)
+    ring = np.zeros((12, o.rec_words), np.float32)
+    n_term = n_trunc = n_alive = 0
+    for t in range(14):
+        o.actor_step(1)
+        for e in range(3):
+            if bf16:
+                q = orc.mlp_forward(used, D, 8, 5, state[e], f64=True).astype(np.float32)
+            else:
+                q = orc.mlp_forward(used, D, 8, 5, state[e])
+            w = orc.stream_words(4321, orc.STREAM_ACTION, 0, e, t)
+            a = orc.select_eps_greedy(q, w[0], w[1], thr)
+            noise = np.concatenate([orc.normal4(orc.stream_words(4321, orc.STREAM_NOISE, b, e, t)) for b in range(D // 4)])
+            # the configuration holds both constants as FP32
+            sn, r, term, _ = orc.lingauss_step(state[e], a, A, B, noise, float(np.float32(0.01)), float(np.float32(done_norm)))
+            ep[e] += 1
+            done = int(term or ep[e] >= 6)
+            n_term += term
+            n_trunc += int(not term and ep[e] >= 6)
+            n_alive += 1 - done
+            slot = (3 * t + e) % 12
+            ring[slot, :D] = state[e]
+            ring[slot, D:2 * D] = sn
+            ring[slot].view(np.int32)[2 * D] = a
+            ring[slot, 2 * D + 1] = r
+            ring[slot].view(np.int32)[2 * D + 2] = done
+            ring[slot].view(np.int32)[2 * D + 3] = 1
+            assert np.array_equal(o.last("logits")[e], q)
+            assert o.last("act")[e] == a and o.last("done")[e] == done and o.last("rew")[e] == np.float32(r)
+            if done:
+                for b in range(D // 4):
+                    rw = orc.stream_words(4321, orc.STREAM_RESET, b, e, t)
+                    state[e, 4 * b:4 * b + 4] = [_uniform(orc, x, -0.1, 0.2) for x in rw]
+                ep[e] = 0
+            else:
+                state[e] = sn
+        assert np.array_equal(o.state, state) and np.array_equal(o.ep_step, ep)
+        assert np.array_equal(o.ring.view(np.int32), ring.view(np.int32))
+    assert n_term > 0 and n_alive > 0        # the chosen threshold exercises both branches
+    assert n_trunc > 0 or D == 128
+
+
+def test_lingauss_noise_blocks_are_distinct_per_block_env_and_step(orc):
+    """A wrong block, env or step index in the noise keying would repeat normals somewhere: with A = 0 and B = 0 the new
+    state is 0.01 times the normals, so every component of every env at every step must differ."""
+    D = 16
+    o, _, _ = _mk_lingauss(orc, D, lg_A=np.zeros((D, D), np.float32), lg_B=np.zeros((5, D), np.float32), lg_done_norm=1e9)
+    o.publish(_blob(o, 1))
+    seen = []
+    for t in range(3):
+        o.actor_step(1)
+        seen.append(o.last("next_obs").copy())
+    allv = np.concatenate([s.ravel() for s in seen])
+    assert len(np.unique(allv)) == allv.size
+    assert abs(allv.std() / 0.01 - 1.0) < 0.2
+    # and each is 0.01 * the normal of its (block, env, step)
+    for t in range(3):
+        for e in range(3):
+            for b in range(D // 4):
+                z = orc.normal4(orc.stream_words(4321, orc.STREAM_NOISE, b, e, t))
+                assert np.array_equal(seen[t][e, 4 * b:4 * b + 4], (float(np.float32(0.01)) * z).astype(np.float32))
+
+
+def test_lingauss_default_step_limit_is_200(orc):
+    D = 8
+    o, _, _ = _mk_lingauss(orc, D, lg_A=np.zeros((D, D), np.float32), lg_B=np.zeros((5, D), np.float32), lg_noise_std=0.0,
+                           n_envs=2, replay_capacity=4)
+    o.publish(_blob(o, 1))
+    for t in range(1, 201):
+        o.actor_step(1)
+        assert np.all(o.last("done") == (1 if t == 200 else 0)), t
+        assert np.all(o.last("rew") == 0.0)
+    assert np.all(o.ep_step == 0) and o.stats()["episodes_finished"] == 2
+
+
+def _mk_acrobot(orc, **kw):
+    base = dict(env_kind=orc.ENV_ACROBOT, n_envs=3, obs_dim=6, n_actions=3, hidden=8, epsilon=0.3, seed=777,
+                replay_capacity=12, minibatch=4, staleness_bound=2, warmup=0, gamma=0.99, huber_delta=1.0)
+    base.update(kw)
+    return orc.Oracle(**base)
+
+
+def test_acrobot_actor_step_is_the_composition_of_its_blocks(orc):
+    """The record holds the six-component observation of the state before and after the step, the state itself stays
+    four angles and velocities; reset U(-0.1, 0.1)^4 from RESET block 0; reward 0 on a terminating step, -1 otherwise."""
+    o = _mk_acrobot(orc, max_episode_steps=9)
+    blob = _blob(o, 1)
+    o.publish(blob)
+    thr = orc.explore_threshold(0.3)
+    state = np.zeros((3, 4), np.float32)
+    for e in range(3):
+        w = orc.stream_words(777, orc.STREAM_RESET, 0, e, 2**64 - 1)
+        state[e] = [_uniform(orc, x, -0.1, 0.2) for x in w]
+    assert np.array_equal(o.state, state) and np.abs(state).max() > 0.05
+    # one env is started near the top so that a terminating step occurs within the run
+    state[2] = np.array([3.0, 0.1, 0.5, 0.0], np.float32)
+    o.state[2] = state[2]
+    ep = np.zeros(3, np.int32)
+    ring = np.zeros((12, o.rec_words), np.float32)
+    n_term = 0
+    for t in range(20):
+        o.actor_step(1)
+        for e in range(3):
+            obs = orc.acrobot_obs(state[e])
+            q = orc.mlp_forward(blob, 6, 8, 3, obs)
+            w = orc.stream_words(777, orc.STREAM_ACTION, 0, e, t)
+            a = orc.select_eps_greedy(q, w[0], w[1], thr)
+            sn, r, term, _ = orc.acrobot_step(state[e], a)
+            assert r == (0.0 if term else -1.0)
+            n_term += term
+            ep[e] += 1
+            done = int(term or ep[e] >= 9)
+            slot = (3 * t + e) % 12
+            ring[slot, :6] = obs
+            ring[slot, 6:12] = orc.acrobot_obs(sn)
+            ring[slot].view(np.int32)[12] = a
+            ring[slot, 13] = r
+            ring[slot].view(np.int32)[14] = done
+            ring[slot].view(np.int32)[15] = 1
+            assert o.last("act")[e] == a and o.last("done")[e] == done
+            if done:
+                rw = orc.stream_words(777, orc.STREAM_RESET, 0, e, t)
+                state[e] = [_uniform(orc, x, -0.1, 0.2) for x in rw]
+                ep[e] = 0
+            else:
+                state[e] = sn
+        assert np.array_equal(o.state, state) and np.array_equal(o.ep_step, ep)
+        assert np.array_equal(o.ring.view(np.int32), ring.view(np.int32))
+    assert n_term > 0
+
+
+def test_acrobot_default_step_limit_is_500(orc):
+    o = _mk_acrobot(orc, n_envs=2, replay_capacity=4)
+    o.publish(_blob(o, 1))
+    hanging = np.zeros((2, 4), np.float32)
+    for t in range(1, 501):
+        o.state[:] = hanging                       # at rest, hanging down: the tip stays far below the line
+        o.actor_step(1)
+        assert np.all(o.last("done") == (1 if t == 500 else 0)), t
+        assert np.all(o.last("rew") == -1.0)
+    assert o.stats()["episodes_finished"] == 2 and o.stats()["return_sum"] == -1000.0
