@@ -54,8 +54,8 @@ typedef enum {
   TJ_ERR_NO_WEIGHTS = -5,    /* actor or learner called before the first publish */
   TJ_ERR_WARMUP = -6,        /* fewer resident records than cfg.warmup (Table 2: buffer warmup size) */
   TJ_ERR_STARVED = -7,       /* nothing eligible: the consumer is ahead of the producer (Eq. 3: TR_L ~ TR_A) */
-  TJ_ERR_STALE_SEGMENT = -8, /* reserved */
-  TJ_ERR_TIMEOUT = -9,       /* reserved */
+  TJ_ERR_STALE_SEGMENT = -8, /* tj_segment_check: the producer has begun to overwrite the segment's slot */
+  TJ_ERR_TIMEOUT = -9,       /* tj_stats: a kernel's bounded wait ran out (device_error holds the code) */
   TJ_ERR_UNSUPPORTED = -10   /* valid request this build does not implement */
 } tj_status;
 
@@ -64,8 +64,8 @@ enum { TJ_POLICY_EPS_GREEDY = 0, TJ_POLICY_CATEGORICAL = 1 };
 enum { TJ_W_FP32 = 0, TJ_W_BF16 = 1 };
 /* kernel classes reported by tj_stats (Sec. 3.3: performance analysis measures the production and the
  * consumption side separately) */
-enum { TJ_K_ACTOR_FUSED = 0,  /* MLP + selection + env step + insert in one kernel (FP32 path) */
-       TJ_K_MLP_TENSOR = 1,   /* tensor-core MLP forward (actor or learner) */
+enum { TJ_K_ACTOR_FUSED = 0,  /* MLP + selection + env step + insert in one kernel (FP32 path, or the fused tensor-core actor) */
+       TJ_K_MLP_TENSOR = 1,   /* tensor-core MLP forward alone (the learner's two forwards; the actor's where it is not fused) */
        TJ_K_ENV = 2,          /* selection + env step + insert fed by the tensor-core MLP */
        TJ_K_SAMPLE = 3,       /* eligible list + sample + gather */
        TJ_K_TD = 4,           /* TD error (FP32 forward, or the elementwise pass after tensor-core forwards) */
@@ -141,7 +141,9 @@ typedef struct {
 typedef struct {
   int64_t produced;             /* transitions written */
   int64_t consumed;             /* transitions handed to the learner */
-  int64_t dropped_stale;        /* resident records (or segment transitions) refused for staleness */
+  int64_t dropped_stale;        /* summed over sample calls: resident records outside the bound at that call (a record
+                                   that stays resident and stale is counted by every call that passes it over);
+                                   segment mode: transitions of segments dropped for staleness, each once */
   int64_t dropped_overwritten;  /* segment transitions overwritten before they were consumed */
   int64_t starved_calls;
   int64_t actor_version, learner_version, actor_steps, learner_steps;
@@ -199,7 +201,10 @@ int tj_replay_sample(tj_ctx *ctx, int32_t staleness_bound, int32_t *idx_out, con
 /* Learner, step 2, forward half (Algorithm 1: delta = r + gamma V(s') - V(s), here with a target network
  * and a done mask): q = Q_online(obs)[act]; q' = max_a Q_target(next_obs); y = r + gamma (1-done) q';
  * delta = y - q; Huber(delta; huber_delta).  td_out, huber_out: [n] (nullable); loss_mean_out: 1 float
- * (nullable), the mean Huber loss summed in a fixed order. */
+ * (nullable), the mean Huber loss summed in a fixed order.  1 <= batch.n <= 1,048,576.  In a TJ_W_BF16 context both
+ * forwards run on the tensor cores for every batch size (batches above 65,536 rows in chunks of that many rows).
+ * Should a kernel's bounded wait for its staged parameters run out, the rows of that thread block and the loss are
+ * NaN and device_error is latched (tj_stats). */
 int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_out, float *loss_mean_out);
 
 /* The same computation as tj_td_error for callers that must not allocate and have no scratch to lend.
@@ -216,8 +221,11 @@ int tj_td_error(tj_ctx *ctx, const tj_batch *batch, float *td_out, float *huber_
  * Limits and rules:
  *   - at most 65,536 rows per call; a larger batch.n is refused with TJ_ERR_INVALID_ARG and a message naming
  *     the limit (split the batch or use tj_td_error);
- *   - the first call on each device looks up the array's device address (once per device, with that device
- *     current).  Make that first call at set-up, before any stream capture is under way;
+ *   - the first call on each device looks up the array's device address (once per device; the context's device must
+ *     be the current device, else TJ_ERR_INVALID_ARG).  Make that first call at set-up, before any stream capture
+ *     is under way.  The look-up is guarded by a lock, so first calls from several threads (one context each) are safe;
+ *   - while per-kernel timing is on (tj_set_profiling) the call is timed only if two of the context's CUDA events are
+ *     free for reuse: it never creates one;
  *   - every call, from every context on the device, shares the one array.  Each call rewrites the part it
  *     reads, so nothing needs clearing between calls, but two calls that overlap on the GPU (different
  *     streams) race on it: keep them on one stream or order them with events;
@@ -283,12 +291,21 @@ int tj_gae(tj_ctx *ctx, const float *rew, const float *val, const uint8_t *done,
  * are dropped and counted.  Errors: STARVED. */
 int tj_segment_acquire(tj_ctx *ctx, tj_segment *out);
 
+/* Does a segment view handed out by tj_segment_acquire still show the segment it was acquired as?  TJ_OK while the
+ * producer has not come round to its slot again; TJ_ERR_STALE_SEGMENT once a later segment has begun to fill the slot
+ * (the consumer was lapped: what it reads from the view may be a mixture).  Host bookkeeping only, nothing is enqueued. */
+int tj_segment_check(tj_ctx *ctx, const tj_segment *seg);
+
 /* Views of the env state and the counters; no copy, no synchronisation. */
 int tj_get_state(tj_ctx *ctx, tj_state_view *out);
-/* Restore env state (device pointers, nullable = keep) and the cursor / t / k counters; versions are ignored. */
+/* Restore env state (device pointers, nullable = keep) and the t / k counters; versions are ignored.  The ring, its
+ * per-block versions and the segment slots are not part of the view, so the counters that index them cannot move:
+ * in ring mode `cursor` must equal the current cursor, in segment mode `t` must equal the current t; anything else
+ * is refused with TJ_ERR_UNSUPPORTED and changes nothing. */
 int tj_set_state(tj_ctx *ctx, const tj_state_view *in);
 
-/* Counters (Eq. 2-3: produced vs consumed, sampled staleness).  Synchronises the stream. */
+/* Counters (Eq. 2-3: produced vs consumed, sampled staleness).  Synchronises the stream.  Returns TJ_ERR_TIMEOUT,
+ * with host_out filled all the same, when a kernel has latched device_error. */
 int tj_stats(tj_ctx *ctx, tj_stats_t *host_out);
 
 /* Turn per-kernel timing on or off.  While on, every launch is bracketed by two CUDA events on the context's
@@ -299,6 +316,12 @@ int tj_set_profiling(tj_ctx *ctx, int32_t on);
 /* Views into the ring for inspection: records [C][2D+4] (obs, next_obs, act, rew, done, ver as 32-bit words)
  * and the per-block version summary [C/N]. */
 int tj_ring_view(tj_ctx *ctx, const float **records, const int32_t **block_version, int32_t *record_words);
+
+/* Measured FP32 fused-multiply-add rate of the context's device, in TFLOP/s (Sec. 3.3: resources are sized from measured
+ * rates; this is the rate the FP32 policy kernels are held against).  Runs a register-only FMA loop on every SM five times
+ * on the context's stream and reports the best; synchronises.  scratch: device memory of at least sm_count * 8 KiB (each
+ * thread stores one word so that the loop cannot be optimised away); tflops_out: host.  About 10 ms of GPU time. */
+int tj_calibrate_fp32(tj_ctx *ctx, float *scratch, size_t scratch_bytes, double *tflops_out);
 
 const char *tj_last_error(const tj_ctx *ctx);
 

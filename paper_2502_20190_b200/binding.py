@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view",
+           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_segment_check", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view", "tj_calibrate_fp32",
            "tj_last_error")
 
 
@@ -93,11 +93,13 @@ def load_library():
     L.tj_adam_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, vp, vp, vp, vp, vp]
     L.tj_ppo_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, f32, f32, f32, vp, vp, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
+    L.tj_segment_check.argtypes = [vp, vp]
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
     L.tj_stats.argtypes = [vp, vp]
     L.tj_set_profiling.argtypes = [vp, i32]
     L.tj_ring_view.argtypes = [vp, vp, vp, vp]
+    L.tj_calibrate_fp32.argtypes = [vp, vp, C.c_size_t, vp]
     L.tj_last_error.argtypes = [vp]
     L.tj_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -185,6 +187,10 @@ def tj_segment_acquire(h):
     return st, seg
 
 
+def tj_segment_check(h, seg: TjSegment):
+    return load_library().tj_segment_check(h, C.byref(seg))
+
+
 def tj_get_state(h):
     v = TjStateView()
     st = load_library().tj_get_state(h, C.byref(v))
@@ -209,6 +215,12 @@ def tj_ring_view(h):
     rec, bv, rw = C.c_void_p(), C.c_void_p(), C.c_int32()
     st = load_library().tj_ring_view(h, C.byref(rec), C.byref(bv), C.byref(rw))
     return st, rec.value, bv.value, rw.value
+
+
+def tj_calibrate_fp32(h, scratch_ptr: int, scratch_bytes: int):
+    out = C.c_double()
+    st = load_library().tj_calibrate_fp32(h, scratch_ptr, scratch_bytes, C.byref(out))
+    return st, out.value
 
 
 def tj_last_error(h=None) -> str:
@@ -396,11 +408,14 @@ class Context:
         if st != TJ_OK:
             return st, None
         T, N, D = seg.T, seg.N, self.D
-        return st, dict(T=T, N=N, version=seg.version,
+        return st, dict(T=T, N=N, version=seg.version, c=seg,
                         obs=self._view(seg.obs, (T, N, D), torch.float32), act=self._view(seg.act, (T, N), torch.int32),
                         rew=self._view(seg.rew, (T, N), torch.float32), done=self._view(seg.done, (T, N), torch.uint8),
                         logp=self._view(seg.logp, (T, N), torch.float32),
                         val=self._view(seg.val, (T + 1, N), torch.float32))
+
+    def segment_check(self, seg, allow=(TJ_OK, TJ_ERR_STALE_SEGMENT)):
+        return self._check(tj_segment_check(self.h, seg["c"]), allow)
 
     def get_state(self):
         torch = self.torch
@@ -417,12 +432,19 @@ class Context:
 
     def stats(self):
         st, s = tj_stats(self.h)
-        self._check(st)
+        self._check(st, (TJ_OK, TJ_ERR_TIMEOUT))   # on a latched device error the counters are filled all the same
         arrays = ("staleness_hist", "kernel_count", "kernel_ms")
         d = {k: getattr(s, k) for k, _ in TjStats._fields_ if k not in arrays}
         for k in arrays:
             d[k] = list(getattr(s, k))
         return d
+
+    def calibrate_fp32(self):
+        """Measured FP32 FMA rate of the device in TFLOP/s (a register-only FMA loop on every SM)."""
+        scratch = self.torch.empty(256 * 8192, dtype=self.torch.uint8, device=self.device)
+        st, v = tj_calibrate_fp32(self.h, scratch.data_ptr(), scratch.numel())
+        self._check(st)
+        return v
 
     def set_profiling(self, on):
         return self._check(tj_set_profiling(self.h, on))

@@ -50,33 +50,6 @@ __device__ inline ActorSmem carve(float* base, int TE, int D, int Hp, int Ap, bo
   return s;
 }
 
-// Queue the bulk copies of the staged parameter ranges (one thread) and name where each part is read from.
-template <int STAGE>
-__device__ __forceinline__ MlpWeights stage_weights(const ActorParams& p, float* wsm, uint64_t* bar, bool issue) {
-  MlpWeights w;
-  if (STAGE == 0) {
-    w.W1t = p.W + p.off_W1t; w.b1 = p.W + p.off_b1; w.W2t = p.W + p.off_W2t; w.b2 = p.W + p.off_b2;
-    w.W3t = p.W + p.off_W3t; w.b3 = p.W + p.off_b3;
-    return w;
-  }
-  const size_t gap = STAGE == 1 ? p.off_b2 - p.off_W2t : 0;
-  if (issue) {
-    if (STAGE == 2) {
-      mbar_expect_tx(bar, (uint32_t)(p.w_total * sizeof(float)));
-      bulk_copy_chunks(wsm, p.W, p.w_total * sizeof(float), bar);
-    } else {
-      const size_t head = p.off_W2t, tail = p.w_total - p.off_b2;
-      mbar_expect_tx(bar, (uint32_t)((head + tail) * sizeof(float)));
-      bulk_copy_chunks(wsm, p.W, head * sizeof(float), bar);
-      bulk_copy_chunks(wsm + head, p.W + p.off_b2, tail * sizeof(float), bar);
-    }
-  }
-  w.W1t = wsm + p.off_W1t; w.b1 = wsm + p.off_b1;
-  w.W2t = STAGE == 2 ? wsm + p.off_W2t : p.W + p.off_W2t;
-  w.b2 = wsm + p.off_b2 - gap; w.W3t = wsm + p.off_W3t - gap; w.b3 = wsm + p.off_b3 - gap;
-  return w;
-}
-
 __device__ __forceinline__ float4 reset4(uint2 seed, uint32_t block, uint32_t e, unsigned long long step, float lo,
                                          float width) {
   const uint4 w = stream_words(seed, STREAM_RESET, block, e, step);
@@ -100,7 +73,7 @@ __global__ void __launch_bounds__(NT) actor_small_env_kernel(const ActorParams p
     if (tid == 0) mbar_init(&wbar, 1);
     __syncthreads();
   }
-  const MlpWeights mw = stage_weights<STAGE>(p, sm.w, &wbar, tid == 0);
+  const MlpWeights mw = stage_mlp_weights<STAGE>(p, p.W, sm.w, &wbar, tid == 0);
 
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   int ep = 0;
@@ -243,7 +216,7 @@ __global__ void __launch_bounds__(NT) actor_lingauss_kernel(const ActorParams p)
   const bool ext = p.logits_in != nullptr;   // network outputs come from the tensor-core kernel
   const ActorSmem sm = carve(smem, TE, p.D, ext ? 0 : p.Hp, ext ? 0 : p.Ap, true, 0);
   __shared__ uint64_t unused_bar;
-  const MlpWeights mw = stage_weights<0>(p, nullptr, &unused_bar, false);
+  const MlpWeights mw = stage_mlp_weights<0>(p, p.W, nullptr, &unused_bar, false);
   const int tid = threadIdx.x;
   const int e0 = blockIdx.x * TE;
   const int D = p.D, Dp = (p.D + 3) & ~3;

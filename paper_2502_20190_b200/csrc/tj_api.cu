@@ -164,9 +164,12 @@ struct LaunchScope {
   tj_ctx* x;
   cudaEvent_t a = nullptr, b = nullptr;
   int cls;
-  LaunchScope(tj_ctx* ctx, int kernel_class, int n_launches) : x(ctx), cls(kernel_class) {
+  // may_create = false: time the launches only if two pooled events are free (an entry point that must not create
+  // anything skips the timing rather than make events)
+  LaunchScope(tj_ctx* ctx, int kernel_class, int n_launches, bool may_create = true) : x(ctx), cls(kernel_class) {
     x->hs.kernel_launches += n_launches;
     if (!x->profiling) return;
+    if (!may_create && x->ev_pool.size() < 2) return;
     a = take(); b = take();
     if (a && b) cudaEventRecord(a, x->stream);
   }
@@ -391,7 +394,7 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
         ev.ring = x->ring; ev.C = c.replay_capacity; ev.cursor = x->cursor + (uint64_t)i * x->N; ev.block_ver = x->block_ver;
         ev.lgA_hi = x->lgA_hi; ev.lgA_lo = x->lgA_lo; ev.lgB = x->lgB;
         ev.noise_std = c.lg_noise_std; ev.done_norm = c.lg_done_norm; ev.stats = x->dstats;
-        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
+        LaunchScope scope(x, TJ_K_ACTOR_FUSED, 1);
         if (x->use_tc_pipelined) {
           t.wtc = x->wtc_pipe[x->active];
           ev.z_scratch = x->z_scratch;
@@ -479,12 +482,17 @@ int tj_replay_sample(tj_ctx* x, int32_t staleness_bound, int32_t* idx_out, const
   return TJ_OK;
 }
 
-int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out) {
-  if (!x) return TJ_ERR_INVALID_ARG;
+namespace {
+// checks shared by the two TD-error entry points; 0 = fine
+int td_check(tj_ctx* x, const tj_batch* b) {
   if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
-  if (b->n < 1 || b->n > kMaxTdRows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n out of range");
+  if (b->n < 1) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be positive");
   if (x->cfg.policy_kind != TJ_POLICY_EPS_GREEDY) return fail(x, TJ_ERR_UNSUPPORTED, "TD error needs the Q head");
   if (x->version == 0 || !x->has_target) return fail(x, TJ_ERR_NO_WEIGHTS, "TD error called before the first publish");
+  return TJ_OK;
+}
+
+TdParams td_params(const tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out, float* partial) {
   TdParams p{};
   p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
   p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
@@ -492,26 +500,45 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
   p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3; p.w_total = x->wl.total;
   p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
   p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
-  p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = x->td_partial;
+  p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = partial;
+  p.error = &x->dstats->error;
+  return p;
+}
+}  // namespace
+
+int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (int st = td_check(x, b)) return st;
+  if (b->n > kMaxTdRows) return fail(x, TJ_ERR_INVALID_ARG, "batch.n out of range");
+  const TdParams p = td_params(x, b, td_out, huber_out, loss_mean_out, x->td_partial);
   cudaError_t e;
-  if (x->use_tc && b->n <= kMaxTcTdRows) {
-    // two tensor-core forwards (online on obs, target on next_obs), then the elementwise TD/Huber pass
-    for (int which = 0; which < 2; ++which) {
-      const float* W = which == 0 ? x->wbuf[x->active] : x->wtarget;
-      TcMlpParams t{};
-      t.x = which == 0 ? b->obs : b->next_obs; t.n = b->n; t.D = x->D; t.H = x->H; t.Aout = x->A;
-      t.wtc = which == 0 ? x->wtc[x->active] : x->wtc_target;
-      t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
-      t.out = x->tdq[which]; t.error = &x->dstats->error;
-      LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
-      if ((e = launch_tc_mlp(t, x->sm_count, x->stream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
+  if (x->use_tc) {
+    // per chunk of at most kMaxTcTdRows rows (what the Q-value buffers hold): two tensor-core forwards (online on obs,
+    // target on next_obs), then the elementwise TD/Huber pass.  The chunk length is a multiple of the 16 rows one
+    // partial sum covers, so the partial sums lie exactly as they would for a single pass.
+    for (int r0 = 0; r0 < b->n; r0 += kMaxTcTdRows) {
+      const int rows = std::min(kMaxTcTdRows, b->n - r0);
+      for (int which = 0; which < 2; ++which) {
+        const float* W = which == 0 ? x->wbuf[x->active] : x->wtarget;
+        TcMlpParams t{};
+        t.x = (which == 0 ? b->obs : b->next_obs) + (size_t)r0 * x->D; t.n = rows; t.D = x->D; t.H = x->H; t.Aout = x->A;
+        t.wtc = which == 0 ? x->wtc[x->active] : x->wtc_target;
+        t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
+        t.out = x->tdq[which]; t.error = &x->dstats->error;
+        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
+        if ((e = launch_tc_mlp(t, x->sm_count, x->stream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
+      }
+      LaunchScope scope(x, TJ_K_TD, 1);
+      if ((e = launch_td_from_q(x->tdq[0], x->tdq[1], rows, x->A, b->act + r0, b->rew + r0, b->done + r0, p.gamma, p.kappa,
+                                td_out ? td_out + r0 : nullptr, huber_out ? huber_out + r0 : nullptr,
+                                x->td_partial + r0 / 16, x->stream)) != cudaSuccess)
+        return cuda_fail(x, e, "TD error (elementwise)");
     }
-    LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1);
-    if ((e = launch_td_from_q(x->tdq[0], x->tdq[1], b->n, x->A, b->act, b->rew, b->done, p.gamma, p.kappa, td_out,
-                              huber_out, x->td_partial, x->stream)) != cudaSuccess)
-      return cuda_fail(x, e, "TD error (elementwise)");
-    if (loss_mean_out && (e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
-      return cuda_fail(x, e, "TD error (loss reduction)");
+    if (loss_mean_out) {
+      LaunchScope scope(x, TJ_K_TD, 1);
+      if ((e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
+        return cuda_fail(x, e, "TD error (loss reduction)");
+    }
     return TJ_OK;
   }
   LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1);
@@ -522,27 +549,19 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
 
 int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, float* loss_mean_out) {
   if (!x) return TJ_ERR_INVALID_ARG;
-  if (!b || !b->obs || !b->act || !b->rew || !b->next_obs || !b->done) return fail(x, TJ_ERR_INVALID_ARG, "batch arrays must not be null");
-  if (b->n < 1) return fail(x, TJ_ERR_INVALID_ARG, "batch.n must be positive");
-  if (x->cfg.policy_kind != TJ_POLICY_EPS_GREEDY) return fail(x, TJ_ERR_UNSUPPORTED, "TD error needs the Q head");
-  if (x->version == 0 || !x->has_target) return fail(x, TJ_ERR_NO_WEIGHTS, "TD error called before the first publish");
-  TdParams p{};
-  p.n = b->n; p.D = x->D; p.H = x->H; p.A = x->A; p.Hp = x->wl.Hp; p.Ap = x->wl.Ap;
-  p.Wonline = x->wbuf[x->active]; p.Wtarget = x->wtarget;
-  p.off_W1t = x->wl.off_W1t; p.off_b1 = x->wl.off_b1; p.off_W2t = x->wl.off_W2t; p.off_b2 = x->wl.off_b2;
-  p.off_W3t = x->wl.off_W3t; p.off_b3 = x->wl.off_b3; p.w_total = x->wl.total;
-  p.obs = b->obs; p.act = b->act; p.rew = b->rew; p.next_obs = b->next_obs; p.done = b->done;
-  p.gamma = x->cfg.gamma; p.kappa = x->cfg.huber_delta;
-  p.td_out = td_out; p.huber_out = huber_out; p.loss_out = loss_mean_out; p.partial = nullptr;
-  bool too_large = false;
-  x->hs.kernel_launches += loss_mean_out ? 2 : 1;
-  cudaError_t e = launch_td_static(p, x->stream, &too_large);
-  if (too_large) {
+  if (int st = td_check(x, b)) return st;
+  if (b->n > td_static_max_rows()) {
     char msg[160];
     std::snprintf(msg, sizeof(msg), "tj_td_error_static takes at most %d rows per call (got %d); use tj_td_error or split the batch",
                   td_static_max_rows(), b->n);
     return fail(x, TJ_ERR_INVALID_ARG, msg);
   }
+  const TdParams p = td_params(x, b, td_out, huber_out, loss_mean_out, nullptr);
+  bool too_large = false;
+  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1, /*may_create=*/false);
+  cudaError_t e = launch_td_static(p, x->cfg.device, x->stream, &too_large);
+  if (too_large) return fail(x, TJ_ERR_INVALID_ARG, "tj_td_error_static: batch too large for the library's scratch");
+  if (e == cudaErrorInvalidDevice) return fail(x, TJ_ERR_INVALID_ARG, "tj_td_error_static: the context's device must be the current device");
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error (library scratch)");
   return TJ_OK;
 }
@@ -675,6 +694,7 @@ int tj_segment_acquire(tj_ctx* x, tj_segment* out) {
     out->logp = x->seg_logp + slot * TN;
     out->val = x->seg_val + slot * ((size_t)T + 1) * N;
     sl.state = 3;
+    sl.acquired_index = sl.index;
     x->next_consume += 1;
     x->k += 1;
     x->hs.learner_steps += 1;
@@ -688,6 +708,20 @@ int tj_segment_acquire(tj_ctx* x, tj_segment* out) {
   return fail(x, TJ_ERR_STARVED, "no complete segment within the staleness bound");
 }
 
+int tj_segment_check(tj_ctx* x, const tj_segment* segv) {
+  if (!x || !segv) return TJ_ERR_INVALID_ARG;
+  const tj_config& c = x->cfg;
+  if (c.replay_capacity != 0) return fail(x, TJ_ERR_INVALID_ARG, "segments exist only in segment mode");
+  const size_t TN = (size_t)c.rollout_len * x->N;
+  if (!segv->rew || segv->rew < x->seg_rew || (size_t)(segv->rew - x->seg_rew) % TN) return fail(x, TJ_ERR_INVALID_ARG, "not a segment of this context");
+  const size_t slot = (size_t)(segv->rew - x->seg_rew) / TN;
+  if (slot >= (size_t)c.n_segments) return fail(x, TJ_ERR_INVALID_ARG, "not a segment of this context");
+  const SegSlot& sl = x->seg[slot];
+  // consumed (3) and still holding the segment it was acquired as: the producer has not come round to the slot
+  if (sl.state == 3 && sl.version == segv->version && sl.index == sl.acquired_index) return TJ_OK;
+  return fail(x, TJ_ERR_STALE_SEGMENT, "the producer has started to overwrite this segment's slot");
+}
+
 int tj_get_state(tj_ctx* x, tj_state_view* out) {
   if (!x || !out) return TJ_ERR_INVALID_ARG;
   out->state = x->state; out->ep_step = x->ep_step;
@@ -699,7 +733,13 @@ int tj_get_state(tj_ctx* x, tj_state_view* out) {
 int tj_set_state(tj_ctx* x, const tj_state_view* in) {
   if (!x || !in) return TJ_ERR_INVALID_ARG;
   if (in->t < 0 || in->k < 0) return fail(x, TJ_ERR_INVALID_ARG, "counters must not be negative");
-  if (x->cfg.replay_capacity > 0 && in->cursor % (uint64_t)x->N) return fail(x, TJ_ERR_INVALID_ARG, "cursor must be a multiple of n_envs");
+  // The ring's contents, its per-block versions and the segment slots are not part of the view, so the counters that index
+  // them cannot move: another cursor (ring mode) or another step count (segment mode) would leave the sampler and the
+  // segment bookkeeping describing records that are not the resident ones.
+  if (x->cfg.replay_capacity > 0 && in->cursor != x->cursor)
+    return fail(x, TJ_ERR_UNSUPPORTED, "the cursor cannot be moved: the ring and its block versions are not part of the state view");
+  if (x->cfg.replay_capacity == 0 && in->t != x->t)
+    return fail(x, TJ_ERR_UNSUPPORTED, "t cannot be moved in segment mode: the segment slots are not part of the state view");
   cudaError_t e;
   if (in->state && in->state != x->state &&
       (e = cudaMemcpyAsync(x->state, in->state, sizeof(float) * (size_t)x->N * x->S_d, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
@@ -707,7 +747,7 @@ int tj_set_state(tj_ctx* x, const tj_state_view* in) {
   if (in->ep_step && in->ep_step != x->ep_step &&
       (e = cudaMemcpyAsync(x->ep_step, in->ep_step, sizeof(int) * (size_t)x->N, cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
     return cuda_fail(x, e, "set episode steps");
-  x->cursor = in->cursor; x->t = in->t; x->k = in->k;
+  x->t = in->t; x->k = in->k;
   return TJ_OK;
 }
 
@@ -727,6 +767,7 @@ int tj_stats(tj_ctx* x, tj_stats_t* o) {
     o->max_sampled_staleness = (int64_t)d.max_stale;
     for (int i = 0; i < 33; ++i) o->staleness_hist[i] = (int64_t)d.hist[i];
   }
+  if (d.error) return fail(x, TJ_ERR_TIMEOUT, "a kernel's bounded wait ran out (device_error holds the code); its outputs are not valid");
   return TJ_OK;
 }
 
@@ -735,6 +776,32 @@ int tj_ring_view(tj_ctx* x, const float** records, const int32_t** block_version
   if (records) *records = x->ring;
   if (block_version) *block_version = x->block_ver;
   if (record_words) *record_words = x->rec_words;
+  return TJ_OK;
+}
+
+int tj_calibrate_fp32(tj_ctx* x, float* scratch, size_t scratch_bytes, double* tflops_out) {
+  if (!x || !tflops_out) return TJ_ERR_INVALID_ARG;
+  const size_t need = fma_rate_sink_floats(x->sm_count) * sizeof(float);
+  if (!scratch || scratch_bytes < need) return fail(x, TJ_ERR_WORKSPACE, "calibration scratch too small (needs sm_count * 8 KiB)");
+  cudaEvent_t a = nullptr, b = nullptr;
+  if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return fail(x, TJ_ERR_CUDA, "calibration: event creation failed");
+  cudaError_t e = cudaSuccess;
+  double best = 0.0;
+  launch_fma_rate(scratch, x->sm_count, 64, x->stream, &e);            // warm-up
+  for (int rep = 0; rep < 5 && e == cudaSuccess; ++rep) {
+    cudaEventRecord(a, x->stream);
+    const double flops = launch_fma_rate(scratch, x->sm_count, 4096, x->stream, &e);
+    cudaEventRecord(b, x->stream);
+    if (e != cudaSuccess) break;
+    if ((e = cudaEventSynchronize(b)) != cudaSuccess) break;
+    float ms = 0.f;
+    if ((e = cudaEventElapsedTime(&ms, a, b)) != cudaSuccess) break;
+    if (ms > 0.f) best = std::max(best, flops / (ms * 1e-3) / 1e12);
+  }
+  cudaEventDestroy(a);
+  cudaEventDestroy(b);
+  if (e != cudaSuccess) return cuda_fail(x, e, "calibration");
+  *tflops_out = best;
   return TJ_OK;
 }
 

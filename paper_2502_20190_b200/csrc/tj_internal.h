@@ -91,6 +91,7 @@ struct TdParams {
   float* huber_out;
   float* loss_out;
   float* partial;  // scratch: one float per thread block
+  unsigned long long* error;  // device error word of the context (a bounded wait that ran out)
 };
 
 struct SgdParams {
@@ -207,9 +208,11 @@ int ppo_step_launches(const SgdParams& p, bool with_stats);
 cudaError_t launch_ppo_step(const SgdParams& p, float lr, const AdamParams* adam, float* stats_out /* device [5], nullable */,
                             cudaStream_t s);
 int td_static_max_rows();
-cudaError_t launch_td_static(const TdParams& p, cudaStream_t s, bool* too_large);
+cudaError_t launch_td_static(const TdParams& p, int device, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
                        float* adv, float* ret, cudaStream_t s);
+size_t fma_rate_sink_floats(int sm_count);
+double launch_fma_rate(float* sink, int sm_count, int outer, cudaStream_t s, cudaError_t* err);
 cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);
 
 }  // namespace tj
@@ -218,6 +221,7 @@ struct SegSlot {
   int64_t index = -1;   // which segment number sits in the slot
   int64_t version = 0;
   int state = 0;        // 0 empty, 1 filling, 2 complete, 3 consumed or dropped
+  int64_t acquired_index = -1;   // segment number handed out by the last tj_segment_acquire of this slot
 };
 
 struct tj_ctx {

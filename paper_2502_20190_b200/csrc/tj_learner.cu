@@ -1,5 +1,7 @@
 // Learner-side kernels: parameter publish (repack), eligible-block list, staleness-bounded sampling with
 // gather, TD error / Huber loss, and the GAE reverse scan.
+#include <mutex>
+
 #include "tj_async.cuh"
 #include "tj_device.cuh"
 #include "tj_internal.h"
@@ -164,32 +166,19 @@ __global__ void sample_gather_vec_kernel(const SampleParams p) {
 }
 
 // TD error on a tile of TE samples: online forward on obs, target forward on next_obs.
-// STAGE as in the actor kernel: 0 = parameters from global memory, 1 = all but the HxH matrix staged in shared
-// memory, 2 = all staged.  The staging buffer is filled twice (online, then target parameters).
-template <int STAGE>
-__device__ __forceinline__ MlpWeights td_stage(const TdParams& p, const float* W, float* wsm, uint64_t* bar, bool issue) {
-  MlpWeights w;
-  if (STAGE == 0) {
-    w.W1t = W + p.off_W1t; w.b1 = W + p.off_b1; w.W2t = W + p.off_W2t; w.b2 = W + p.off_b2;
-    w.W3t = W + p.off_W3t; w.b3 = W + p.off_b3;
-    return w;
+// STAGE as in the actor kernel (stage_mlp_weights); the staging buffer is filled twice (online, then target parameters).
+// A staging wait that ran out: latch the context's error word and leave defined outputs (NaN) for this block's rows and
+// its partial sum, so that neither the caller nor the loss reduction reads what an earlier call left there.
+__device__ __forceinline__ void td_give_up(const TdParams& p, int n_here, int j0) {
+  const float nan = __int_as_float(0x7FC00000);
+  if (threadIdx.x == 0) {
+    if (p.error) atomicExch(p.error, 3ull);
+    p.partial[blockIdx.x] = nan;
   }
-  const size_t gap = STAGE == 1 ? p.off_b2 - p.off_W2t : 0;
-  if (issue) {
-    if (STAGE == 2) {
-      mbar_expect_tx(bar, (uint32_t)(p.w_total * sizeof(float)));
-      bulk_copy_chunks(wsm, W, p.w_total * sizeof(float), bar);
-    } else {
-      const size_t head = p.off_W2t, tail = p.w_total - p.off_b2;
-      mbar_expect_tx(bar, (uint32_t)((head + tail) * sizeof(float)));
-      bulk_copy_chunks(wsm, W, head * sizeof(float), bar);
-      bulk_copy_chunks(wsm + head, W + p.off_b2, tail * sizeof(float), bar);
-    }
+  if ((int)threadIdx.x < n_here) {
+    if (p.td_out) p.td_out[j0 + threadIdx.x] = nan;
+    if (p.huber_out) p.huber_out[j0 + threadIdx.x] = nan;
   }
-  w.W1t = wsm + p.off_W1t; w.b1 = wsm + p.off_b1;
-  w.W2t = STAGE == 2 ? wsm + p.off_W2t : W + p.off_W2t;
-  w.b2 = wsm + p.off_b2 - gap; w.W3t = wsm + p.off_W3t - gap; w.b3 = wsm + p.off_b3 - gap;
-  return w;
 }
 
 template <int TE, int NT, int EPT, int NPT, int STAGE>
@@ -210,13 +199,13 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
     if (tid == 0) mbar_init(&wbar, 1);
     __syncthreads();
   }
-  MlpWeights mw = td_stage<STAGE>(p, p.Wonline, wsm, &wbar, tid == 0);
+  MlpWeights mw = stage_mlp_weights<STAGE>(p, p.Wonline, wsm, &wbar, tid == 0);
 
   for (int i = tid; i < TE * D; i += NT) {
     const int el = i / D, k = i % D;
     xs[k * TE + el] = el < n_here ? p.obs[(size_t)(j0 + el) * D + k] : 0.f;
   }
-  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) return;
+  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 0)) { td_give_up(p, n_here, j0); return; }
   __syncthreads();
   mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < n_here) {
@@ -225,12 +214,12 @@ __global__ void __launch_bounds__(NT) td_kernel(const TdParams p) {
     qsel[tid] = out[a * TE + tid];
   }
   __syncthreads();  // every thread is done with the online parameters: the buffer may be refilled
-  mw = td_stage<STAGE>(p, p.Wtarget, wsm, &wbar, tid == 0);
+  mw = stage_mlp_weights<STAGE>(p, p.Wtarget, wsm, &wbar, tid == 0);
   for (int i = tid; i < TE * D; i += NT) {
     const int el = i / D, k = i % D;
     xs[k * TE + el] = el < n_here ? p.next_obs[(size_t)(j0 + el) * D + k] : 0.f;
   }
-  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 1)) return;
+  if (STAGE > 0 && !mbar_wait_bounded(&wbar, 1)) { td_give_up(p, n_here, j0); return; }
   __syncthreads();
   mlp_forward_tile<TE, NT, EPT, (STAGE > 0), (STAGE == 2), NPT>(mw, D, p.H, p.Hp, p.A, p.Ap, xs, h1, h2, out);
   if (tid < TE) {
@@ -416,23 +405,31 @@ static __device__ __align__(256) float g_td_static_partial[kStaticTdPartials];
 
 int td_static_max_rows() { return 65536; }
 
-cudaError_t launch_td_static(const TdParams& p_in, cudaStream_t s, bool* too_large) {
+cudaError_t launch_td_static(const TdParams& p_in, int device, cudaStream_t s, bool* too_large) {
   *too_large = p_in.n > td_static_max_rows() || td_grid(p_in.n) > kStaticTdPartials;
   if (*too_large) return cudaSuccess;
-  // In host code the array's name is only a stand-in; the device address has to be asked for, once per device.
+  // In host code the array's name is only a stand-in; the device address has to be asked for, once per device, with
+  // that device current.  The table is keyed by the context's device and filled under a lock, so first calls from
+  // several threads (one context each) do not race.
   static float* addr_by_device[64] = {};
+  static std::mutex addr_lock;
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!addr_by_device[dev]) {
-    float* q = nullptr;
-    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&q), g_td_static_partial);
-    if (e != cudaSuccess) return e;
-    addr_by_device[dev] = q;
+  if (device < 0 || device >= 64 || dev != device) return cudaErrorInvalidDevice;
+  float* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> hold(addr_lock);
+    if (!addr_by_device[device]) {
+      float* q = nullptr;
+      e = cudaGetSymbolAddress(reinterpret_cast<void**>(&q), g_td_static_partial);
+      if (e != cudaSuccess) return e;
+      addr_by_device[device] = q;
+    }
+    scratch = addr_by_device[device];
   }
   TdParams p = p_in;
-  p.partial = addr_by_device[dev];
+  p.partial = scratch;
   return launch_td(p, s);
 }
 

@@ -7,6 +7,8 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include "tj_async.cuh"
+
 namespace tj {
 
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_TANH = 2 };
@@ -120,6 +122,35 @@ __device__ __forceinline__ void head_layer(const float* __restrict__ Wt, const f
 struct MlpWeights {
   const float *W1t, *b1, *W2t, *b2, *W3t, *b3;
 };
+
+// Queue the bulk copies of the staged parameter ranges (one thread, `issue`) and name where each part is read from.
+// STAGE 0: everything from global memory; 1: all but the H x H matrix staged in shared memory; 2: all staged.
+// P is a parameter struct with the packed layout's offsets (off_W1t .. off_b3, w_total); W the packed parameters.
+template <int STAGE, typename P>
+__device__ __forceinline__ MlpWeights stage_mlp_weights(const P& p, const float* W, float* wsm, uint64_t* bar, bool issue) {
+  MlpWeights w;
+  if (STAGE == 0) {
+    w.W1t = W + p.off_W1t; w.b1 = W + p.off_b1; w.W2t = W + p.off_W2t; w.b2 = W + p.off_b2;
+    w.W3t = W + p.off_W3t; w.b3 = W + p.off_b3;
+    return w;
+  }
+  const size_t gap = STAGE == 1 ? p.off_b2 - p.off_W2t : 0;
+  if (issue) {
+    if (STAGE == 2) {
+      mbar_expect_tx(bar, (uint32_t)(p.w_total * sizeof(float)));
+      bulk_copy_chunks(wsm, W, p.w_total * sizeof(float), bar);
+    } else {
+      const size_t head = p.off_W2t, tail = p.w_total - p.off_b2;
+      mbar_expect_tx(bar, (uint32_t)((head + tail) * sizeof(float)));
+      bulk_copy_chunks(wsm, W, head * sizeof(float), bar);
+      bulk_copy_chunks(wsm + head, W + p.off_b2, tail * sizeof(float), bar);
+    }
+  }
+  w.W1t = wsm + p.off_W1t; w.b1 = wsm + p.off_b1;
+  w.W2t = STAGE == 2 ? wsm + p.off_W2t : W + p.off_W2t;
+  w.b2 = wsm + p.off_b2 - gap; w.W3t = wsm + p.off_W3t - gap; w.b3 = wsm + p.off_b3 - gap;
+  return w;
+}
 
 // Policy forward for the tile: x [D][TE] -> h1 -> h2 -> out [Ap][TE]; ends with a barrier.
 // SMALL_SMEM: W1t, the biases and W3t are in shared memory;  W2_SMEM: W2t is too.

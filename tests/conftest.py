@@ -17,3 +17,15 @@ def orc():
     import oracle
     oracle.build()
     return oracle
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Shares of margin-rule decisions recorded by the parity tests (shown whether or not output is captured)."""
+    try:
+        import parity_util
+    except ImportError:
+        return
+    if parity_util.REPORT:
+        terminalreporter.write_sep("-", "decisions inside the oracle's margins")
+        for line in parity_util.REPORT:
+            terminalreporter.write_line(line)

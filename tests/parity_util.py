@@ -48,6 +48,9 @@ def blob_for(fields, version, seed=None):
                              fields["n_actions"], vh, bf16_exact=False)
 
 
+REPORT = []          # lines the terminal summary prints after the run (tests/conftest.py)
+
+
 class Tally:
     """Counts decisions that fell inside the oracle's margin (compared for validity, not equality)."""
 
@@ -55,6 +58,23 @@ class Tally:
         self.total = 0
         self.ambiguous_done = 0
         self.ambiguous_act = 0
+        self.max_logit_dev = 0.0      # largest |GPU - oracle| network output seen, relative to the oracle's rms
+
+    def report(self, name):
+        """Record the shares of decisions that fell inside a margin: they are counted and shown, never dropped silently."""
+        n = max(self.total, 1)
+        line = "%s: %d decisions, ambiguous actions %.3f %%, ambiguous done flags %.3f %%, largest output deviation %.2e of rms" % (
+            name, self.total, 100.0 * self.ambiguous_act / n, 100.0 * self.ambiguous_done / n, self.max_logit_dev)
+        REPORT.append(line)
+        print(line)
+        return self.ambiguous_act / n, self.ambiguous_done / n
+
+
+def measured_margin(g_logits, o_logits):
+    """Twice the largest deviation between the two sides' outputs on this step.  When the oracle's gap between its two
+    largest outputs exceeds it, both sides must pick the same maximum whatever the rounding: a margin taken from what
+    was measured, not from the tolerance (which the outputs are checked against separately)."""
+    return 2.0 * float(np.max(np.abs(np.asarray(g_logits, np.float64) - np.asarray(o_logits, np.float64)))) + 1e-12
 
 
 def lockstep_step(ctx, o, torch, *, rtol, env_kind, tally, logits_exact=None, act_rtol=None, dbg=None):
@@ -82,6 +102,8 @@ def lockstep_step(ctx, o, torch, *, rtol, env_kind, tally, logits_exact=None, ac
         assert np.array_equal(g_logits.view(np.uint32), o_logits.view(np.uint32)), "logits differ bitwise"
     else:
         close(g_logits, o_logits, rtol, "logits")
+        rms = math.sqrt(float(np.mean(o_logits.astype(np.float64) ** 2))) + 1e-30
+        tally.max_logit_dev = max(tally.max_logit_dev, float(np.max(np.abs(g_logits.astype(np.float64) - o_logits))) / rms)
     st1 = ctx.get_state()
     g_state = st1["state"].cpu().numpy()
     g_ep = st1["ep_step"].cpu().numpy()

@@ -8,7 +8,8 @@ compared exactly whenever the oracle's distance to the threshold exceeds the tol
 import numpy as np
 import pytest
 
-from parity_util import (RTOL_FP32, Tally, blob_for, close, compare_ring_step, fields_for, lockstep_step, make_pair)
+from parity_util import (RTOL_FP32, Tally, blob_for, close, compare_ring_step, fields_for, lockstep_step, make_pair,
+                         measured_margin)
 
 pytestmark = pytest.mark.gpu
 
@@ -92,6 +93,7 @@ def test_cfg1_full_run_lockstep(env):
                 assert np.array_equal(batch["idx"].cpu().numpy(), oidx)
                 assert np.array_equal(batch["ver"].cpu().numpy(), orec.view(np.int32)[:, 11])
                 assert int((version - batch["ver"]).max().item()) <= f["staleness_bound"]
+    tally.report("cfg1 lock-step")
     assert tally.ambiguous_done <= 0.001 * tally.total + 2
     gs, os_ = ctx.stats(), o.stats()
     for key in ("produced", "consumed", "dropped_stale", "starved_calls", "actor_steps", "learner_steps",
@@ -118,6 +120,7 @@ def test_small_env_lockstep_ragged_shapes(env, kind, D, A, H, N, steps):
         scale = float(np.sqrt(np.mean(r["o_logits"].astype(np.float64) ** 2)))
         compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=kind, tally=tally, act_exact=(kind != 1),
                           act_margin_scale=8 * RTOL_FP32 * scale)
+    tally.report("small env lock-step kind %d H %d N %d" % (kind, H, N))
     assert tally.ambiguous_done <= 0.002 * tally.total + 2 and tally.ambiguous_act <= 0.002 * tally.total + 2
     assert ctx.stats()["episodes_finished"] > 0
 
@@ -136,11 +139,12 @@ def test_lingauss_lockstep(env, wd):
             ctx.publish_weights(blob)
             o.publish(blob)
         r = lockstep_step(ctx, o, torch, rtol=rtol, env_kind=2, tally=tally, logits_exact=(wd == 0))
-        scale = float(np.sqrt(np.mean(r["o_logits"].astype(np.float64) ** 2)))
         compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=2, tally=tally, act_exact=(wd == 0),
-                          act_margin_scale=8 * rtol * scale)
+                          act_margin_scale=measured_margin(r["g_logits"], r["o_logits"]))
     st = ctx.stats()
+    amb_act, _ = tally.report("LinGauss lock-step weight_dtype %d" % wd)
     assert st["episodes_finished"] > 0 and tally.ambiguous_done <= 0.01 * tally.total + 2
+    assert amb_act <= 0.08
 
 
 def test_lingauss_literal_constants_terminate_almost_every_step(env):
@@ -240,15 +244,19 @@ def test_td_error_parity(env, kind, D, A, H, B):
     f = _small(env_kind=kind, obs_dim=D, n_actions=A, hidden=H, n_envs=32, replay_capacity=32 * 16, minibatch=B,
                warmup=32, staleness_bound=50, target_sync_interval=2, max_episode_steps=11, lg_done_norm=9.0)
     ctx, o = make_pair(orc, binding, **f)
+    fresh = orc.Oracle(**dict(f, target_sync_interval=1))     # a learner whose target network never lags
     tally = Tally()
+    lagging_versions = 0
     for v in range(1, 6):
         blob = blob_for(f, v)
         ctx.publish_weights(blob)
         o.publish(blob)
+        fresh.publish(blob)
         for _ in range(4):
             lockstep_step(ctx, o, torch, rtol=RTOL_FP32, env_kind=kind, tally=tally)
         _, batch = ctx.replay_sample()
         o.sample()
+        fresh.set_counters(0, 0, v)                            # one learner step per version, as on the other two
         out = ctx.td_error(batch)
         # the oracle evaluates the batch the GPU gathered
         rec = np.zeros((B, 2 * D + 4), np.float32)
@@ -266,8 +274,21 @@ def test_td_error_parity(env, kind, D, A, H, B):
         g_h = out["huber"].cpu().numpy().astype(np.float64)
         assert np.all(np.abs(g_h - hub) <= 2 * RTOL_FP32 * (hub + terms * np.maximum(1.0, np.abs(td))))
         assert abs(float(out["loss"].item()) - loss) <= 2 * RTOL_FP32 * (abs(loss) + float(terms.mean()))
-    # the target network really lags: with target_sync_interval = 2 it is not the newest blob every time
-    assert not np.array_equal(o.online_blob, o.target_blob) or True
+        # The target network lags: refreshed on the first publish and then after every second learner step, it is the
+        # newest parameters at versions 1, 3, 5 and one version behind at 2 and 4.  There the GPU's TD errors must
+        # follow the lagging target, i.e. differ from those of a learner whose target is always the newest.
+        assert np.array_equal(o.online_blob, blob)
+        if v in (2, 4):
+            assert np.array_equal(o.target_blob, blob_for(f, v - 1)) and not np.array_equal(o.target_blob, o.online_blob)
+            _, td_fresh, _, _, _, _ = fresh.td(rec)
+            moved = np.abs(td_fresh - td) > 100 * RTOL_FP32 * (np.abs(td) + terms)
+            live = rec.view(np.int32)[:, 2 * D + 2] == 0       # a done row has no bootstrap term, so no target at all
+            assert moved[live].mean() > 0.9
+            assert np.all(np.abs(g_td - td_fresh)[moved] > RTOL_FP32 * (np.abs(td) + terms)[moved])
+            lagging_versions += 1
+        else:
+            assert np.array_equal(o.target_blob, blob)
+    assert lagging_versions == 2
 
 
 def test_gae_parity_and_closed_forms(env):
@@ -410,10 +431,13 @@ def test_bf16_tensor_core_actor_lockstep(env, D, H, A, N):
             ctx.publish_weights(blob)
             o.publish(blob)
         r = lockstep_step(ctx, o, torch, rtol=2e-2, env_kind=2, tally=tally, logits_exact=False)
-        scale = float(np.sqrt(np.mean(r["o_logits"].astype(np.float64) ** 2)))
-        compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=2, tally=tally, act_exact=False, act_margin_scale=8 * 2e-2 * scale)
+        # outputs are held to 2e-2; the action must equal the oracle's wherever the oracle's top-2 gap exceeds twice the
+        # deviation actually measured on this step (then no rounding can change the maximum)
+        compare_ring_step(r, o, rtol=RTOL_FP32, env_kind=2, tally=tally, act_exact=False,
+                          act_margin_scale=measured_margin(r["g_logits"], r["o_logits"]))
     assert ctx.stats()["device_error"] == 0 and ctx.stats()["episodes_finished"] > 0
-    assert tally.ambiguous_act < 0.6 * tally.total          # the margin rule must still bind most decisions
+    amb_act, _ = tally.report("BF16 tensor-core actor D %d H %d A %d N %d" % (D, H, A, N))
+    assert amb_act <= 0.08                                  # a few per cent at most: the rule binds nearly every decision
     # TD error through the same tensor-core forward
     _, batch = ctx.replay_sample()
     out = ctx.td_error(batch)

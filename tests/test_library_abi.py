@@ -21,7 +21,7 @@ def lib():
 
 def test_every_declared_symbol_is_exported(lib):
     header = open(os.path.join(ROOT, "include", "tj.h")).read()
-    declared = set(re.findall(r"^(?:int|const char \*)\s*(tj_[a-z_]+)\s*\(", header, re.M))
+    declared = set(re.findall(r"^(?:int|const char \*)\s*(tj_[a-z0-9_]+)\s*\(", header, re.M))
     assert declared == set(b.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name

@@ -59,3 +59,14 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["n_gpus"] == 2
+
+
+def test_gpus_flag_must_agree_with_the_launcher():
+    """`--gpus N` under a launcher that started another number of ranks is an error, not a silent single-GPU run."""
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "1"], env=env,
+                         capture_output=True, text=True, timeout=120)
+    assert out.returncode != 0 and "--gpus 4" in (out.stderr + out.stdout) and "2 ranks" in (out.stderr + out.stdout)
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "1"], env=env, capture_output=True,
+                         text=True, timeout=120)
+    assert out.returncode != 0 and "2 ranks" in (out.stderr + out.stdout)
