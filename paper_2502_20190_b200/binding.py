@@ -14,7 +14,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtj.so")
+# TJ_LIB_PATH names another build of the library (same ABI), e.g. one compiled with different options
+LIB_PATH = os.environ.get("TJ_LIB_PATH") or os.path.join(_HERE, "libtj.so")
 
 TJ_OK, TJ_ERR_INVALID_ARG, TJ_ERR_CONFIG, TJ_ERR_WORKSPACE, TJ_ERR_CUDA = 0, -1, -2, -3, -4
 TJ_ERR_NO_WEIGHTS, TJ_ERR_WARMUP, TJ_ERR_STARVED, TJ_ERR_STALE_SEGMENT, TJ_ERR_TIMEOUT, TJ_ERR_UNSUPPORTED = (

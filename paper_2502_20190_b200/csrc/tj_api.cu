@@ -144,6 +144,8 @@ size_t carve(tj_ctx* x, void* base) {
     x->wtc_pipe[0] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
     x->wtc_pipe[1] = cv.take<uint16_t>(tc_weight_elems(D, c.hidden));
     x->z_scratch = cv.take<float>(tc_pipelined_scratch_floats());
+    x->lgA16 = cv.take<uint16_t>(tc_pipelined_env_halfs());
+    x->lgB_t = cv.take<float>((size_t)c.n_actions * D);
   }
   return (cv.off + kAlign - 1) & ~(kAlign - 1);
 }
@@ -277,6 +279,19 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
       return bail(e, "copy B to its place");
     if (x->use_tc_fused && (e = launch_pack_env_matrix(stage, x->lgA_hi, x->lgA_lo, D, x->stream)) != cudaSuccess)
       return bail(e, "tile env matrix");
+    if (x->use_tc_pipelined) {
+      // FP16 split of the matrix: a power-of-two scale puts its largest entry in [1024, 2048), well inside FP16's range,
+      // so that the low parts of all but the tiniest entries are normal numbers
+      float amax = 0.f;
+      for (size_t i = 0; i < (size_t)D * D; ++i) amax = std::max(amax, std::fabs(cfg->host_lg_A[i]));
+      int ea = 0;
+      if (amax > 0.f && std::isfinite(amax)) ea = 10 - (int)std::floor(std::log2((double)amax));
+      ea = std::min(std::max(ea, -24), 24);
+      const float scale = std::ldexp(1.0f, ea);
+      x->z_to_t = 2.88539008177792681472f / (tc_pipelined_state_scale() * scale);
+      if ((e = launch_pack_pipelined_env(stage, stage + (size_t)D * D, scale, A, x->lgA16, x->lgB_t, x->stream)) != cudaSuccess)
+        return bail(e, "split env matrix");
+    }
     if ((e = cudaStreamSynchronize(x->stream)) != cudaSuccess) return bail(e, "sync after LinGauss set-up");
   }
   const uint2 seed = make_uint2((uint32_t)cfg->seed, (uint32_t)(cfg->seed >> 32));
@@ -398,6 +413,8 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
         if (x->use_tc_pipelined) {
           t.wtc = x->wtc_pipe[x->active];
           ev.z_scratch = x->z_scratch;
+          ev.slot0 = ev.cursor % (unsigned long long)c.replay_capacity;
+          ev.lgA16 = x->lgA16; ev.lgB_t = x->lgB_t; ev.z_to_t = x->z_to_t;
           e = launch_actor_tc_pipelined(t, x->sm_count, x->stream);
         } else {
           e = launch_tc_mlp(t, x->sm_count, x->stream);

@@ -160,6 +160,10 @@ struct TcEnvParams {
   float noise_std, done_norm;
   DevStats* stats;
   float* z_scratch;                  // pipelined actor: per thread block two tiles of z, [2][32][128][4] floats
+  unsigned long long slot0;          // pipelined actor: cursor mod C, the ring slot of env 0 in this step
+  const uint16_t* lgA16;             // pipelined actor: scaled env matrix as FP16 high / low chunks
+  const float* lgB_t;                // pipelined actor: B [A][D] times 2 log2(e)
+  float z_to_t;                      // pipelined actor: accumulator of the scaled product -> 2 log2(e) * z
 };
 
 struct TcMlpParams {
@@ -183,6 +187,10 @@ bool tc_pipelined_supported(int D, int H, int A);
 cudaError_t launch_pack_pipelined_weights(const float* blob, uint16_t* dst, int D, int H, int A, cudaStream_t s);
 cudaError_t launch_actor_tc_pipelined(const TcMlpParams& p, int sm_count, cudaStream_t s);
 size_t tc_pipelined_scratch_floats();   // z scratch for the largest grid the launcher uses
+size_t tc_pipelined_env_halfs();        // FP16 high / low chunks of the env matrix
+float tc_pipelined_state_scale();       // power of two the state is multiplied by before its FP16 split
+cudaError_t launch_pack_pipelined_env(const float* A, const float* B, float scale, int n_actions, uint16_t* dst, float* b_t,
+                                      cudaStream_t s);
 cudaError_t launch_td_from_q(const float* q_online, const float* q_target, int n, int A, const int* act, const float* rew,
                              const int* done, float gamma, float kappa, float* td_out, float* huber_out, float* partial,
                              cudaStream_t s);
@@ -258,6 +266,9 @@ struct tj_ctx {
   bool use_tc_pipelined;
   uint16_t* wtc_pipe[2];   // weight chunks in the pipelined actor's order, double buffered like wtc
   float* z_scratch;
+  uint16_t* lgA16;      // pipelined actor: env matrix, FP16 high / low chunks, scaled by lg_scale
+  float* lgB_t;         // pipelined actor: B times 2 log2(e)
+  float z_to_t;
   uint32_t *lgA_hi, *lgA_lo;
   float* tdq[2];       // [kMaxTcTdRows][A] online / target outputs
   float *seg_obs, *seg_rew, *seg_logp, *seg_val;

@@ -2,24 +2,28 @@
 // network, action selection, z = A s, env epilogue, record and reset in one persistent kernel whose roles overlap.
 //
 // A thread block owns 128 rows (envs) per tile, one row per TMEM lane, and walks tiles persistently.  Roles:
-//   warp 0, one lane    producer: streams operand chunks (32 KB of weights, 16 KB of the env matrix) from L2 into a ring of
-//                       two 32 KB slots
+//   warp 0, one lane    producer: streams 32 KB operand chunks (weights, the env matrix) from L2 into a ring of two slots
 //   warp 1, one lane    MMA issuer (tcgen05.mma, M = 128, N = 128 per hidden block)
 //   warps 4-11          network warps (two threads per row): state rows -> BF16 (layer-1 operand); per 128-neuron block of a
-//                       hidden layer:
-//                       accumulator -> bias, ReLU, BF16 -> next layer's operand; z -> a scratch tile in global memory
-//   warps 12-19         env warps: the TF32 parts of the next tile's state rows and the record's observation; take the head
+//                       hidden layer: accumulator -> bias, ReLU, BF16 -> next layer's operand; z -> a scratch tile in global
+//                       memory
+//   warps 12-19         env warps: the FP16 parts of the next tile's state rows and the record's observation; take the head
 //                       outputs out of TMEM, select the action, read z back and finish the step (tanh, Philox noise, reward,
 //                       done, record, reset or new state, counters), eight rows x four 16-byte pieces per warp instruction
 // The env warps work on tile i while the network warps and the tensor pipe are already on tile i + 1.
 //
 // Per tile the tensor pipe runs ten accumulator blocks that alternate between two 128-column accumulators:
-//   layer 1 (4 blocks, A operand = X in shared memory), z (one block, TF32), layer 2 (4 blocks, A operand = h1 in tensor
+//   layer 1 (4 blocks, A operand = X in shared memory), z (one block), layer 2 (4 blocks, A operand = h1 in tensor
 //   memory), head (16 columns).  The epilogue of one block overlaps the MMAs of the next.
+// z = A s keeps FP32 accuracy on the FP16 tensor path: state and matrix are each split into a high and a low FP16 part
+// (power-of-two scaled so the low parts stay normal numbers), z = hi*hi + lo*hi + hi*lo with FP32 accumulation: 24
+// instructions of K = 16, relative error about 2^-22 per term (the dropped lo*lo term and the low parts' rounding).
 // Tensor memory (512 columns): [0, H/2) h1 as packed BF16 pairs; [256, 384) and [384, 512) the two accumulators.
-// Shared memory: X (BF16 state tile, 32 KB) | U (128 KB: TF32 high and low parts of the state tile until z is done, then
-// h2, the head's A operand) | ring (64 KB) | barriers.
+// Shared memory: X (BF16 state tile, 32 KB) | U (128 KB: the FP16 high and low parts of the state tile in its first 64 KB
+// until z is done, then h2, the head's A operand) | ring (64 KB) | barriers.
 // Every wait is bounded: on a timeout the block raises an abort flag, records an error, frees its TMEM and leaves.
+#include <cuda_fp16.h>
+
 #include "tj_internal.h"
 #include "tj_tc.cuh"
 
@@ -30,12 +34,11 @@ namespace {
 constexpr int PA_M = 128;                  // rows per tile
 constexpr int PA_D = 128;                  // observation / state width this kernel is built for
 constexpr int PA_NB = 128;                 // neurons per accumulator block
-constexpr int PA_KC = 128;                 // K elements per weight chunk (128 x 128 BF16 = 32 KB)
-constexpr int PA_W_BYTES = PA_NB * PA_KC * 2;              // bytes of a hidden-layer weight chunk
-constexpr int PA_Z_BYTES = 16384;                          // bytes of an env-matrix chunk (128 x 32 TF32)
-constexpr int PA_STAGE_BYTES = PA_W_BYTES > PA_Z_BYTES ? PA_W_BYTES : PA_Z_BYTES;
+constexpr int PA_KC = 128;                 // K elements per weight chunk (128 x 128 x 2 bytes = 32 KB)
+constexpr int PA_W_BYTES = PA_NB * PA_KC * 2;              // bytes of a hidden-layer weight chunk, and of one env-matrix part
+constexpr int PA_STAGE_BYTES = PA_W_BYTES;
 constexpr int PA_STAGES = 65536 / PA_STAGE_BYTES;
-constexpr uint32_t PA_B_SBO = (PA_KC / 8) * 128;           // bytes between 8-row groups of a weight chunk
+constexpr uint32_t PA_B_SBO = (PA_KC / 8) * 128;           // bytes between 8-row groups of a chunk
 constexpr int PA_X_BYTES = PA_M * PA_D * 2;
 constexpr int PA_U_BYTES = 131072;
 constexpr int PA_THREADS = 640;            // warps 0-3: producer, MMA issuer, two idle; 4-11 network; 12-19 env
@@ -43,11 +46,12 @@ constexpr int PA_GROUP_WARPS = 8;          // warps of the network group and of 
 constexpr uint32_t PA_COL_HB = 0, PA_COL_ACC0 = 256, PA_COL_ACC1 = 384;
 constexpr int PA_N3 = 16;                  // head width on the tensor cores
 constexpr int PA_MAX_GRID = 192;           // thread blocks the z scratch is sized for
+constexpr float PA_S_SCALE = 256.0f;       // state values are split after this scaling (|s| < 1.2: far below FP16's range)
 
 struct PaSmem {
   uint64_t full[PA_STAGES], empty[PA_STAGES];
   uint64_t x_ready;        // network -> MMA: X holds the tile's BF16 rows
-  uint64_t u_ready;        // env -> MMA: U holds the tile's TF32 high / low parts
+  uint64_t u_ready;        // env -> MMA: U holds the tile's FP16 high / low parts
   uint64_t acc_full[2];    // MMA -> network: an accumulator block is complete
   uint64_t acc_empty[2];   // network -> MMA: it has been drained (and its result stored)
   uint64_t head_full;      // MMA -> env and network: head outputs complete; U may be rewritten
@@ -75,7 +79,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
   // Thread blocks walk the neuron blocks of a layer in rotated order, so that at any moment they stream different
   // parts of the weights from L2 (the arithmetic per neuron is unchanged)
   const int rot = (int)(blockIdx.x % (unsigned)n_hb);
-  const int n_kc2 = H / PA_KC;           // K chunks of a layer-2 block (a layer-1 block has PA_D / PA_KC)
+  const int n_kc2 = H / PA_KC;           // K chunks of a layer-2 block (a layer-1 block has one)
 
   if (tid == 0) {
     for (int s = 0; s < PA_STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
@@ -104,24 +108,24 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
   const TcEnvParams& ev = p.env;
 
   if (warp < 4) {
-    // registers: 640 threads x 96 at launch = 61,440; 128 x 40 + 256 x 96 + 256 x 120 = 60,416 after the two changes
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    // registers: 640 threads x 96 at launch = 61,440; 128 x 64 + 256 x 96 + 256 x 112 = 61,440 after the two changes.  The
+    // issuing lane's loop is the pace-maker of the whole block: it must not spill, so its warpgroup keeps 64 registers.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     if (warp == 0 && lane == 0) {
       // ---------------------------------------------------------------- producer
-      // order per tile (the order the MMA issuer consumes): layer 1 (one chunk per block), env matrix (4 high, 4 low),
-      // layer 2 (H/128 chunks per block), head
+      // order per tile (the order the MMA issuer consumes): layer 1 (one chunk per block), env matrix (high part, low
+      // part), layer 2 (H/128 chunks per block), head
       uint32_t it = 0;
       const uint32_t head_bytes = (uint32_t)PA_N3 * H * 2;
-      const int n1 = n_hb * (PA_D / PA_KC), n2 = n_hb * n_kc2;
+      const int n1 = n_hb, n2 = n_hb * n_kc2;
       for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
-        for (int c = 0; c < n1 + 8 + n2 + 1; ++c, ++it) {
+        for (int c = 0; c < n1 + 2 + n2 + 1; ++c, ++it) {
           const uint8_t* src;
           uint32_t bytes = PA_W_BYTES;
-          constexpr int cpb1 = PA_D / PA_KC;
-          if (c < n1) src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(((c / cpb1 + rot) % n_hb) * cpb1 + c % cpb1) * PA_W_BYTES;
-          else if (c < n1 + 8) { src = reinterpret_cast<const uint8_t*>(c - n1 < 4 ? ev.lgA_hi : ev.lgA_lo) + (size_t)((c - n1) & 3) * PA_Z_BYTES; bytes = PA_Z_BYTES; }
-          else if (c < n1 + 8 + n2) {
-            const int idx = c - n1 - 8;
+          if (c < n1) src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)((c + rot) % n_hb) * PA_W_BYTES;
+          else if (c < n1 + 2) src = reinterpret_cast<const uint8_t*>(ev.lgA16) + (size_t)(c - n1) * PA_W_BYTES;
+          else if (c < n1 + 2 + n2) {
+            const int idx = c - n1 - 2;
             src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(n1 + ((idx / n_kc2 + rot) % n_hb) * n_kc2 + idx % n_kc2) * PA_W_BYTES;
           }
           else { src = reinterpret_cast<const uint8_t*>(p.wtc) + (size_t)(n1 + n2) * PA_W_BYTES; bytes = head_bytes; }
@@ -137,8 +141,13 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       // writes accumulator u & 1 (the count per tile is even, so the pattern repeats).  The network warps drain every use
       // but the head (acc_empty), the env warps take the head (env_taken).
       uint32_t it = 0, tiles = 0, nwait0 = 0, nwait1 = 0;
-      const uint32_t idesc_h = make_idesc(PA_NB), idesc16 = make_idesc(PA_N3), idesc_z = make_idesc_tf32(D);
-      const uint32_t x_addr = smem_addr(xbuf), u_addr = smem_addr(ubuf);
+      const uint32_t idesc_h = make_idesc(PA_NB), idesc16 = make_idesc(PA_N3), idesc_z = make_idesc_f16(D);
+      // descriptors as (low, high) words: the high word is fixed per operand shape, the low word steps by 16 per K = 16
+      const uint32_t x_lo = desc_lo(smem_addr(xbuf), 128u), u_lo = desc_lo(smem_addr(ubuf), 128u);
+      const uint32_t ulo_lo = desc_lo(smem_addr(ubuf) + (uint32_t)PA_X_BYTES, 128u);
+      const uint32_t ring_lo = desc_lo(smem_addr(ring), 128u);
+      const uint32_t hi_k128 = desc_hi(2048u);                       // operands 128 K-elements wide (X, U, weight chunks)
+      const uint32_t hi_head = desc_hi((uint32_t)(H / 8) * 128u);    // operands H K-elements wide (h2, head weights)
       // before use u may overwrite its accumulator, the previous use of that accumulator must have been read out
       auto acquire = [&](int u) -> bool {
         if (u == 0) return true;      // accumulator 0: its last drain was awaited before the previous tile's head
@@ -147,49 +156,37 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       };
       for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tiles) {
         if (!tc_wait(&ctl->x_ready, tiles & 1, abort_flag)) goto done;
-        // layer 1: per 128-neuron block PA_D / PA_KC chunks; A operand = X in shared memory
-        for (int b = 0; b < n_hb; ++b) {
+        // layer 1: one chunk per 128-neuron block; A operand = X in shared memory
+        for (int b = 0; b < n_hb; ++b, ++it) {
           const int u = b;
           if (!acquire(u)) goto done;
-          tc_fence_after();
           const uint32_t acc = tmem + ((u & 1) ? PA_COL_ACC1 : PA_COL_ACC0);
-          for (int c = 0; c < PA_D / PA_KC; ++c, ++it) {
-            const int s = it % PA_STAGES;
-            if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
-            const uint32_t b_base = smem_addr(ring + (size_t)s * PA_STAGE_BYTES);
-            const uint32_t a_base = x_addr + (uint32_t)(c * (PA_KC / 8)) * 128u;
+          const uint32_t s = it % PA_STAGES;
+          if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
+          tc_fence_after();
+          const uint32_t b_lo = ring_lo + s * (PA_STAGE_BYTES / 16);
 #pragma unroll
-            for (int j = 0; j < PA_KC / 16; ++j)
-              umma_bf16(acc, make_desc(a_base + j * 256u, 128u, 2048u), make_desc(b_base + j * 256u, 128u, PA_B_SBO), idesc_h,
-                        (c | j) != 0);
-            umma_commit(&ctl->empty[s]);
-          }
+          for (int j = 0; j < PA_KC / 16; ++j) umma_ss(acc, x_lo + j * 16u, hi_k128, b_lo + j * 16u, hi_k128, idesc_h, j != 0);
+          umma_commit(&ctl->empty[s]);
           umma_commit((u & 1) ? &ctl->acc_full[1] : &ctl->acc_full[0]);
         }
-        // z = A s as three TF32 products: (s_hi, A_hi), (s_lo, A_hi), (s_hi, A_lo); K = 8 per instruction
+        // z = A s from the FP16 parts: (s_hi, A_hi) + (s_lo, A_hi) with the first chunk, (s_hi, A_lo) with the second
         {
           const int u = n_hb;
           if (!tc_wait(&ctl->u_ready, tiles & 1, abort_flag)) goto done;
           if (!acquire(u)) goto done;
-          tc_fence_after();
-          const uint32_t a_sbo = (uint32_t)(D / 4) * 128u, b_sbo = (uint32_t)(32 / 4) * 128u, lo_off = (uint32_t)PA_M * D * 4;
           const uint32_t acc = tmem + ((u & 1) ? PA_COL_ACC1 : PA_COL_ACC0);
-          for (int half = 0; half < 2; ++half) {
-            for (int kc = 0; kc < 4; ++kc, ++it) {
-              const int s = it % PA_STAGES;
-              if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
-              const uint32_t b_base = smem_addr(ring + (size_t)s * PA_STAGE_BYTES);
-              const uint32_t a_base = u_addr + (uint32_t)(kc * 8) * 128u;
+          for (int part = 0; part < 2; ++part, ++it) {
+            const uint32_t s = it % PA_STAGES;
+            if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
+            tc_fence_after();
+            const uint32_t b_lo = ring_lo + s * (PA_STAGE_BYTES / 16);
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                umma_tf32(acc, make_desc(a_base + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, b_sbo), idesc_z,
-                          (half | kc | j) != 0);
-                if (half == 0)
-                  umma_tf32(acc, make_desc(a_base + lo_off + j * 256u, 128u, a_sbo), make_desc(b_base + j * 256u, 128u, b_sbo),
-                            idesc_z, true);
-              }
-              umma_commit(&ctl->empty[s]);
+            for (int j = 0; j < D / 16; ++j) {
+              umma_ss(acc, u_lo + j * 16u, hi_k128, b_lo + j * 16u, hi_k128, idesc_z, (part | j) != 0);
+              if (part == 0) umma_ss(acc, ulo_lo + j * 16u, hi_k128, b_lo + j * 16u, hi_k128, idesc_z, 1u);
             }
+            umma_commit(&ctl->empty[s]);
           }
           umma_commit((u & 1) ? &ctl->acc_full[1] : &ctl->acc_full[0]);
         }
@@ -198,16 +195,15 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         for (int b = 0; b < n_hb; ++b) {
           const int u = n_hb + 1 + b;
           if (!acquire(u)) goto done;
-          tc_fence_after();
           const uint32_t acc = tmem + ((u & 1) ? PA_COL_ACC1 : PA_COL_ACC0);
           for (int c = 0; c < n_kc2; ++c, ++it) {
-            const int s = it % PA_STAGES;
+            const uint32_t s = it % PA_STAGES;
             if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
-            const uint32_t b_base = smem_addr(ring + (size_t)s * PA_STAGE_BYTES);
+            tc_fence_after();
+            const uint32_t b_lo = ring_lo + s * (PA_STAGE_BYTES / 16);
             const uint32_t a_col = tmem + PA_COL_HB + (uint32_t)(c * (PA_KC / 2));
 #pragma unroll
-            for (int j = 0; j < PA_KC / 16; ++j)
-              umma_bf16_ts(acc, a_col + (uint32_t)(j * 8), make_desc(b_base + j * 256u, 128u, PA_B_SBO), idesc_h, (c | j) != 0);
+            for (int j = 0; j < PA_KC / 16; ++j) umma_ts(acc, a_col + (uint32_t)(j * 8), b_lo + j * 16u, hi_k128, idesc_h, (c | j) != 0);
             umma_commit(&ctl->empty[s]);
           }
           umma_commit((u & 1) ? &ctl->acc_full[1] : &ctl->acc_full[0]);
@@ -216,14 +212,11 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         {
           if (!acquire(2 * n_hb + 1)) goto done;
           if (!tc_wait(&ctl->acc_empty[0], (nwait0++) & 1, abort_flag)) goto done;
-          tc_fence_after();
-          const int s = it % PA_STAGES;
+          const uint32_t s = it % PA_STAGES;
           if (!tc_wait(&ctl->full[s], (it / PA_STAGES) & 1, abort_flag)) goto done;
-          const uint32_t b_base = smem_addr(ring + (size_t)s * PA_STAGE_BYTES);
-          const uint32_t sbo = (uint32_t)(H / 8) * 128u;
-          for (int j = 0; j < H / 16; ++j)
-            umma_bf16(tmem + PA_COL_ACC1, make_desc(u_addr + j * 256u, 128u, sbo), make_desc(b_base + j * 256u, 128u, sbo), idesc16,
-                      j != 0);
+          tc_fence_after();
+          const uint32_t b_lo = ring_lo + s * (PA_STAGE_BYTES / 16);
+          for (int j = 0; j < H / 16; ++j) umma_ss(tmem + PA_COL_ACC1, u_lo + j * 16u, hi_head, b_lo + j * 16u, hi_head, idesc16, j != 0);
           umma_commit(&ctl->empty[s]);
           umma_commit(&ctl->head_full);
           ++it;
@@ -249,7 +242,8 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         const float* xr = p.x + (size_t)(row < p.n ? row : 0) * D;
         float4 v[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = row < p.n ? __ldg(reinterpret_cast<const float4*>(xr + (c_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < 8; ++i)
+          v[i] = row < p.n ? __ldg(reinterpret_cast<const float4*>(xr + (c_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
         uint8_t* dx = xbuf + ((size_t)(rr >> 3) * (D / 8)) * 128 + (rr & 7) * 16;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -311,11 +305,10 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           uint32_t o[16];
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
+            float f0 = __uint_as_float(v[hh * 32 + 4 * j4 + 0]), f1 = __uint_as_float(v[hh * 32 + 4 * j4 + 1]);
+            float f2 = __uint_as_float(v[hh * 32 + 4 * j4 + 2]), f3 = __uint_as_float(v[hh * 32 + 4 * j4 + 3]);
             const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + c0 + hh * 32 + 4 * j4));
-            const float f0 = __uint_as_float(v[hh * 32 + 4 * j4 + 0]) + bb.x;
-            const float f1 = __uint_as_float(v[hh * 32 + 4 * j4 + 1]) + bb.y;
-            const float f2 = __uint_as_float(v[hh * 32 + 4 * j4 + 2]) + bb.z;
-            const float f3 = __uint_as_float(v[hh * 32 + 4 * j4 + 3]) + bb.w;
+            f0 += bb.x; f1 += bb.y; f2 += bb.z; f3 += bb.w;
             o[2 * j4] = pack_bf16x2_relu(f0, f1);
             o[2 * j4 + 1] = pack_bf16x2_relu(f2, f3);
           }
@@ -336,11 +329,11 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
     }
   } else {
     // ------------------------------------------------------------------ env warps
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 120;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 112;");
     const int ew = warp - 12;                      // 0..7; the first four also read the head outputs (one TMEM quarter each)
     const int e_r8 = lane >> 2, e_kq = lane & 3;   // env step: eight rows x four 16-byte pieces per warp instruction
     uint32_t tiles = 0;
-    // TF32 high / low parts of a tile's rows -> U (A operand of z = A s); the FP32 row is the record's observation
+    // FP16 high / low parts of a tile's scaled rows -> U (A operand of z = A s); the FP32 row is the record's observation
     auto convert_u = [&](int tile) {
 #pragma unroll
       for (int g = 0; g < 2; ++g) {
@@ -350,22 +343,25 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         const float* xr = p.x + (size_t)(live ? row : 0) * D;
         float4 v[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = live ? __ldg(reinterpret_cast<const float4*>(xr + (e_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        uint8_t* dhi = ubuf + ((size_t)(rr >> 3) * (D / 4)) * 128 + (rr & 7) * 16;
-        uint8_t* dlo = dhi + (size_t)PA_M * D * 4;
-        const unsigned long long slot = (ev.cursor + (unsigned long long)(live ? row : 0)) % (unsigned long long)ev.C;
-        float* rec = ev.ring + slot * ev.rec_words;
+        for (int i = 0; i < 8; ++i)
+          v[i] = live ? __ldg(reinterpret_cast<const float4*>(xr + (e_kq + 4 * i) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        uint8_t* dhi = ubuf + ((size_t)(rr >> 3) * (D / 8)) * 128 + (rr & 7) * 16;
+        uint8_t* dlo = dhi + PA_X_BYTES;
+        float* rec = ev.ring + (ev.slot0 + (unsigned long long)(live ? row : 0)) * ev.rec_words;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int k4 = e_kq + 4 * i;
           const float4 sv = v[i];
-          float4 hi, lo;
-          hi.x = __uint_as_float(__float_as_uint(sv.x) & 0xFFFFE000u); lo.x = sv.x - hi.x;
-          hi.y = __uint_as_float(__float_as_uint(sv.y) & 0xFFFFE000u); lo.y = sv.y - hi.y;
-          hi.z = __uint_as_float(__float_as_uint(sv.z) & 0xFFFFE000u); lo.z = sv.z - hi.z;
-          hi.w = __uint_as_float(__float_as_uint(sv.w) & 0xFFFFE000u); lo.w = sv.w - hi.w;
-          *reinterpret_cast<float4*>(dhi + (size_t)k4 * 128) = hi;
-          *reinterpret_cast<float4*>(dlo + (size_t)k4 * 128) = lo;
+          // high part: the scaled value cut to 11 significant bits (exact in FP16); low part: the exact remainder, rounded
+          float4 s4, hi, lo;
+          s4.x = sv.x * PA_S_SCALE; s4.y = sv.y * PA_S_SCALE; s4.z = sv.z * PA_S_SCALE; s4.w = sv.w * PA_S_SCALE;
+          hi.x = __uint_as_float(__float_as_uint(s4.x) & 0xFFFFE000u); lo.x = s4.x - hi.x;
+          hi.y = __uint_as_float(__float_as_uint(s4.y) & 0xFFFFE000u); lo.y = s4.y - hi.y;
+          hi.z = __uint_as_float(__float_as_uint(s4.z) & 0xFFFFE000u); lo.z = s4.z - hi.z;
+          hi.w = __uint_as_float(__float_as_uint(s4.w) & 0xFFFFE000u); lo.w = s4.w - hi.w;
+          const size_t off = (size_t)(k4 >> 1) * 128 + (k4 & 1) * 8;
+          *reinterpret_cast<uint2*>(dhi + off) = make_uint2(pack_f16x2(hi.x, hi.y), pack_f16x2(hi.z, hi.w));
+          *reinterpret_cast<uint2*>(dlo + off) = make_uint2(pack_f16x2(lo.x, lo.y), pack_f16x2(lo.z, lo.w));
           if (live) *reinterpret_cast<float4*>(rec + k4 * 4) = sv;
         }
       }
@@ -375,6 +371,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
     if ((int)blockIdx.x < n_tiles) convert_u(blockIdx.x);
     unsigned long long n_episodes = 0;
     double ret_sum = 0.0;
+    const float zc = ev.z_to_t;                    // accumulator -> 2 log2(e) * z
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tiles) {
       if (ew < 4) {
         const int r = ew * 32 + lane;              // row of the tile = TMEM lane
@@ -408,7 +405,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         mbar_arrive_warp(&ctl->env_taken);         // this warp has finished the previous tile
         if (!tc_wait_elect(&ctl->head_full, tiles & 1, abort_flag)) goto done;
       }
-      // the head of this tile is complete, so U is free: the next tile's TF32 parts go in before this tile's env step
+      // the head of this tile is complete, so U is free: the next tile's FP16 parts go in before this tile's env step
       if (tile + (int)gridDim.x < n_tiles) convert_u(tile + (int)gridDim.x);
       if (!tc_wait_elect(&ctl->act_ready, tiles & 1, abort_flag)) goto done;
       // z was stored long before the head finished; the wait orders the loads below after those stores
@@ -420,11 +417,10 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         const long long row = (long long)tile * PA_M + rr;
         const bool live = row < p.n;
         const int action = ctl->act[tiles & 1][rr];
-        const unsigned long long slot = (ev.cursor + (unsigned long long)(live ? row : 0)) % (unsigned long long)ev.C;
-        float* rec = ev.ring + slot * ev.rec_words;
+        float* rec = ev.ring + (ev.slot0 + (unsigned long long)(live ? row : 0)) * ev.rec_words;
         const int ep0 = live ? ev.ep_step[row] : 0;
         const float ret0 = live ? ev.ep_return[row] : 0.f;
-        const float* Ba = ev.lgB + (size_t)action * D;
+        const float* Ba = ev.lgB_t + (size_t)action * D;     // B[a] times 2 log2(e)
         // s' = tanh(z + B[a]) + noise; piece k4 = components 4 k4 .. 4 k4 + 3 = one Philox block
         float4 zz[8], sn[8];
 #pragma unroll
@@ -434,13 +430,13 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         for (int i = 0; i < 8; ++i) {
           const int k4 = e_kq + 4 * i;
           const uint4 w = stream_words(ev.seed, STREAM_NOISE, (uint32_t)k4, (uint32_t)row, ev.t);
-          const float2 z01 = box_muller_fast(w.x, w.y), z23 = box_muller_fast(w.z, w.w);
+          const float2 n01 = box_muller_scaled(w.x, w.y, ev.noise_std), n23 = box_muller_scaled(w.z, w.w, ev.noise_std);
           const float4 bb = __ldg(reinterpret_cast<const float4*>(Ba + 4 * k4));
           float4 o;
-          o.x = tanh_fast(zz[i].x + bb.x) + ev.noise_std * z01.x;
-          o.y = tanh_fast(zz[i].y + bb.y) + ev.noise_std * z01.y;
-          o.z = tanh_fast(zz[i].z + bb.z) + ev.noise_std * z23.x;
-          o.w = tanh_fast(zz[i].w + bb.w) + ev.noise_std * z23.y;
+          o.x = tanh_from_t(fmaf(zz[i].x, zc, bb.x)) + n01.x;
+          o.y = tanh_from_t(fmaf(zz[i].y, zc, bb.y)) + n01.y;
+          o.z = tanh_from_t(fmaf(zz[i].z, zc, bb.z)) + n23.x;
+          o.w = tanh_from_t(fmaf(zz[i].w, zc, bb.w)) + n23.y;
           sq = fmaf(o.x, o.x, sq); sq = fmaf(o.y, o.y, sq); sq = fmaf(o.z, o.z, sq); sq = fmaf(o.w, o.w, sq);
           sn[i] = o;
           if (live) *reinterpret_cast<float4*>(rec + D + 4 * k4) = o;
@@ -493,8 +489,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
         atomicAdd(&ev.stats->episodes, n);
         atomicAdd(&ev.stats->return_sum, rs);
       }
-      if (blockIdx.x == 0 && tid == 12 * 32)
-        ev.block_ver[(ev.cursor % (unsigned long long)ev.C) / (unsigned long long)p.n] = ev.version;
+      if (blockIdx.x == 0 && tid == 12 * 32) ev.block_ver[ev.slot0 / (unsigned long long)p.n] = ev.version;
     }
   }
 done:
@@ -508,7 +503,7 @@ done:
 }
 
 // FP32 blob -> BF16 chunks in the order the pipelined actor streams them.  Hidden layers: per 128-neuron block, chunks of
-// 128 rows x 64 columns; element (r, k) of a chunk sits at ((r/8) * 8 + k/8) * 64 + (r%8) * 8 + k%8.  Head: one chunk of
+// 128 rows x 128 columns; element (r, k) of a chunk sits at ((r/8) * 16 + k/8) * 64 + (r%8) * 8 + k%8.  Head: one chunk of
 // 16 rows x H columns, element (r, k) at ((r/8) * (H/8) + k/8) * 64 + (r%8) * 8 + k%8.
 __global__ void pack_pipelined_weights_kernel(const float* __restrict__ blob, uint16_t* __restrict__ dst, int D, int H, int A) {
   const size_t n1 = (size_t)H * D, n2 = (size_t)H * H, n3 = (size_t)PA_N3 * H;
@@ -541,6 +536,24 @@ __global__ void pack_pipelined_weights_kernel(const float* __restrict__ blob, ui
   dst[i] = (uint16_t)(u >> 16);
 }
 
+// The env matrix A [128][128] scaled by `scale` (a power of two) as two FP16 chunks, high parts then low parts, each in the
+// layout of a weight chunk (row = component of z, column = component of s); B [n_actions][128] times 2 log2(e).
+__global__ void pack_env_f16_kernel(const float* __restrict__ A, const float* __restrict__ B, float scale, int n_b,
+                                    uint16_t* __restrict__ dst, float* __restrict__ b_t) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < PA_D * PA_D) {
+    const int core = i / 64, in_core = i % 64;
+    const int rg = core / (PA_D / 8), kg = core % (PA_D / 8);
+    const int n = rg * 8 + in_core / 8, k = kg * 8 + in_core % 8;
+    const float v = A[(size_t)n * PA_D + k] * scale;
+    const __half hi = __float2half_rn(v);
+    const __half lo = __float2half_rn(v - __half2float(hi));
+    dst[i] = __half_as_ushort(hi);
+    dst[PA_D * PA_D + i] = __half_as_ushort(lo);
+  }
+  if (i < n_b) b_t[i] = B[i] * 2.88539008177792681472f;
+}
+
 }  // namespace
 
 bool tc_pipelined_supported(int D, int H, int A) {
@@ -548,10 +561,19 @@ bool tc_pipelined_supported(int D, int H, int A) {
 }
 
 size_t tc_pipelined_scratch_floats() { return (size_t)PA_MAX_GRID * 2 * PA_M * PA_D; }
+size_t tc_pipelined_env_halfs() { return (size_t)2 * PA_D * PA_D; }
+float tc_pipelined_state_scale() { return PA_S_SCALE; }
 
 cudaError_t launch_pack_pipelined_weights(const float* blob, uint16_t* dst, int D, int H, int A, cudaStream_t s) {
   const size_t n = tc_weight_elems(D, H);
   pack_pipelined_weights_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(blob, dst, D, H, A);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pack_pipelined_env(const float* A, const float* B, float scale, int n_actions, uint16_t* dst, float* b_t,
+                                      cudaStream_t s) {
+  const int n = PA_D * PA_D > n_actions * PA_D ? PA_D * PA_D : n_actions * PA_D;
+  pack_env_f16_kernel<<<(n + 255) / 256, 256, 0, s>>>(A, B, scale, n_actions * PA_D, dst, b_t);
   return cudaGetLastError();
 }
 
@@ -564,7 +586,7 @@ cudaError_t launch_actor_tc_pipelined(const TcMlpParams& p, int sm_count, cudaSt
   const int n_tiles = (p.n + PA_M - 1) / PA_M;
   int grid = n_tiles < sm_count ? n_tiles : sm_count;
   if (grid > PA_MAX_GRID) grid = PA_MAX_GRID;
-  if (!p.env.z_scratch) return cudaErrorInvalidValue;
+  if (!p.env.z_scratch || !p.env.lgA16 || !p.env.lgB_t) return cudaErrorInvalidValue;
   actor_tc_pipelined_kernel<<<grid, PA_THREADS, smem, s>>>(p);
   return cudaGetLastError();
 }
