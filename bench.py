@@ -37,7 +37,7 @@ from paper_2502_20190_b200 import synth  # noqa: E402
 NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": None}
 L2_FLUSH_BYTES = 256 << 20
 # passes of the path per bench step: about 50 ms of GPU time per step
-PATTERNS_PER_STEP = {"cfg1": 512, "cfg2": 256, "cfg3": 128, "cfg4": 8, "cfg5": 32}
+PATTERNS_PER_STEP = {"cfg1": 512, "cfg2": 256, "cfg3": 128, "cfg4": 8, "cfg5": 64}
 
 
 def load_peaks():

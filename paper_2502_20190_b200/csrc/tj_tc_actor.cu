@@ -116,6 +116,9 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
       // order per tile (the order the MMA issuer consumes): layer 1 (one chunk per block), env matrix (high part, low
       // part), layer 2 (H/128 chunks per block), head
       uint32_t it = 0;
+      // every block re-reads the same chunks each tile while state rows and records stream through L2 once: the chunks
+      // are fetched with an evict-last policy, the streams are written with evict-first stores
+      const unsigned long long keep_policy = l2_evict_last_policy();
       const uint32_t head_bytes = (uint32_t)PA_N3 * H * 2;
       const int n1 = n_hb, n2 = n_hb * n_kc2;
       for (int tile = blockIdx.x; tile < n_tiles && !*abort_flag; tile += gridDim.x) {
@@ -132,7 +135,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           const int s = it % PA_STAGES;
           if (!tc_wait(&ctl->empty[s], ((it / PA_STAGES) & 1) ^ 1, abort_flag)) goto done;
           mbar_expect_tx(&ctl->full[s], bytes);
-          bulk_copy_g2s(ring + (size_t)s * PA_STAGE_BYTES, src, bytes, &ctl->full[s]);
+          bulk_copy_g2s_keep(ring + (size_t)s * PA_STAGE_BYTES, src, bytes, &ctl->full[s], keep_policy);
         }
       }
     } else if (warp == 1 && lane == 0) {
@@ -362,7 +365,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           const size_t off = (size_t)(k4 >> 1) * 128 + (k4 & 1) * 8;
           *reinterpret_cast<uint2*>(dhi + off) = make_uint2(pack_f16x2(hi.x, hi.y), pack_f16x2(hi.z, hi.w));
           *reinterpret_cast<uint2*>(dlo + off) = make_uint2(pack_f16x2(lo.x, lo.y), pack_f16x2(lo.z, lo.w));
-          if (live) *reinterpret_cast<float4*>(rec + k4 * 4) = sv;
+          if (live) __stcs(reinterpret_cast<float4*>(rec + k4 * 4), sv);
         }
       }
       fence_async_smem();
@@ -439,7 +442,7 @@ __global__ void __launch_bounds__(PA_THREADS, 1) actor_tc_pipelined_kernel(const
           o.w = tanh_from_t(fmaf(zz[i].w, zc, bb.w)) + n23.y;
           sq = fmaf(o.x, o.x, sq); sq = fmaf(o.y, o.y, sq); sq = fmaf(o.z, o.z, sq); sq = fmaf(o.w, o.w, sq);
           sn[i] = o;
-          if (live) *reinterpret_cast<float4*>(rec + D + 4 * k4) = o;
+          if (live) __stcs(reinterpret_cast<float4*>(rec + D + 4 * k4), o);
         }
         // the four lanes of a row add their partial squared norms (same order in every lane)
         sq += __shfl_xor_sync(0xffffffffu, sq, 1);
