@@ -21,7 +21,7 @@ OK, ERR_ARG, ERR_CONFIG, ERR_NO_WEIGHTS, ERR_WARMUP, ERR_STARVED = 0, -1, -2, -5
 ENV_CARTPOLE, ENV_ACROBOT, ENV_LINGAUSS = 0, 1, 2
 POLICY_EPS_GREEDY, POLICY_CATEGORICAL = 0, 1
 W_FP32, W_BF16 = 0, 1
-STREAM_ACTION, STREAM_RESET, STREAM_NOISE, STREAM_SAMPLE = 0, 1, 2, 3
+STREAM_ACTION, STREAM_RESET, STREAM_NOISE, STREAM_SAMPLE, STREAM_SHUFFLE = 0, 1, 2, 3, 4
 
 
 def build(force: bool = False) -> str:
@@ -98,6 +98,8 @@ def lib():
         "orc_select_categorical": (i32, [vp, i32, f32, vp, vp]),
         "orc_td_one": (None, [f64, f64, f64, i32, f64, f64, vp, vp]),
         "orc_gae": (None, [vp, vp, vp, i32, i32, f64, f64, vp, vp]),
+        "orc_shuffle_index": (i64, [u64, u64, i64, i64]),
+        "orc_normalize": (None, [vp, i64, f64, vp]),
         "orc_create": (vp, [vp, vp]),
         "orc_destroy": (None, [vp]),
         "orc_publish": (i32, [vp, vp, i64]),
@@ -356,6 +358,22 @@ def gae(rew, val, done, gamma, lam):
     ret = np.zeros((T, N), np.float64)
     lib().orc_gae(_p(rew), _p(val), _p(done), T, N, float(gamma), float(lam), _p(adv), _p(ret))
     return adv, ret
+
+
+def shuffle_index(seed, shuffle_id, R, i):
+    """Row that position i of shuffle `shuffle_id` takes, out of R rows."""
+    return int(lib().orc_shuffle_index(int(seed) & (2**64 - 1), int(shuffle_id) & (2**64 - 1), int(R), int(i)))
+
+
+def shuffle_order(seed, shuffle_id, R):
+    return np.array([shuffle_index(seed, shuffle_id, R, i) for i in range(R)], np.int64)
+
+
+def normalize(x, eps=1e-8):
+    x = np.ascontiguousarray(x, np.float32).ravel()
+    out = np.zeros(x.size, np.float64)
+    lib().orc_normalize(_p(x), x.size, float(eps), _p(out))
+    return out
 
 
 # --------------------------------------------------------------------------- the whole path

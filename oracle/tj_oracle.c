@@ -578,6 +578,59 @@ void orc_gae(const float *rew, const float *val, const uint8_t *done, int T, int
 }
 
 /* ===================================================================== */
+/* On-policy consumer (App. C synchronous mode; Table 2's PPO batch settings): per-segment advantage            */
+/* normalisation and shuffled minibatches.                                                                      */
+/*                                                                                                              */
+/* The row order of a shuffle is a keyed bijection of [0, R): a four-round balanced Feistel network on          */
+/* 2*hb bits (hb = half the bits of R - 1, rounded up, at least 1) whose round function is the first            */
+/* Philox word of the SHUFFLE stream at (index = right half, step = shuffle id, block = round), followed        */
+/* by cycle walking (apply again until the value falls below R).  A Feistel network is a bijection of its       */
+/* power-of-two domain and cycle walking restricts it to [0, R) (Black & Rogaway, "Ciphers with arbitrary       */
+/* finite domains", 2002).                                                                                      */
+/* ===================================================================== */
+static int shuffle_half_bits(uint64_t R) {
+  int bits = 0;
+  while (bits < 62 && ((uint64_t)1 << bits) < R) ++bits; /* 2^bits >= R */
+  int hb = (bits + 1) / 2;
+  return hb < 1 ? 1 : hb;
+}
+
+static uint64_t shuffle_feistel(uint64_t seed, uint64_t shuffle_id, int hb, uint64_t x) {
+  const uint64_t mask = ((uint64_t)1 << hb) - 1;
+  uint64_t left = x >> hb, right = x & mask;
+  for (uint32_t round = 0; round < 4; ++round) {
+    uint32_t w[4];
+    orc_stream_words(seed, ORC_STREAM_SHUFFLE, round, (uint32_t)right, shuffle_id, w);
+    uint64_t f = (uint64_t)w[0] & mask;
+    uint64_t new_right = left ^ f;
+    left = right;
+    right = new_right;
+  }
+  return (left << hb) | right;
+}
+
+/* row that position i of the shuffled order takes, out of R rows */
+int64_t orc_shuffle_index(uint64_t seed, uint64_t shuffle_id, int64_t R, int64_t i) {
+  if (R <= 0 || i < 0 || i >= R) return -1;
+  const int hb = shuffle_half_bits((uint64_t)R);
+  uint64_t y = shuffle_feistel(seed, shuffle_id, hb, (uint64_t)i);
+  while (y >= (uint64_t)R) y = shuffle_feistel(seed, shuffle_id, hb, y);
+  return (int64_t)y;
+}
+
+/* out_i = (x_i - mean) / (sqrt(var) + eps): mean and population variance over all n entries, in double */
+void orc_normalize(const float *x, int64_t n, double eps, double *out) {
+  if (n <= 0) return;
+  double sum = 0.0;
+  for (int64_t i = 0; i < n; ++i) sum += (double)x[i];
+  const double mean = sum / (double)n;
+  double sq = 0.0;
+  for (int64_t i = 0; i < n; ++i) sq += ((double)x[i] - mean) * ((double)x[i] - mean);
+  const double sd = sqrt(sq / (double)n);
+  for (int64_t i = 0; i < n; ++i) out[i] = ((double)x[i] - mean) / (sd + eps);
+}
+
+/* ===================================================================== */
 /* The whole path as a state machine                                      */
 /* ===================================================================== */
 struct orc_ctx {

@@ -30,7 +30,8 @@
  * Pinned by tests (CPU only): hand-worked CartPole step, Acrobot energy
  * conservation and RK4 order, Philox against an independent big-integer
  * restatement, MLP against a float64 library matmul, ring/sampler against brute
- * force, TD hand values, GAE closed forms.  Unpinned: nothing.
+ * force, TD hand values, GAE closed forms, the shuffle as a bijection with uniform positions, the
+ * normalisation's moments and hand values.  Unpinned: nothing.
  */
 #ifndef TJ_ORACLE_H
 #define TJ_ORACLE_H
@@ -43,7 +44,7 @@ extern "C" {
 enum { ORC_ENV_CARTPOLE = 0, ORC_ENV_ACROBOT = 1, ORC_ENV_LINGAUSS = 2 };
 enum { ORC_POLICY_EPS_GREEDY = 0, ORC_POLICY_CATEGORICAL = 1 };
 enum { ORC_W_FP32 = 0, ORC_W_BF16 = 1 };
-enum { ORC_STREAM_ACTION = 0, ORC_STREAM_RESET = 1, ORC_STREAM_NOISE = 2, ORC_STREAM_SAMPLE = 3 };
+enum { ORC_STREAM_ACTION = 0, ORC_STREAM_RESET = 1, ORC_STREAM_NOISE = 2, ORC_STREAM_SAMPLE = 3, ORC_STREAM_SHUFFLE = 4 };
 enum { ORC_OK = 0, ORC_ERR_ARG = -1, ORC_ERR_CONFIG = -2, ORC_ERR_NO_WEIGHTS = -5, ORC_ERR_WARMUP = -6,
        ORC_ERR_STARVED = -7 };
 
@@ -78,6 +79,10 @@ typedef struct {
   const float *logp;      /* [T][N] */
   const float *val;       /* [T+1][N] */
 } orc_segment;
+
+/* ---- on-policy consumer: shuffled row order of a segment and advantage normalisation (App. C; Table 2) ---- */
+int64_t orc_shuffle_index(uint64_t seed, uint64_t shuffle_id, int64_t R, int64_t i);
+void    orc_normalize(const float *x, int64_t n, double eps, double *out);
 
 /* ---- building blocks (each callable on its own so that it can be pinned) ---- */
 void     orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
