@@ -291,6 +291,33 @@ int tj_gae(tj_ctx *ctx, const float *rew, const float *val, const uint8_t *done,
  * are dropped and counted.  Errors: STARVED. */
 int tj_segment_acquire(tj_ctx *ctx, tj_segment *out);
 
+/* On-policy consumer (App. C, synchronous mode; Table 2: PPO's batch settings), the two steps between tj_gae and tj_ppo_step.
+ *
+ * tj_normalize: out_i = (x_i - mean) / (sqrt(var) + eps) with the mean and the population variance of all n entries
+ * (advantages of one segment: mean 0, variance 1).  Both sums are taken in double in a fixed order, so the result is
+ * reproducible.  x and out: device, n floats, may be the same array.  eps >= 0. */
+int tj_normalize(tj_ctx *ctx, const float *x, int64_t n, float eps, float *out);
+
+/* tj_segment_minibatch: rows of a segment in shuffled order.  Shuffle `shuffle_id` (one per epoch, say) is a keyed
+ * bijection of the segment's R = T * N rows: position i takes row perm(i) = walk(F(i)), where F is a four-round balanced
+ * Feistel network on 2 * hb bits (hb = half the bits of R - 1, rounded up, at least 1) whose round function is the first
+ * Philox word of the SHUFFLE stream at (index = right half, step = shuffle_id, block = round), and walk applies F again
+ * until the value is below R.  The call copies the rows at positions first .. first + out->n - 1 into dense arrays:
+ * obs [n][obs_dim], act, logp_old (the segment's logp), adv, ret (from the caller's [T][N] arrays, e.g. tj_gae's outputs,
+ * normalised or not) and, if row is not null, the source row indices.  Every position of 0 .. R - 1 occurs exactly once
+ * over the minibatches of one shuffle.  Errors: INVALID_ARG (null arrays, positions outside the segment). */
+typedef struct {
+  int32_t n;
+  float *obs;
+  int32_t *act;
+  float *logp_old;
+  float *adv;
+  float *ret;
+  int32_t *row;      /* nullable */
+} tj_ppo_minibatch;
+int tj_segment_minibatch(tj_ctx *ctx, const tj_segment *seg, const float *adv, const float *ret, uint64_t shuffle_id, int64_t first,
+                         const tj_ppo_minibatch *out);
+
 /* Does a segment view handed out by tj_segment_acquire still show the segment it was acquired as?  TJ_OK while the
  * producer has not come round to its slot again; TJ_ERR_STALE_SEGMENT once a later segment has begun to fill the slot
  * (the consumer was lapped: what it reads from the view may be a mixture).  Host bookkeeping only, nothing is enqueued. */

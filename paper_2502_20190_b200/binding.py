@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
 EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
-           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_segment_check", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view", "tj_calibrate_fp32",
+           "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_segment_check", "tj_normalize", "tj_segment_minibatch", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view", "tj_calibrate_fp32",
            "tj_last_error")
 
 
@@ -95,6 +95,8 @@ def load_library():
     L.tj_ppo_step.argtypes = [vp, vp, f32, f32, f32, f32, i64, f32, f32, f32, vp, vp, vp, vp]
     L.tj_segment_acquire.argtypes = [vp, vp]
     L.tj_segment_check.argtypes = [vp, vp]
+    L.tj_normalize.argtypes = [vp, vp, i64, f32, vp]
+    L.tj_segment_minibatch.argtypes = [vp, vp, vp, vp, C.c_uint64, i64, vp]
     L.tj_get_state.argtypes = [vp, vp]
     L.tj_set_state.argtypes = [vp, vp]
     L.tj_stats.argtypes = [vp, vp]
@@ -186,6 +188,19 @@ def tj_segment_acquire(h):
     seg = TjSegment()
     st = load_library().tj_segment_acquire(h, C.byref(seg))
     return st, seg
+
+
+class TjPpoMinibatch(C.Structure):
+    _fields_ = [("n", C.c_int32), ("obs", C.c_void_p), ("act", C.c_void_p), ("logp_old", C.c_void_p), ("adv", C.c_void_p),
+                ("ret", C.c_void_p), ("row", C.c_void_p)]
+
+
+def tj_normalize(h, x_ptr: int, n: int, eps: float, out_ptr: int):
+    return load_library().tj_normalize(h, x_ptr, n, eps, out_ptr)
+
+
+def tj_segment_minibatch(h, seg: TjSegment, adv_ptr: int, ret_ptr: int, shuffle_id: int, first: int, out: TjPpoMinibatch):
+    return load_library().tj_segment_minibatch(h, C.byref(seg), adv_ptr, ret_ptr, shuffle_id, first, C.byref(out))
 
 
 def tj_segment_check(h, seg: TjSegment):
@@ -414,6 +429,29 @@ class Context:
                         rew=self._view(seg.rew, (T, N), torch.float32), done=self._view(seg.done, (T, N), torch.uint8),
                         logp=self._view(seg.logp, (T, N), torch.float32),
                         val=self._view(seg.val, (T + 1, N), torch.float32))
+
+    def normalize(self, x, eps=1e-8, out=None):
+        """(x - mean) / (std + eps) over all entries of a float32 device tensor, in the library's kernels."""
+        assert x.is_cuda and x.dtype == self.torch.float32 and x.is_contiguous()
+        if out is None:
+            out = self.torch.empty_like(x)
+        self._check(tj_normalize(self.h, x.data_ptr(), x.numel(), float(eps), out.data_ptr()))
+        return out
+
+    def alloc_minibatch(self, n):
+        torch, dev = self.torch, self.device
+        t = dict(obs=torch.empty((n, self.D), dtype=torch.float32, device=dev), act=torch.empty(n, dtype=torch.int32, device=dev),
+                 logp_old=torch.empty(n, dtype=torch.float32, device=dev), adv=torch.empty(n, dtype=torch.float32, device=dev),
+                 ret=torch.empty(n, dtype=torch.float32, device=dev), row=torch.empty(n, dtype=torch.int32, device=dev))
+        t["c"] = TjPpoMinibatch(n, t["obs"].data_ptr(), t["act"].data_ptr(), t["logp_old"].data_ptr(), t["adv"].data_ptr(),
+                                t["ret"].data_ptr(), t["row"].data_ptr())
+        return t
+
+    def segment_minibatch(self, seg, adv, ret, shuffle_id, first, mb):
+        """Rows at positions first .. first + n - 1 of shuffle `shuffle_id` of the segment, copied into the minibatch arrays."""
+        assert adv.is_contiguous() and ret.is_contiguous() and adv.numel() == seg["T"] * seg["N"] == ret.numel()
+        self._check(tj_segment_minibatch(self.h, seg["c"], adv.data_ptr(), ret.data_ptr(), int(shuffle_id), int(first), mb["c"]))
+        return mb
 
     def segment_check(self, seg, allow=(TJ_OK, TJ_ERR_STALE_SEGMENT)):
         return self._check(tj_segment_check(self.h, seg["c"]), allow)

@@ -92,6 +92,7 @@ size_t carve(tj_ctx* x, void* base) {
   x->blob_stage = cv.take<float>(blob_floats(D, c.hidden, c.n_actions, vh));
   x->dstats = cv.take<DevStats>(1);
   x->td_partial = cv.take<float>((size_t)td_grid(kMaxTdRows));
+  x->norm_scratch = cv.take<double>(normalize_scratch_doubles());
   if (c.replay_capacity > 0) {
     const size_t nb = (size_t)(c.replay_capacity / N);
     x->ring = cv.take<float>((size_t)c.replay_capacity * (2 * D + 4));
@@ -723,6 +724,39 @@ int tj_segment_acquire(tj_ctx* x, tj_segment* out) {
   }
   x->hs.starved_calls += 1;
   return fail(x, TJ_ERR_STARVED, "no complete segment within the staleness bound");
+}
+
+int tj_normalize(tj_ctx* x, const float* in, int64_t n, float eps, float* out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!in || !out) return fail(x, TJ_ERR_INVALID_ARG, "arrays must not be null");
+  if (n < 0 || !(eps >= 0.f)) return fail(x, TJ_ERR_INVALID_ARG, "n and eps must not be negative");
+  if (n == 0) return TJ_OK;
+  LaunchScope scope(x, TJ_K_GAE, 3);
+  cudaError_t e = launch_normalize(in, n, (double)eps, out, x->norm_scratch, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "normalisation");
+  return TJ_OK;
+}
+
+int tj_segment_minibatch(tj_ctx* x, const tj_segment* segv, const float* adv, const float* ret, uint64_t shuffle_id, int64_t first,
+                         const tj_ppo_minibatch* out) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (!segv || !adv || !ret || !out) return fail(x, TJ_ERR_INVALID_ARG, "arguments must not be null");
+  if (!out->obs || !out->act || !out->logp_old || !out->adv || !out->ret) return fail(x, TJ_ERR_INVALID_ARG, "minibatch arrays must not be null");
+  if (!segv->obs || !segv->act || !segv->logp || segv->T < 1 || segv->N < 1) return fail(x, TJ_ERR_INVALID_ARG, "not a segment");
+  const int64_t R = (int64_t)segv->T * segv->N;
+  if (out->n < 0 || first < 0 || first + out->n > R) return fail(x, TJ_ERR_INVALID_ARG, "positions first .. first + n must lie inside the segment's T * N rows");
+  if (R > ((int64_t)1 << 31)) return fail(x, TJ_ERR_UNSUPPORTED, "segments of more than 2^31 rows");
+  if (out->n == 0) return TJ_OK;
+  MinibatchParams p{};
+  p.n = out->n; p.D = x->D; p.hb = shuffle_half_bits(R); p.R = R; p.first = first;
+  p.seed = make_uint2((uint32_t)x->cfg.seed, (uint32_t)(x->cfg.seed >> 32));
+  p.shuffle_id = shuffle_id;
+  p.seg_obs = segv->obs; p.seg_act = segv->act; p.seg_logp = segv->logp; p.adv_in = adv; p.ret_in = ret;
+  p.obs = out->obs; p.act = out->act; p.logp = out->logp_old; p.adv = out->adv; p.ret = out->ret; p.row = out->row;
+  LaunchScope scope(x, TJ_K_SAMPLE, 1);
+  cudaError_t e = launch_segment_minibatch(p, x->stream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "segment minibatch");
+  return TJ_OK;
 }
 
 int tj_segment_check(tj_ctx* x, const tj_segment* segv) {

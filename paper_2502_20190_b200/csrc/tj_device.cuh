@@ -6,7 +6,7 @@
 
 namespace tj {
 
-enum : uint32_t { STREAM_ACTION = 0, STREAM_RESET = 1, STREAM_NOISE = 2, STREAM_SAMPLE = 3 };
+enum : uint32_t { STREAM_ACTION = 0, STREAM_RESET = 1, STREAM_NOISE = 2, STREAM_SAMPLE = 3, STREAM_SHUFFLE = 4 };
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and xors, the key
 // advancing by the two Weyl constants each round.

@@ -143,6 +143,24 @@ struct SampleParams {
   DevStats* stats;
 };
 
+struct MinibatchParams {
+  int n, D, hb;
+  long long R, first;
+  uint2 seed;
+  unsigned long long shuffle_id;
+  const float* seg_obs;
+  const int* seg_act;
+  const float* seg_logp;
+  const float* adv_in;
+  const float* ret_in;
+  float* obs;
+  int* act;
+  float* logp;
+  float* adv;
+  float* ret;
+  int* row;
+};
+
 struct TcEnvParams {
   int fused;                 // 0: network only
   int A, max_ep, rec_words, version;
@@ -219,6 +237,10 @@ int td_static_max_rows();
 cudaError_t launch_td_static(const TdParams& p, int device, cudaStream_t s, bool* too_large);
 cudaError_t launch_gae(const float* rew, const float* val, const uint8_t* done, int T, int N, float gamma, float lambda,
                        float* adv, float* ret, cudaStream_t s);
+int shuffle_half_bits(long long R);
+size_t normalize_scratch_doubles();
+cudaError_t launch_normalize(const float* x, long long n, double eps, float* out, double* scratch, cudaStream_t s);
+cudaError_t launch_segment_minibatch(const MinibatchParams& p, cudaStream_t s);
 size_t fma_rate_sink_floats(int sm_count);
 double launch_fma_rate(float* sink, int sm_count, int outer, cudaStream_t s, cudaError_t* err);
 cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);
@@ -250,6 +272,7 @@ struct tj_ctx {
   int* elig_list;
   int* elig_count;
   float* td_partial;
+  double* norm_scratch;  // per-block partial sums of tj_normalize
   float* sgd_scratch;   // learner update: activations and their gradients for one minibatch (FP32 replay contexts)
   int sgd_rows;         // rows the scratch holds
   tj::DevStats* dstats;

@@ -38,7 +38,6 @@ constexpr int PA_KC = 128;                 // K elements per weight chunk (128 x
 constexpr int PA_W_BYTES = PA_NB * PA_KC * 2;              // bytes of a hidden-layer weight chunk, and of one env-matrix part
 constexpr int PA_STAGE_BYTES = PA_W_BYTES;
 constexpr int PA_STAGES = 65536 / PA_STAGE_BYTES;
-constexpr uint32_t PA_B_SBO = (PA_KC / 8) * 128;           // bytes between 8-row groups of a chunk
 constexpr int PA_X_BYTES = PA_M * PA_D * 2;
 constexpr int PA_U_BYTES = 131072;
 constexpr int PA_THREADS = 640;            // warps 0-3: producer, MMA issuer, two idle; 4-11 network; 12-19 env

@@ -4,13 +4,14 @@
 
 Per iteration the actor rolls out one segment with the newest published parameters (tj_actor_step), the learner takes the
 oldest unconsumed segment (tj_segment_acquire), computes advantages (tj_gae), runs a few epochs of minibatch updates
-(tj_ppo_step) and publishes the result as the next parameter version (tj_publish_weights).  With `lag` segments rolled out
+over shuffled rows (tj_normalize, tj_segment_minibatch, tj_ppo_step) and publishes the result as the next parameter
+version (tj_publish_weights).  With `lag` segments rolled out
 ahead of the first update, every consumed segment is exactly `lag` versions older than the learner -- the on-policy form of
 the staleness that the paper controls through its production/consumption balance (Sec. 3.3; the "New / Lag" curves of
 Sec. 4.3.2 and App. D.1).  lag = 0 is the synchronous mode of App. C.  The library's staleness bound is set to `lag`, so a
 staler segment would be dropped, and the statistics confirm none is.
 
-Driver-side arithmetic: only the per-segment normalisation of the advantages (mean 0, variance 1), done with torch."""
+Every arithmetic step runs in the library's kernels; torch only holds the device arrays."""
 from __future__ import annotations
 
 import argparse
@@ -35,6 +36,7 @@ def train(lag=0, iters=150, n_envs=1024, rollout=32, hidden=64, minibatch=4096, 
     for _ in range(lag):                       # the producer runs `lag` segments ahead of the consumer
         ctx.actor_step(rollout)
     hist, t_adam, last_eps, last_ret = [], 0, 0, 0.0
+    n_shuffles, mbs = 0, {}
     rows = rollout * n_envs
     for it in range(1, iters + 1):
         ctx.actor_step(rollout)
@@ -43,15 +45,16 @@ def train(lag=0, iters=150, n_envs=1024, rollout=32, hidden=64, minibatch=4096, 
             continue
         seg_lag = ctx.stats()["learner_version"] - seg["version"]
         adv, ret = ctx.gae(seg["rew"], seg["val"], seg["done"], gamma, lam)
-        adv = ((adv - adv.mean()) / (adv.std() + 1e-8)).reshape(-1).contiguous()
-        ret = ret.reshape(-1)
-        obs, act, logp = seg["obs"].reshape(rows, 4), seg["act"].reshape(-1), seg["logp"].reshape(-1)
+        ctx.normalize(adv, 1e-8, out=adv)              # advantages of the segment: mean 0, variance 1
         stats = None
         for _ in range(epochs):
+            n_shuffles += 1                            # a fresh row order per epoch
             for r0 in range(0, rows, minibatch):
-                r1 = min(rows, r0 + minibatch)
+                n = min(rows, r0 + minibatch) - r0
+                mb = mbs.get(n) or mbs.setdefault(n, ctx.alloc_minibatch(n))
+                ctx.segment_minibatch(seg, adv, ret, n_shuffles, r0, mb)
                 t_adam += 1
-                stats = ctx.ppo_step(obs[r0:r1], act[r0:r1], logp[r0:r1], adv[r0:r1], ret[r0:r1], lr, theta, m, v, t_adam,
+                stats = ctx.ppo_step(mb["obs"], mb["act"], mb["logp_old"], mb["adv"], mb["ret"], lr, theta, m, v, t_adam,
                                      clip_eps, c_v, c_e)
         ctx.publish_weights(theta)
         s = ctx.stats()
