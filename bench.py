@@ -140,7 +140,7 @@ def aggregate_throughput(units_per_replica, world, max_ms):
 class Runner:
     """Drives one context through the workload's call pattern."""
 
-    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False):
+    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False, two_stream=False):
         self.torch, self.name = torch, name
         self.w = dict(synth.WORKLOADS[name])
         if n_envs:
@@ -181,13 +181,24 @@ class Runner:
             self.ret = torch.empty((T, N), dtype=torch.float32, device="cuda")
             self.host_adv_mean = torch.empty(1, dtype=torch.float32).pin_memory()
         self.publish(False)
+        # --two-stream: the learner's calls on a second CUDA stream; a pass then runs the learner on what was produced so far,
+        # the actor's next block beside it, and the publish last (replay workloads)
+        self.two_stream = bool(two_stream) and not self.on_policy
+        if self.two_stream:
+            self.ctx.use_learner_stream(True)
+            self.lstream = self.ctx.learner_stream
+            self.actor()
 
     def publish(self, from_host):
         if self.with_update:
             self.ctx.publish_weights(self.theta)
             self.version += 1
             if self.version % 1000 == 0:
-                self.theta_target.copy_(self.theta)
+                if getattr(self, "two_stream", False):
+                    with self.torch.cuda.stream(self.lstream):
+                        self.theta_target.copy_(self.theta)
+                else:
+                    self.theta_target.copy_(self.theta)
             return
         blob = (self.host_blobs if from_host else self.dev_blobs)[self.version % self.n_pool]
         if from_host:
@@ -217,6 +228,17 @@ class Runner:
 
     def one_pass(self, e2e=False):
         torch = self.torch
+        if self.two_stream:
+            self.learner()
+            self.actor()
+            self.publish(e2e)
+            if e2e:
+                with torch.cuda.stream(self.lstream):
+                    self.host_td.copy_(self.out["td"], non_blocking=True)
+                    self.host_loss.copy_(self.out["loss"], non_blocking=True)
+                self.lstream.synchronize()
+                torch.cuda.current_stream().synchronize()
+            return
         self.actor()
         self.learner()
         self.publish(e2e)
@@ -233,6 +255,8 @@ class Runner:
             events[0].record()
         for _ in range(patterns):
             self.one_pass(e2e)
+        if self.two_stream:      # the step ends when both streams have finished it
+            self.torch.cuda.current_stream().wait_event(self.lstream.record_event())
         if events:
             events[1].record()
 
@@ -274,7 +298,7 @@ def run_ours(args):
     binding.load_library()
     peaks = load_peaks()
     name = args.workload
-    r = Runner(name, torch, binding, local, args.envs, args.with_update)
+    r = Runner(name, torch, binding, local, args.envs, args.with_update, args.two_stream)
     w = r.w
     N = w["n_envs"]
     R = args.patterns or PATTERNS_PER_STEP[name]
@@ -398,7 +422,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "bf16" if w["weight_dtype"] == synth.W_BF16 else "f32", "data": "synthetic",
         "config": {"workload": name, "n_envs": N, "patterns_per_step": R, "actor_steps_per_pattern": r.actor_steps,
                    "minibatch": w.get("minibatch"), "mlp": "%d-%d-%d-%d" % (w["obs_dim"], w["hidden"], w["hidden"], w["n_actions"]),
-                   "replicas": world, "learner_update": r.with_update,
+                   "replicas": world, "learner_update": r.with_update, "two_stream": r.two_stream,
                    "l2": "flushed between steps (256 MiB write outside the per-step event pairs)" if need_flush
                    else "ring larger than L2"},
         "consumed_samples_per_s": consumed / (tot_ms * 1e-3),
@@ -617,6 +641,7 @@ def main():
     ap.add_argument("--envs", type=int, default=0, help="profiling aid: run the workload with this many envs (ring scaled to the same number of steps)")
     ap.add_argument("--patterns", type=int, default=0, help="passes of the path per step (default: per workload, about 50 ms of GPU time)")
     ap.add_argument("--with-update", action="store_true", help="FP32 replay workloads: the learner step also runs tj_sgd_step and publishes the parameters it trains")
+    ap.add_argument("--two-stream", action="store_true", help="replay workloads: learner calls on a second CUDA stream, passes software-pipelined (learner on the previous block beside the actor's next one)")
     ap.add_argument("--sweep", action="store_true", help="also report consumed samples/s for each staleness bound the workload names")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=16.0)

@@ -55,7 +55,7 @@ typedef enum {
   TJ_ERR_WARMUP = -6,        /* fewer resident records than cfg.warmup (Table 2: buffer warmup size) */
   TJ_ERR_STARVED = -7,       /* nothing eligible: the consumer is ahead of the producer (Eq. 3: TR_L ~ TR_A) */
   TJ_ERR_STALE_SEGMENT = -8, /* tj_segment_check: the producer has begun to overwrite the segment's slot */
-  TJ_ERR_TIMEOUT = -9,       /* tj_stats: a kernel's bounded wait ran out (device_error holds the code) */
+  TJ_ERR_TIMEOUT = -9,       /* tj_stats: a kernel's bounded wait ran out (device_error holds the code); tj_wait: time limit */
   TJ_ERR_UNSUPPORTED = -10   /* valid request this build does not implement */
 } tj_status;
 
@@ -166,6 +166,24 @@ int tj_query_workspace(const tj_config *cfg, size_t *bytes, size_t *align);
  * (a cudaStream_t; NULL = the legacy default stream).  Seeds every environment from the reset stream.
  * Errors: INVALID_ARG, CONFIG, WORKSPACE, CUDA. */
 int tj_create(const tj_config *cfg, void *workspace, size_t bytes, void *cuda_stream, tj_ctx **out);
+
+/* Concurrent actor and learner (Sec. 3.1, Fig. 2: the actor, buffer and learner loops run side by side; dependencies I and
+ * III become asynchronous hand-overs).  After this call the learner-side entry points -- tj_replay_sample, tj_td_error(_static),
+ * tj_sgd_step, tj_adam_step, tj_ppo_step, tj_gae, tj_normalize, tj_segment_minibatch and tj_publish_weights -- enqueue on
+ * `cuda_stream`, tj_actor_step stays on the stream given to tj_create, and the library orders the two with CUDA events at
+ * the hand-overs only:
+ *   - a sample (or a segment acquisition) waits for the actor launches enqueued before it (it reads their records);
+ *   - an actor call waits for the sampler launched before it (ring blocks it may overwrite), for the last publish (it reads
+ *     the newest parameters) and, in segment mode, for the learner calls enqueued before it;
+ *   - a publish waits for the actor launches enqueued before it (they may still read the buffer it rewrites).
+ * TD error and parameter updates therefore overlap with the actor steps the host enqueues after the sample.  Results depend
+ * only on the host's call order, exactly as on one stream.  The caller's arrays passed to learner-side calls must be safe to
+ * use on that stream.  NULL or the create stream switches back.  Synchronises both streams. */
+int tj_set_learner_stream(tj_ctx *ctx, void *cuda_stream);
+
+/* Host-side bounded wait: returns TJ_OK once everything enqueued on the actor stream (which = 0) or the learner stream
+ * (which = 1) has finished, TJ_ERR_TIMEOUT if that takes longer than timeout_ms (nothing is cancelled; call again). */
+int tj_wait(tj_ctx *ctx, int32_t which, int32_t timeout_ms);
 
 /* Free the host object.  Does not touch the workspace.  Synchronises the stream. */
 int tj_destroy(tj_ctx *ctx);

@@ -67,3 +67,35 @@ def starved_fraction(staleness_bound: int, publishes_per_block: float) -> float:
     if publishes_per_block <= 0:
         raise ValueError("publishes_per_block must be positive")
     return max(0.0, 1.0 - (staleness_bound + 1) / publishes_per_block)
+
+
+def balanced_cadence(actor_step_s: float, learner_step_s: float, minibatch: int, n_envs: int, staleness_bound: int,
+                     max_steps: int = 64) -> dict:
+    """Cadence for CONCURRENT actor and learner streams (Sec. 3.1, Fig. 2; Eq. 3's TR_L ~ TR_A): per iteration the actor
+    takes k env steps of all n_envs while the learner takes u steps on what was produced before, so an iteration lasts about
+    max(k * actor_step_s, u * learner_step_s) and neither stream idles when the two are equal.  With one parameter version
+    per iteration the consumed samples are at most one iteration behind, so any bound >= 1 admits the cadence; bound 0 needs
+    the streams in lock step (k = u = 1 and no overlap).  Returns k, u (one of them 1, the other at most max_steps), the
+    realised consumed : produced ratio P, both streams' busy time per iteration and the share of the iteration the slower
+    one leaves the faster one idle."""
+    if actor_step_s <= 0 or learner_step_s <= 0:
+        raise ValueError("step times must be positive")
+    if staleness_bound < 1:
+        k, u = 1, 1
+    elif actor_step_s >= learner_step_s:
+        k, u = 1, max(1, min(max_steps, int(round(actor_step_s / learner_step_s))))
+    else:
+        k, u = max(1, min(max_steps, int(round(learner_step_s / actor_step_s)))), 1
+    t_a, t_l = k * actor_step_s, u * learner_step_s
+    return dict(actor_steps=k, learner_steps=u, P=realised_ratio(k, minibatch, n_envs, u), actor_busy_s=t_a, learner_busy_s=t_l,
+                idle_share=abs(t_a - t_l) / max(t_a, t_l))
+
+
+def step_times_from_stats(stats: dict, actor_steps: int, learner_steps: int) -> tuple:
+    """(seconds per actor step of all envs, seconds per learner step) from a context's per-kernel-class times."""
+    ms = stats["kernel_ms"]
+    t_a = (ms[0] + ms[1] + ms[2]) * 1e-3
+    t_l = (ms[3] + ms[4] + ms[5] + ms[7]) * 1e-3
+    if actor_steps <= 0 or learner_steps <= 0 or t_a <= 0 or t_l <= 0:
+        raise ValueError("no timed launches")
+    return t_a / actor_steps, t_l / learner_steps

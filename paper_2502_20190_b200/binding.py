@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "TJ_OK", -1: "TJ_ERR_INVALID_ARG", -2: "TJ_ERR_CONFIG", -3: "
                 -5: "TJ_ERR_NO_WEIGHTS", -6: "TJ_ERR_WARMUP", -7: "TJ_ERR_STARVED", -8: "TJ_ERR_STALE_SEGMENT",
                 -9: "TJ_ERR_TIMEOUT", -10: "TJ_ERR_UNSUPPORTED"}
 
-EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
+EXPORTS = ("tj_query_workspace", "tj_create", "tj_destroy", "tj_set_learner_stream", "tj_wait", "tj_publish_weights", "tj_actor_step", "tj_replay_sample",
            "tj_td_error", "tj_td_error_static", "tj_sgd_step", "tj_adam_step", "tj_ppo_step", "tj_gae", "tj_segment_acquire", "tj_segment_check", "tj_normalize", "tj_segment_minibatch", "tj_get_state", "tj_set_state", "tj_stats", "tj_set_profiling", "tj_ring_view", "tj_calibrate_fp32",
            "tj_last_error")
 
@@ -84,6 +84,8 @@ def load_library():
     L.tj_query_workspace.argtypes = [vp, vp, vp]
     L.tj_create.argtypes = [vp, vp, C.c_size_t, vp, vp]
     L.tj_destroy.argtypes = [vp]
+    L.tj_set_learner_stream.argtypes = [vp, vp]
+    L.tj_wait.argtypes = [vp, i32, i32]
     L.tj_publish_weights.argtypes = [vp, vp, C.c_size_t, i32, vp]
     L.tj_actor_step.argtypes = [vp, i32, vp]
     L.tj_replay_sample.argtypes = [vp, i32, vp, vp]
@@ -133,6 +135,14 @@ def tj_create(cfg: TjConfig, workspace_ptr: int, nbytes: int, stream_ptr: int):
 
 def tj_destroy(h):
     return load_library().tj_destroy(h)
+
+
+def tj_set_learner_stream(h, stream_ptr: int):
+    return load_library().tj_set_learner_stream(h, stream_ptr or None)
+
+
+def tj_wait(h, which: int, timeout_ms: int):
+    return load_library().tj_wait(h, which, timeout_ms)
 
 
 def tj_publish_weights(h, blob_ptr: int, nbytes: int, on_device: int):
@@ -291,6 +301,17 @@ class Context:
         self.value_head = c.policy_kind == 1
         self.rec_words = 2 * self.D + 4
         self._batch = None
+
+    def use_learner_stream(self, on=True):
+        """Learner-side calls on a second torch stream (concurrent with the actor), or back on the one stream."""
+        if on:
+            if getattr(self, "learner_stream", None) is None:
+                self.learner_stream = self.torch.cuda.Stream(self.device)
+            return self._check(tj_set_learner_stream(self.h, self.learner_stream.cuda_stream))
+        return self._check(tj_set_learner_stream(self.h, 0))
+
+    def wait(self, which, timeout_ms, allow=(TJ_OK, TJ_ERR_TIMEOUT)):
+        return self._check(tj_wait(self.h, which, timeout_ms), allow)
 
     def close(self):
         if getattr(self, "h", None):

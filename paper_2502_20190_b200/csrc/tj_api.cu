@@ -1,6 +1,8 @@
 // C ABI shell: configuration checks, workspace carving, host-side bookkeeping (versions, cursor, segment
 // slots, counters) and the kernel launches behind each entry point.
 #include <algorithm>
+#include <chrono>
+#include <thread>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -167,18 +169,20 @@ struct LaunchScope {
   tj_ctx* x;
   cudaEvent_t a = nullptr, b = nullptr;
   int cls;
+  cudaStream_t st;
   // may_create = false: time the launches only if two pooled events are free (an entry point that must not create
-  // anything skips the timing rather than make events)
-  LaunchScope(tj_ctx* ctx, int kernel_class, int n_launches, bool may_create = true) : x(ctx), cls(kernel_class) {
+  // anything skips the timing rather than make events).  on_learner: the launches go to the learner stream.
+  LaunchScope(tj_ctx* ctx, int kernel_class, int n_launches, bool may_create = true, bool on_learner = false)
+      : x(ctx), cls(kernel_class), st(on_learner ? ctx->lstream : ctx->stream) {
     x->hs.kernel_launches += n_launches;
     if (!x->profiling) return;
     if (!may_create && x->ev_pool.size() < 2) return;
     a = take(); b = take();
-    if (a && b) cudaEventRecord(a, x->stream);
+    if (a && b) cudaEventRecord(a, st);
   }
   ~LaunchScope() {
     if (!a || !b) return;
-    cudaEventRecord(b, x->stream);
+    cudaEventRecord(b, st);
     x->spans.push_back({a, b, cls});
   }
   cudaEvent_t take() {
@@ -200,6 +204,17 @@ void drain_spans(tj_ctx* x) {
     x->ev_pool.push_back(sp.b);
   }
   x->spans.clear();
+}
+
+// ---- ordering between the actor stream and the learner stream (no-ops while they are the same stream)
+void learner_waits_for_actor(tj_ctx* x) {      // the learner is about to read what actor launches wrote (ring, segments)
+  if (x->two_stream && x->has_actor) cudaStreamWaitEvent(x->lstream, x->ev_actor, 0);
+}
+void actor_launched(tj_ctx* x) {
+  if (x->two_stream) { cudaEventRecord(x->ev_actor, x->stream); x->has_actor = true; }
+}
+void learner_launched(tj_ctx* x) {
+  if (x->two_stream) { cudaEventRecord(x->ev_learner, x->lstream); x->has_learner = true; }
 }
 
 uint64_t explore_threshold(float eps) {
@@ -238,6 +253,9 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
   const size_t need = carve(x, workspace);
   if (bytes < need) { delete x; g_err = "workspace smaller than tj_query_workspace reports"; return TJ_ERR_WORKSPACE; }
   x->stream = static_cast<cudaStream_t>(cuda_stream);
+  x->lstream = x->stream; x->two_stream = false;
+  x->ev_actor = x->ev_sample = x->ev_publish = x->ev_learner = nullptr;
+  x->has_actor = x->has_sample = x->has_publish = x->has_learner = false;
   x->N = cfg->n_envs; x->D = cfg->obs_dim; x->H = cfg->hidden; x->A = cfg->n_actions;
   x->S_d = env_state_dim(*cfg);
   x->value_head = cfg->policy_kind == TJ_POLICY_CATEGORICAL;
@@ -305,16 +323,54 @@ int tj_create(const tj_config* cfg, void* workspace, size_t bytes, void* cuda_st
 int tj_destroy(tj_ctx* ctx) {
   if (!ctx) return TJ_ERR_INVALID_ARG;
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->two_stream) cudaStreamSynchronize(ctx->lstream);
   drain_spans(ctx);
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : {ctx->ev_actor, ctx->ev_sample, ctx->ev_publish, ctx->ev_learner})
+    if (e) cudaEventDestroy(e);
   delete ctx;
   return TJ_OK;
+}
+
+int tj_set_learner_stream(tj_ctx* x, void* cuda_stream) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  cudaStream_t ls = static_cast<cudaStream_t>(cuda_stream);
+  // everything enqueued so far is ordered before the switch
+  cudaError_t e = cudaStreamSynchronize(x->stream);
+  if (e == cudaSuccess && x->two_stream) e = cudaStreamSynchronize(x->lstream);
+  if (e != cudaSuccess) return cuda_fail(x, e, "set learner stream: synchronise");
+  if (ls == x->stream || !cuda_stream) {
+    x->lstream = x->stream; x->two_stream = false;
+    x->has_actor = x->has_sample = x->has_publish = x->has_learner = false;
+    return TJ_OK;
+  }
+  for (cudaEvent_t* ev : {&x->ev_actor, &x->ev_sample, &x->ev_publish, &x->ev_learner})
+    if (!*ev && (e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(x, e, "set learner stream: events");
+  x->lstream = ls; x->two_stream = true;
+  x->has_actor = x->has_sample = x->has_publish = x->has_learner = false;
+  return TJ_OK;
+}
+
+int tj_wait(tj_ctx* x, int32_t which, int32_t timeout_ms) {
+  if (!x) return TJ_ERR_INVALID_ARG;
+  if (which < 0 || which > 1 || timeout_ms < 0) return fail(x, TJ_ERR_INVALID_ARG, "which must be 0 (actor stream) or 1 (learner stream), timeout_ms >= 0");
+  cudaStream_t st = which == 0 ? x->stream : x->lstream;
+  const auto t0 = std::chrono::steady_clock::now();
+  for (;;) {
+    const cudaError_t q = cudaStreamQuery(st);
+    if (q == cudaSuccess) return TJ_OK;
+    if (q != cudaErrorNotReady) return cuda_fail(x, q, "wait");
+    const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(std::chrono::steady_clock::now() - t0).count();
+    if (ms >= timeout_ms) return fail(x, TJ_ERR_TIMEOUT, which == 0 ? "the actor stream has not drained within the time limit" : "the learner stream has not drained within the time limit");
+    std::this_thread::sleep_for(std::chrono::microseconds(50));
+  }
 }
 
 int tj_set_profiling(tj_ctx* x, int32_t on) {
   if (!x) return TJ_ERR_INVALID_ARG;
   if (on && !x->profiling) {
     cudaStreamSynchronize(x->stream);
+    if (x->two_stream) cudaStreamSynchronize(x->lstream);
     drain_spans(x);
     for (int i = 0; i < TJ_KERNEL_CLASSES; ++i) { x->hs.kernel_ms[i] = 0.0; x->hs.kernel_count[i] = 0; }
   }
@@ -327,40 +383,43 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
   if (!blob) return fail(x, TJ_ERR_INVALID_ARG, "blob is null");
   if (nbytes != x->n_blob * sizeof(float)) return fail(x, TJ_ERR_INVALID_ARG, "blob size does not match the configured network");
   cudaError_t e;
+  // the buffer about to be rewritten may still be read by actor launches that are in flight
+  learner_waits_for_actor(x);
   const float* src = static_cast<const float*>(blob);
   if (!on_device) {
-    if ((e = cudaMemcpyAsync(x->blob_stage, blob, nbytes, cudaMemcpyHostToDevice, x->stream)) != cudaSuccess)
+    if ((e = cudaMemcpyAsync(x->blob_stage, blob, nbytes, cudaMemcpyHostToDevice, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: host to device copy");
     src = x->blob_stage;
   }
-  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : 1));
+  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : 1), true, true);
   const int next = x->active ^ 1;
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
-  if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->stream)) != cudaSuccess)
+  if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->lstream)) != cudaSuccess)
     return cuda_fail(x, e, "publish: repack");
   uint16_t* dst_tc = nullptr;
   if (x->use_tc) {
     dst_tc = x->version == 0 ? x->wtc[x->active] : x->wtc[next];
-    if ((e = launch_pack_tc_weights(src, dst_tc, x->D, x->H, x->A, x->value_head, x->stream)) != cudaSuccess)
+    if ((e = launch_pack_tc_weights(src, dst_tc, x->D, x->H, x->A, x->value_head, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: tensor-core repack");
     if (x->use_tc_pipelined &&
         (e = launch_pack_pipelined_weights(src, x->version == 0 ? x->wtc_pipe[x->active] : x->wtc_pipe[next], x->D, x->H, x->A,
-                                           x->stream)) != cudaSuccess)
+                                           x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: tensor-core repack (pipelined actor)");
   }
   if (x->version != 0) x->active = next;
   x->version += 1;
   if (!x->has_target || (x->cfg.target_sync_interval > 0 && x->k - x->k_last_sync >= x->cfg.target_sync_interval)) {
-    if ((e = cudaMemcpyAsync(x->wtarget, dst, x->wl.total * sizeof(float), cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+    if ((e = cudaMemcpyAsync(x->wtarget, dst, x->wl.total * sizeof(float), cudaMemcpyDeviceToDevice, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: target refresh");
     if (x->use_tc && (e = cudaMemcpyAsync(x->wtc_target, dst_tc, tc_weight_elems(x->D, x->H) * sizeof(uint16_t),
-                                          cudaMemcpyDeviceToDevice, x->stream)) != cudaSuccess)
+                                          cudaMemcpyDeviceToDevice, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: target refresh (tensor-core weights)");
     x->has_target = true;
     x->k_last_sync = x->k;
   }
-  if (!on_device) {
-    // the staging buffer is reused by the next host publish; the copy above already left host memory
+  if (x->two_stream) {   // the next actor call reads the new parameters: it waits for this
+    cudaEventRecord(x->ev_publish, x->lstream);
+    x->has_publish = true;
   }
   if (version_out) *version_out = x->version;
   return TJ_OK;
@@ -371,6 +430,13 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
   if (n_steps < 0) return fail(x, TJ_ERR_INVALID_ARG, "n_steps is negative");
   if (x->version == 0) return fail(x, TJ_ERR_NO_WEIGHTS, "actor called before the first publish");
   if (n_steps == 0) return TJ_OK;
+  if (x->two_stream) {
+    // newest published parameters; the sampler has finished with the ring blocks this call may overwrite; in segment
+    // mode a slot is restarted only after the learner's calls on its last segment have been passed
+    if (x->has_publish) cudaStreamWaitEvent(x->stream, x->ev_publish, 0);
+    if (x->has_sample) cudaStreamWaitEvent(x->stream, x->ev_sample, 0);
+    if (x->cfg.replay_capacity == 0 && x->has_learner) cudaStreamWaitEvent(x->stream, x->ev_learner, 0);
+  }
   const tj_config& c = x->cfg;
   const bool on_policy = c.replay_capacity == 0;
   ActorParams p{};
@@ -439,6 +505,7 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
     e = launch_actor(c.env_kind, p, x->stream);
   }
   if (e != cudaSuccess) return cuda_fail(x, e, "actor step");
+  actor_launched(x);
   // host mirror of what the kernel does to versions, cursor and segment slots
   for (int i = 0; i < n_steps; ++i) {
     if (on_policy) {
@@ -481,8 +548,9 @@ int tj_replay_sample(tj_ctx* x, int32_t staleness_bound, int32_t* idx_out, const
     return fail(x, TJ_ERR_STARVED, "no resident record within the staleness bound");
   }
   if ((uint64_t)n_elig * (uint64_t)x->N > 0xFFFFFFFFull) return fail(x, TJ_ERR_UNSUPPORTED, "eligible set too large");
-  LaunchScope scope(x, TJ_K_SAMPLE, 2);
-  cudaError_t e = launch_eligible(x->block_ver, n_blocks, x->version, S, x->elig_list, x->elig_count, x->stream);
+  learner_waits_for_actor(x);
+  LaunchScope scope(x, TJ_K_SAMPLE, 2, true, true);
+  cudaError_t e = launch_eligible(x->block_ver, n_blocks, x->version, S, x->elig_list, x->elig_count, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "eligible list");
   SampleParams p{};
   p.B = c.minibatch; p.D = x->D; p.N = x->N; p.rec_words = x->rec_words;
@@ -492,7 +560,8 @@ int tj_replay_sample(tj_ctx* x, int32_t staleness_bound, int32_t* idx_out, const
   p.idx_out = idx_out;
   p.obs = out->obs; p.act = out->act; p.rew = out->rew; p.next_obs = out->next_obs; p.done = out->done; p.ver = out->ver;
   p.stats = x->dstats;
-  if ((e = launch_sample_gather(p, x->stream)) != cudaSuccess) return cuda_fail(x, e, "sample and gather");
+  if ((e = launch_sample_gather(p, x->lstream)) != cudaSuccess) return cuda_fail(x, e, "sample and gather");
+  if (x->two_stream) { cudaEventRecord(x->ev_sample, x->lstream); x->has_sample = true; }
   x->k += 1;
   x->hs.learner_steps += 1;
   x->hs.consumed += c.minibatch;
@@ -543,25 +612,27 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
         t.wtc = which == 0 ? x->wtc[x->active] : x->wtc_target;
         t.b1 = W + x->wl.off_b1; t.b2 = W + x->wl.off_b2; t.b3 = W + x->wl.off_b3;
         t.out = x->tdq[which]; t.error = &x->dstats->error;
-        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1);
-        if ((e = launch_tc_mlp(t, x->sm_count, x->stream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
+        LaunchScope scope(x, TJ_K_MLP_TENSOR, 1, true, true);
+        if ((e = launch_tc_mlp(t, x->sm_count, x->lstream)) != cudaSuccess) return cuda_fail(x, e, "TD error (tensor-core forward)");
       }
-      LaunchScope scope(x, TJ_K_TD, 1);
+      LaunchScope scope(x, TJ_K_TD, 1, true, true);
       if ((e = launch_td_from_q(x->tdq[0], x->tdq[1], rows, x->A, b->act + r0, b->rew + r0, b->done + r0, p.gamma, p.kappa,
                                 td_out ? td_out + r0 : nullptr, huber_out ? huber_out + r0 : nullptr,
-                                x->td_partial + r0 / 16, x->stream)) != cudaSuccess)
+                                x->td_partial + r0 / 16, x->lstream)) != cudaSuccess)
         return cuda_fail(x, e, "TD error (elementwise)");
     }
     if (loss_mean_out) {
-      LaunchScope scope(x, TJ_K_TD, 1);
-      if ((e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
+      LaunchScope scope(x, TJ_K_TD, 1, true, true);
+      if ((e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->lstream)) != cudaSuccess)
         return cuda_fail(x, e, "TD error (loss reduction)");
     }
+    learner_launched(x);
     return TJ_OK;
   }
-  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1);
-  e = launch_td(p, x->stream);
+  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1, true, true);
+  e = launch_td(p, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -576,11 +647,12 @@ int tj_td_error_static(tj_ctx* x, const tj_batch* b, float* td_out, float* huber
   }
   const TdParams p = td_params(x, b, td_out, huber_out, loss_mean_out, nullptr);
   bool too_large = false;
-  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1, /*may_create=*/false);
-  cudaError_t e = launch_td_static(p, x->cfg.device, x->stream, &too_large);
+  LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1, /*may_create=*/false, true);
+  cudaError_t e = launch_td_static(p, x->cfg.device, x->lstream, &too_large);
   if (too_large) return fail(x, TJ_ERR_INVALID_ARG, "tj_td_error_static: batch too large for the library's scratch");
   if (e == cudaErrorInvalidDevice) return fail(x, TJ_ERR_INVALID_ARG, "tj_td_error_static: the context's device must be the current device");
   if (e != cudaSuccess) return cuda_fail(x, e, "TD error (library scratch)");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -614,11 +686,12 @@ int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const f
   lay_out_update_scratch(x, p);
   p.ldg = x->A; p.value_head = 0;
   p.error = &x->dstats->error;
-  LaunchScope scope(x, TJ_K_SGD, tj::sgd_step_launches(p) + (loss_mean_out ? 1 : 0));
-  cudaError_t e = launch_sgd_step(p, lr, adam, x->stream);
+  LaunchScope scope(x, TJ_K_SGD, tj::sgd_step_launches(p) + (loss_mean_out ? 1 : 0), true, true);
+  cudaError_t e = launch_sgd_step(p, lr, adam, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "learner update");
-  if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->stream)) != cudaSuccess)
+  if (loss_mean_out && (e = launch_td_finish(p.partial, sgd_partial_count(b->n), b->n, loss_mean_out, x->lstream)) != cudaSuccess)
     return cuda_fail(x, e, "learner update (loss reduction)");
+  learner_launched(x);
   return TJ_OK;
 }
 }  // namespace
@@ -668,9 +741,10 @@ int tj_ppo_step(tj_ctx* x, const tj_ppo_batch* b, float lr, float beta1, float b
   a.m = m; a.v = v; a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
   a.c1 = (float)(1.0 - std::pow((double)beta1, (double)t));
   a.c2 = (float)(1.0 - std::pow((double)beta2, (double)t));
-  LaunchScope scope(x, TJ_K_SGD, tj::ppo_step_launches(p, stats_out != nullptr));
-  cudaError_t e = launch_ppo_step(p, lr, &a, stats_out, x->stream);
+  LaunchScope scope(x, TJ_K_SGD, tj::ppo_step_launches(p, stats_out != nullptr), true, true);
+  cudaError_t e = launch_ppo_step(p, lr, &a, stats_out, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "PPO update");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -680,9 +754,10 @@ int tj_gae(tj_ctx* x, const float* rew, const float* val, const uint8_t* done, i
   if (!rew || !val || !done || !adv_out || !ret_out) return fail(x, TJ_ERR_INVALID_ARG, "GAE arrays must not be null");
   if (T < 0 || N < 0) return fail(x, TJ_ERR_INVALID_ARG, "T and N must not be negative");
   if (T == 0 || N == 0) return TJ_OK;
-  LaunchScope scope(x, TJ_K_GAE, 1);
-  cudaError_t e = launch_gae(rew, val, done, T, N, gamma, lambda, adv_out, ret_out, x->stream);
+  LaunchScope scope(x, TJ_K_GAE, 1, true, true);
+  cudaError_t e = launch_gae(rew, val, done, T, N, gamma, lambda, adv_out, ret_out, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "GAE");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -713,6 +788,7 @@ int tj_segment_acquire(tj_ctx* x, tj_segment* out) {
     out->val = x->seg_val + slot * ((size_t)T + 1) * N;
     sl.state = 3;
     sl.acquired_index = sl.index;
+    learner_waits_for_actor(x);
     x->next_consume += 1;
     x->k += 1;
     x->hs.learner_steps += 1;
@@ -731,9 +807,10 @@ int tj_normalize(tj_ctx* x, const float* in, int64_t n, float eps, float* out) {
   if (!in || !out) return fail(x, TJ_ERR_INVALID_ARG, "arrays must not be null");
   if (n < 0 || !(eps >= 0.f)) return fail(x, TJ_ERR_INVALID_ARG, "n and eps must not be negative");
   if (n == 0) return TJ_OK;
-  LaunchScope scope(x, TJ_K_GAE, 3);
-  cudaError_t e = launch_normalize(in, n, (double)eps, out, x->norm_scratch, x->stream);
+  LaunchScope scope(x, TJ_K_GAE, 3, true, true);
+  cudaError_t e = launch_normalize(in, n, (double)eps, out, x->norm_scratch, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "normalisation");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -753,9 +830,10 @@ int tj_segment_minibatch(tj_ctx* x, const tj_segment* segv, const float* adv, co
   p.shuffle_id = shuffle_id;
   p.seg_obs = segv->obs; p.seg_act = segv->act; p.seg_logp = segv->logp; p.adv_in = adv; p.ret_in = ret;
   p.obs = out->obs; p.act = out->act; p.logp = out->logp_old; p.adv = out->adv; p.ret = out->ret; p.row = out->row;
-  LaunchScope scope(x, TJ_K_SAMPLE, 1);
-  cudaError_t e = launch_segment_minibatch(p, x->stream);
+  LaunchScope scope(x, TJ_K_SAMPLE, 1, true, true);
+  cudaError_t e = launch_segment_minibatch(p, x->lstream);
   if (e != cudaSuccess) return cuda_fail(x, e, "segment minibatch");
+  learner_launched(x);
   return TJ_OK;
 }
 
@@ -805,7 +883,8 @@ int tj_set_state(tj_ctx* x, const tj_state_view* in) {
 int tj_stats(tj_ctx* x, tj_stats_t* o) {
   if (!x || !o) return TJ_ERR_INVALID_ARG;
   DevStats d;
-  cudaError_t e = cudaMemcpyAsync(&d, x->dstats, sizeof(d), cudaMemcpyDeviceToHost, x->stream);
+  cudaError_t e = x->two_stream ? cudaStreamSynchronize(x->lstream) : cudaSuccess;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&d, x->dstats, sizeof(d), cudaMemcpyDeviceToHost, x->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->stream);
   if (e != cudaSuccess) return cuda_fail(x, e, "read counters");
   drain_spans(x);

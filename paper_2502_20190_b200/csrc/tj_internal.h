@@ -256,7 +256,13 @@ struct SegSlot {
 
 struct tj_ctx {
   tj_config cfg;
-  cudaStream_t stream;
+  cudaStream_t stream;        // actor stream (and everything else while no learner stream is set)
+  cudaStream_t lstream;       // learner stream: sample, gather, TD error, updates, GAE, publish
+  bool two_stream;            // lstream differs from stream: the hand-overs below order the two
+  // hand-overs between the streams (Sec. 3.1: dependencies I and III as asynchronous exchanges): each event is recorded
+  // on one stream after the launches of a call and awaited by the other stream before the launches that depend on them
+  cudaEvent_t ev_actor, ev_sample, ev_publish, ev_learner;
+  bool has_actor, has_sample, has_publish, has_learner;
   int N, D, H, A, S_d, value_head, rec_words, max_ep;
   size_t n_blob;
   tj::WeightLayout wl;

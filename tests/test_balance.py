@@ -60,3 +60,22 @@ def test_starved_share_matches_the_oracle_sampler(S, publishes):
             ver += 1
             o.publish(synth.policy_blob(3, ver, D, H, A))
     assert starved / calls == pytest.approx(balance.starved_fraction(S, publishes))
+
+
+def test_balanced_cadence_for_concurrent_streams():
+    """Eq. 3's TR_L ~ TR_A for two streams: the faster side takes as many steps as fit into one step of the slower one."""
+    c = balance.balanced_cadence(actor_step_s=100e-6, learner_step_s=25e-6, minibatch=1024, n_envs=4096, staleness_bound=8)
+    assert (c["actor_steps"], c["learner_steps"]) == (1, 4) and c["idle_share"] == pytest.approx(0.0)
+    assert c["P"] == pytest.approx(4 * 1024 / 4096)
+    c = balance.balanced_cadence(actor_step_s=10e-6, learner_step_s=72e-6, minibatch=256, n_envs=64, staleness_bound=4)
+    assert (c["actor_steps"], c["learner_steps"]) == (7, 1) and c["idle_share"] < 0.05
+    # both streams busy for about the same time: no other small-integer cadence with one side at 1 idles less
+    for k in range(1, 20):
+        assert abs(k * 10e-6 - 72e-6) / max(k * 10e-6, 72e-6) >= c["idle_share"] - 1e-12
+    # bound 0 ("all samples new") cannot overlap production and consumption: lock step
+    c0 = balance.balanced_cadence(10e-6, 72e-6, 256, 64, staleness_bound=0)
+    assert (c0["actor_steps"], c0["learner_steps"]) == (1, 1)
+    with pytest.raises(ValueError):
+        balance.balanced_cadence(0.0, 1.0, 1, 1, 1)
+    a, l = balance.step_times_from_stats(dict(kernel_ms=[8.0, 0, 0, 1.0, 2.0, 0.5, 0, 0.5]), actor_steps=4, learner_steps=2)
+    assert a == pytest.approx(2e-3) and l == pytest.approx(2e-3)
