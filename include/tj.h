@@ -61,7 +61,13 @@ typedef enum {
 
 enum { TJ_ENV_CARTPOLE = 0, TJ_ENV_ACROBOT = 1, TJ_ENV_LINGAUSS = 2 };
 enum { TJ_POLICY_EPS_GREEDY = 0, TJ_POLICY_CATEGORICAL = 1 };
-enum { TJ_W_FP32 = 0, TJ_W_BF16 = 1 };
+enum { TJ_W_FP32 = 0,      /* FP32 FMA in one fixed rounding order: outputs (and actions) reproducible bit for bit */
+       TJ_W_BF16 = 1,      /* weight matrices rounded to bfloat16, tensor cores, FP32 accumulation: 2e-2 */
+       TJ_W_FP32_TC = 2 }; /* FP32 weights; the actor's hidden x hidden layer on the tensor cores as three products of split
+                              operands (the role a 3 x TF32 product plays, here with FP16 parts at twice that rate; about
+                              2^-22 per term): outputs within 1e-5 of TJ_W_FP32's, actions equal wherever the top-2 gap
+                              exceeds that.  CartPole / Acrobot, hidden 64 / 128 / 192 / 256.  The learner-side calls
+                              (tj_td_error, updates) use the FP32 kernels. */
 /* kernel classes reported by tj_stats (Sec. 3.3: performance analysis measures the production and the
  * consumption side separately) */
 enum { TJ_K_ACTOR_FUSED = 0,  /* MLP + selection + env step + insert in one kernel (FP32 path, or the fused tensor-core actor) */
@@ -90,7 +96,7 @@ typedef struct {
   /* model group */
   int32_t hidden;                /* H, width of both hidden ReLU layers (1..768) */
   int32_t policy_kind;           /* TJ_POLICY_*: Q head, or softmax head + value head */
-  int32_t weight_dtype;          /* TJ_W_FP32: FP32 FMA in a fixed rounding order; TJ_W_BF16: tensor cores */
+  int32_t weight_dtype;          /* TJ_W_* */
   float epsilon;                 /* exploration rate (eps-greedy) */
   uint64_t seed;                 /* Philox key */
   /* training / distribution group */

@@ -54,7 +54,10 @@ const char* validate(const tj_config* c) {
       return "unknown env_kind";
   }
   if (c->policy_kind != TJ_POLICY_EPS_GREEDY && c->policy_kind != TJ_POLICY_CATEGORICAL) return "unknown policy_kind";
-  if (c->weight_dtype != TJ_W_FP32 && c->weight_dtype != TJ_W_BF16) return "unknown weight_dtype";
+  if (c->weight_dtype != TJ_W_FP32 && c->weight_dtype != TJ_W_BF16 && c->weight_dtype != TJ_W_FP32_TC) return "unknown weight_dtype";
+  if (c->weight_dtype == TJ_W_FP32_TC &&
+      !split_actor_supported(c->env_kind, c->obs_dim, c->hidden, c->n_actions + (c->policy_kind == TJ_POLICY_CATEGORICAL ? 1 : 0)))
+    return "TJ_W_FP32_TC needs CartPole or Acrobot and a hidden width of 64, 128, 192 or 256";
   if (!(c->epsilon >= 0.f && c->epsilon <= 1.f)) return "epsilon must lie in [0,1]";
   if (c->max_episode_steps < 0) return "max_episode_steps must not be negative";
   if (c->replay_capacity < 0) return "replay_capacity must not be negative";
@@ -126,6 +129,13 @@ size_t carve(tj_ctx* x, void* base) {
     x->lgAt = cv.take<float>((size_t)D * round_up4(D));
     x->lgB = cv.take<float>((size_t)c.n_actions * round_up4(D));
     x->lg_stage = cv.take<float>((size_t)D * D + (size_t)c.n_actions * D);
+  }
+  x->use_split = c.weight_dtype == TJ_W_FP32_TC;
+  if (x->use_split) {
+    for (int i = 0; i < 2; ++i) {
+      x->wsplit[i] = cv.take<uint16_t>(split_weight_halfs(c.hidden));
+      x->wsplit_scale[i] = cv.take<float>(2);
+    }
   }
   x->use_tc = c.weight_dtype == TJ_W_BF16 && tc_mlp_supported(D, c.hidden, c.n_actions + vh);
   if (x->use_tc) {
@@ -391,11 +401,16 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
       return cuda_fail(x, e, "publish: host to device copy");
     src = x->blob_stage;
   }
-  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : 1), true, true);
+  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : (x->use_split ? 3 : 1)), true, true);
   const int next = x->active ^ 1;
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
   if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->lstream)) != cudaSuccess)
     return cuda_fail(x, e, "publish: repack");
+  if (x->use_split) {
+    const int slot = x->version == 0 ? x->active : next;
+    if ((e = launch_pack_split_weights(src, x->D, x->H, x->wsplit[slot], x->wsplit_scale[slot], x->lstream)) != cudaSuccess)
+      return cuda_fail(x, e, "publish: split of the hidden x hidden matrix");
+  }
   uint16_t* dst_tc = nullptr;
   if (x->use_tc) {
     dst_tc = x->version == 0 ? x->wtc[x->active] : x->wtc[next];
@@ -500,6 +515,9 @@ int tj_actor_step(tj_ctx* x, int32_t n_steps, float* dbg_logits) {
       LaunchScope scope(x, TJ_K_ENV, 1);
       e = launch_actor(c.env_kind, q, x->stream);
     }
+  } else if (x->use_split) {
+    LaunchScope scope(x, TJ_K_ACTOR_FUSED, 1);
+    e = launch_actor_split(c.env_kind, p, x->wsplit[x->active], x->wsplit_scale[x->active], x->sm_count, x->stream);
   } else {
     LaunchScope scope(x, TJ_K_ACTOR_FUSED, 1);
     e = launch_actor(c.env_kind, p, x->stream);

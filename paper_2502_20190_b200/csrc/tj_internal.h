@@ -241,6 +241,12 @@ int shuffle_half_bits(long long R);
 size_t normalize_scratch_doubles();
 cudaError_t launch_normalize(const float* x, long long n, double eps, float* out, double* scratch, cudaStream_t s);
 cudaError_t launch_segment_minibatch(const MinibatchParams& p, cudaStream_t s);
+// FP32-accuracy tensor-core actor for the small envs (hidden x hidden layer as three FP16 products of split operands)
+bool split_actor_supported(int env_kind, int D, int H, int Aout);
+size_t split_weight_halfs(int H);
+cudaError_t launch_pack_split_weights(const float* blob, int D, int H, uint16_t* dst, float* scale, cudaStream_t s);
+cudaError_t launch_actor_split(int env_kind, const ActorParams& p, const uint16_t* w2parts, const float* w2scale, int sm_count,
+                               cudaStream_t s);
 size_t fma_rate_sink_floats(int sm_count);
 double launch_fma_rate(float* sink, int sm_count, int outer, cudaStream_t s, cudaError_t* err);
 cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);
@@ -285,6 +291,10 @@ struct tj_ctx {
   float* lgAt;
   float* lgB;
   float* lg_stage;
+  // FP32-accuracy tensor-core actor (TJ_W_FP32_TC): W2's FP16 parts and their scales, double buffered like wbuf
+  bool use_split;
+  uint16_t* wsplit[2];
+  float* wsplit_scale[2];
   // tensor-core path (BF16 weights, supported shapes only)
   bool use_tc;
   int sm_count;

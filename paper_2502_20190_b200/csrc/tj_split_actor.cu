@@ -1,0 +1,435 @@
+// FP32-accuracy tensor-core actor for the small environments (CartPole, Acrobot) with hidden widths of 64 .. 256: the
+// hidden x hidden layer -- the one dense contraction of these networks (Algorithm 1, task 1: 65,536 of a 6-256-256-3
+// network's 67,840 multiply-adds per env step) -- runs on the tensor cores as three FP16 products of split operands,
+//   W2 h1 = W_hi h_hi + W_hi h_lo + W_lo h_hi,   x = x_hi + x_lo with x_hi the 11 leading bits of the (power-of-two scaled) value,
+// with FP32 accumulation in tensor memory (error about 2^-22 per term, the dropped lo x lo term; FP16 runs at twice the rate
+// of the 3 x TF32 form of the same idea).  Layer 1 (4 or 6 inputs) and the head (2-4 outputs) stay on the FP32 pipes.
+//
+// One thread block keeps a tile of 128 environments for all n_steps of the call (environments are independent): thread e
+// owns env e's state in registers, all 256 threads compute layer 1 and drain the accumulator.  Per step:
+//   observation -> shared memory;  layer 1 in the fixed FMA order of the FP32 path, ReLU, split -> FP16 A operand (128 rows x H);
+//   one lane streams W2's parts in 32-column chunks (bulk copies, four ring slots, the stream running on across steps) and
+//   issues the MMAs (M = 128, N = H);  accumulator -> + b2, ReLU, head partial sums by two threads per row -> outputs;
+//   then exactly the FP32 kernel's selection, env step, record / segment write and reset.
+// Every wait is bounded; a timeout latches the context's error word and the block leaves after freeing its tensor memory.
+#include <cuda_fp16.h>
+
+#include "tj_internal.h"
+#include "tj_mlp.cuh"
+#include "tj_tc.cuh"
+
+namespace tj {
+
+namespace {
+
+constexpr int SA_TE = 128;            // envs per tile = rows of the MMA
+constexpr int SA_NT = 256;
+constexpr int SA_KC = 32;             // K columns per streamed chunk of W2
+constexpr int SA_SLOTS = 4;
+constexpr float SA_H_SCALE = 16.0f;   // hidden activations are split after this scaling (|h1| < 4,094 stays inside FP16)
+
+struct SaCtl {
+  uint64_t full[SA_SLOTS], empty[SA_SLOTS];
+  uint64_t wbar;          // small parameters staged
+  uint64_t acc_full;      // all MMAs of a forward pass complete
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ float4 sa_reset4(uint2 seed, uint32_t e, unsigned long long step, float lo, float width) {
+  const uint4 w = stream_words(seed, STREAM_RESET, 0, e, step);
+  return make_float4(uniform_range(w.x, lo, width), uniform_range(w.y, lo, width), uniform_range(w.z, lo, width),
+                     uniform_range(w.w, lo, width));
+}
+
+template <int ENV>
+__device__ __forceinline__ void sa_observe(float4 s, float* obs) {
+  if (ENV == TJ_ENV_CARTPOLE) {
+    obs[0] = s.x; obs[1] = s.y; obs[2] = s.z; obs[3] = s.w; obs[4] = obs[5] = 0.f;
+  } else {
+    float s1, c1, s2, c2;
+    sincosf(s.x, &s1, &c1);
+    sincosf(s.y, &s2, &c2);
+    obs[0] = c1; obs[1] = s1; obs[2] = c2; obs[3] = s2; obs[4] = s.z; obs[5] = s.w;
+  }
+}
+
+struct SaShared {
+  uint8_t *a_hi, *a_lo, *ring;
+  float *xs, *out, *part;
+  SaCtl* ctl;
+  int a_bytes, chunk_bytes, n_chunks;
+};
+
+// Network outputs of the observations in xs -> out[i][e], i < Aout.  Called by every thread of the block; `pass` counts the
+// calls, `copied` / `used` are the issuing lane's positions in the chunk stream.  Returns false after a timeout.
+__device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeights& mw, const SaShared& sh, const uint16_t* w2parts,
+                                           float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied, uint32_t& used,
+                                           volatile int* abort_flag) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = p.H, D = p.D;
+  // layer 1 in the canonical order (bias, then inputs in index order), ReLU, scale, split, FP16 A operand rows
+  {
+    const int e = tid & (SA_TE - 1), half = tid >> 7;
+    const int n_lo = half * (H / 2), n_hi = n_lo + H / 2;
+    float x[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) x[k] = k < D ? sh.xs[k * SA_TE + e] : 0.f;
+    for (int n0 = n_lo; n0 < n_hi; n0 += 8) {
+      float acc[8];
+      const float4 b0 = *reinterpret_cast<const float4*>(mw.b1 + n0), b1 = *reinterpret_cast<const float4*>(mw.b1 + n0 + 4);
+      acc[0] = b0.x; acc[1] = b0.y; acc[2] = b0.z; acc[3] = b0.w; acc[4] = b1.x; acc[5] = b1.y; acc[6] = b1.z; acc[7] = b1.w;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (k < D) {
+          const float4 w0 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * p.Hp + n0);
+          const float4 w1 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * p.Hp + n0 + 4);
+          acc[0] = fmaf(w0.x, x[k], acc[0]); acc[1] = fmaf(w0.y, x[k], acc[1]); acc[2] = fmaf(w0.z, x[k], acc[2]); acc[3] = fmaf(w0.w, x[k], acc[3]);
+          acc[4] = fmaf(w1.x, x[k], acc[4]); acc[5] = fmaf(w1.y, x[k], acc[5]); acc[6] = fmaf(w1.z, x[k], acc[6]); acc[7] = fmaf(w1.w, x[k], acc[7]);
+        }
+      }
+      uint32_t hi2[4], lo2[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float v0 = fmaxf(acc[2 * i], 0.f) * SA_H_SCALE, v1 = fmaxf(acc[2 * i + 1], 0.f) * SA_H_SCALE;
+        const float h0 = __uint_as_float(__float_as_uint(v0) & 0xFFFFE000u), h1 = __uint_as_float(__float_as_uint(v1) & 0xFFFFE000u);
+        hi2[i] = pack_f16x2(h0, h1);
+        lo2[i] = pack_f16x2(v0 - h0, v1 - h1);
+      }
+      const size_t off = ((size_t)(e >> 3) * (H / 8) + (n0 >> 3)) * 128 + (e & 7) * 16;
+      *reinterpret_cast<uint4*>(sh.a_hi + off) = make_uint4(hi2[0], hi2[1], hi2[2], hi2[3]);
+      *reinterpret_cast<uint4*>(sh.a_lo + off) = make_uint4(lo2[0], lo2[1], lo2[2], lo2[3]);
+    }
+  }
+  fence_async_smem();
+  tc_fence_before();
+  __syncthreads();   // A operand complete; every thread has finished reading the previous pass's accumulator
+  if (tid == 0) {
+    // hidden x hidden layer: per chunk of 32 columns two K steps; the high parts of W2 meet both parts of h1, the low
+    // parts only h1's high part.  After the MMAs of chunk g are issued, the slot of chunk g - 1 is refilled with chunk
+    // g + 3 of the (cyclic) stream, so three copies are in flight while a chunk is multiplied.
+    const uint32_t idesc = make_idesc_f16(H);
+    const uint32_t ahi_lo = desc_lo(smem_addr(sh.a_hi), 128u), alo_lo = desc_lo(smem_addr(sh.a_lo), 128u);
+    const uint32_t a_hiword = desc_hi((uint32_t)(H / 8) * 128u), b_hiword = desc_hi((uint32_t)(SA_KC / 8) * 128u);
+    const uint32_t ring_lo = desc_lo(smem_addr(sh.ring), 128u);
+    tc_fence_after();
+    for (int c = 0; c < sh.n_chunks; ++c, ++used) {
+      const uint32_t s = used % SA_SLOTS;
+      if (!tc_wait(&sh.ctl->full[s], (used / SA_SLOTS) & 1, abort_flag)) break;
+      const bool low_part = c >= sh.n_chunks / 2;
+      const int kc = c % (sh.n_chunks / 2);
+      const uint32_t b_lo = ring_lo + s * (uint32_t)(sh.chunk_bytes / 16);
+#pragma unroll
+      for (int j = 0; j < SA_KC / 16; ++j) {
+        const uint32_t a_off = (uint32_t)(kc * (SA_KC / 8) + 2 * j) * 8u;        // in 16-byte units: 8 per core matrix
+        umma_ss(tmem, ahi_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, (c | j) != 0);
+        if (!low_part) umma_ss(tmem, alo_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, 1u);
+      }
+      umma_commit(&sh.ctl->empty[s]);
+      if (used >= 1) {
+        // chunk `copied` goes into the slot chunk `used - 1` occupied (copied = used - 1 + SLOTS)
+        const uint32_t sp = copied % SA_SLOTS;
+        if (!tc_wait(&sh.ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(&sh.ctl->full[sp], (uint32_t)sh.chunk_bytes);
+        bulk_copy_g2s(sh.ring + (size_t)sp * sh.chunk_bytes,
+                      reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % (uint32_t)sh.n_chunks) * sh.chunk_bytes,
+                      (uint32_t)sh.chunk_bytes, &sh.ctl->full[sp]);
+        ++copied;
+      }
+    }
+    umma_commit(&sh.ctl->acc_full);
+  }
+  if (!tc_wait_warp(&sh.ctl->acc_full, pass & 1, abort_flag)) return false;
+  tc_fence_after();
+  // drain: two threads per row (the two column halves); h2 = relu(acc / scale + b2), head partial sums in column order
+  {
+    const int q = warp & 3, half = warp >> 2, r = q * 32 + lane;
+    float pa[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
+    for (int c0 = half * (H / 2); c0 < (half + 1) * (H / 2); c0 += 16) {
+      uint32_t v[16];
+      tmem_ld16(t_row + (uint32_t)c0, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float h2 = fmaxf(fmaf(__uint_as_float(v[i]), inv_scale, mw.b2[c0 + i]), 0.f);
+        const float* w3 = mw.W3t + (size_t)(c0 + i) * p.Ap;
+        if (p.Ap == 4) {
+          const float4 w = *reinterpret_cast<const float4*>(w3);
+          pa[0] = fmaf(w.x, h2, pa[0]); pa[1] = fmaf(w.y, h2, pa[1]); pa[2] = fmaf(w.z, h2, pa[2]); pa[3] = fmaf(w.w, h2, pa[3]);
+        } else {
+          for (int a = 0; a < p.Aout && a < 4; ++a) pa[a] = fmaf(w3[a], h2, pa[a]);
+        }
+      }
+    }
+    for (int a = 0; a < p.Aout; ++a) sh.part[((size_t)half * p.Ap + a) * SA_TE + r] = pa[a];
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid < SA_TE)
+    for (int a = 0; a < p.Aout; ++a)
+      sh.out[a * SA_TE + tid] = (mw.b3[a] + sh.part[(size_t)a * SA_TE + tid]) + sh.part[((size_t)p.Ap + a) * SA_TE + tid];
+  __syncthreads();
+  return true;
+}
+
+template <int ENV>
+__global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorParams p, const uint16_t* __restrict__ w2parts,
+                                                                 const float* __restrict__ w2scale) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int H = p.H, D = p.D;
+  SaShared sh;
+  sh.a_bytes = SA_TE * H * 2;                                 // one FP16 part of the A operand
+  sh.chunk_bytes = H * SA_KC * 2;                             // one chunk of one part of W2
+  sh.n_chunks = 2 * (H / SA_KC);                              // per forward pass: the high parts' chunks, then the low parts'
+  sh.a_hi = smem_raw;
+  sh.a_lo = sh.a_hi + sh.a_bytes;
+  sh.ring = sh.a_lo + sh.a_bytes;
+  float* wsm = reinterpret_cast<float*>(sh.ring + SA_SLOTS * sh.chunk_bytes);
+  const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);   // everything but the H x H matrix
+  sh.xs = wsm + staged;                                       // [D][TE]
+  sh.out = sh.xs + (size_t)((D + 3) & ~3) * SA_TE;            // [Ap][TE]
+  sh.part = sh.out + (size_t)p.Ap * SA_TE;                    // [2][Ap][TE]
+  sh.ctl = reinterpret_cast<SaCtl*>(sh.part + 2 * (size_t)p.Ap * SA_TE);
+  SaCtl* ctl = sh.ctl;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int n_tiles = (p.N + SA_TE - 1) / SA_TE;
+  const bool on_policy = p.C == 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < SA_SLOTS; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    mbar_init(&ctl->wbar, 1);
+    mbar_init(&ctl->acc_full, 1);
+    ctl->abort_flag = 0;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&ctl->tmem_base)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  const MlpWeights mw = stage_mlp_weights<1>(p, p.W, wsm, &ctl->wbar, tid == 0);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+  bool ok = tc_wait_warp(&ctl->wbar, 0, abort_flag);
+  ok = __syncthreads_and(ok);
+  const float inv_scale = w2scale[1];                         // 1 / (activation scale x weight scale)
+
+  uint32_t copied = 0, used = 0, pass = 0;                     // chunk stream positions (issuing lane), forward passes
+  if (tid == 0 && ok) {
+    for (; copied < SA_SLOTS; ++copied) {
+      mbar_expect_tx(&ctl->full[copied], (uint32_t)sh.chunk_bytes);
+      bulk_copy_g2s(sh.ring + (size_t)copied * sh.chunk_bytes,
+                    reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % (uint32_t)sh.n_chunks) * sh.chunk_bytes,
+                    (uint32_t)sh.chunk_bytes, &ctl->full[copied]);
+    }
+  }
+
+  unsigned long long n_episodes = 0;
+  double ret_sum = 0.0;
+  for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+    const int e = tile * SA_TE + tid;
+    const bool owner = tid < SA_TE && e < p.N;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    int ep = 0;
+    float ep_ret = 0.f;
+    if (owner) {
+      s = reinterpret_cast<const float4*>(p.state)[e];
+      ep = p.ep_step[e];
+      ep_ret = p.ep_return[e];
+    }
+    for (int step = 0; step < p.n_steps && ok; ++step) {
+      const unsigned long long t = (unsigned long long)p.t0 + step;
+      float obs[6];
+      sa_observe<ENV>(s, obs);
+      if (tid < SA_TE) {
+#pragma unroll
+        for (int k = 0; k < 6; ++k)
+          if (k < D) sh.xs[k * SA_TE + tid] = owner ? obs[k] : 0.f;
+      }
+      __syncthreads();
+      ok = sa_forward(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+      ok = __syncthreads_and(ok);
+      if (!ok) break;
+      if (owner) {
+        auto logit = [&](int i) { return sh.out[i * SA_TE + tid]; };
+        if (p.dbg_logits) {
+          float* dl = p.dbg_logits + ((size_t)step * p.N + e) * p.A;
+          for (int i = 0; i < p.A; ++i) dl[i] = logit(i);
+        }
+        const uint4 w = stream_words(p.seed, STREAM_ACTION, 0, (uint32_t)e, t);
+        int a;
+        float logp = 0.f;
+        if (p.policy_kind == TJ_POLICY_EPS_GREEDY) a = select_eps_greedy(p.A, logit, w, p.explore_thr);
+        else a = select_categorical(p.A, logit, u01(w.x), logp);
+        float4 sn;
+        const StepResult r = (ENV == TJ_ENV_CARTPOLE) ? cartpole_step(s, a, sn) : acrobot_step(s, a, sn);
+        ep += 1;
+        const int done = (r.terminated || ep >= p.max_ep) ? 1 : 0;
+        if (on_policy) {
+          const long long g = (long long)(t / (unsigned long long)p.T);
+          const int pos = (int)(t % (unsigned long long)p.T);
+          const int slot = (int)(g % p.G);
+          const size_t i = ((size_t)slot * p.T + pos) * p.N + e;
+          float* so = p.seg_obs + i * p.D;
+          if (ENV == TJ_ENV_CARTPOLE) *reinterpret_cast<float4*>(so) = s;
+          else
+            for (int k = 0; k < 6; ++k) so[k] = obs[k];
+          p.seg_act[i] = a;
+          p.seg_rew[i] = r.reward;
+          p.seg_done[i] = (uint8_t)done;
+          p.seg_logp[i] = logp;
+          p.seg_val[((size_t)slot * (p.T + 1) + pos) * p.N + e] = logit(p.A);  // value head = column A
+        } else {
+          const unsigned long long slot = (p.cursor0 + (unsigned long long)step * p.N + e) % (unsigned long long)p.C;
+          float4* rec = reinterpret_cast<float4*>(p.ring + slot * p.rec_words);
+          const float4 tail = make_float4(__int_as_float(a), r.reward, __int_as_float(done), __int_as_float(p.version));
+          if (ENV == TJ_ENV_CARTPOLE) {
+            rec[0] = s;
+            rec[1] = sn;
+            rec[2] = tail;
+          } else {
+            float s1, c1, s2, c2;
+            sincosf(sn.x, &s1, &c1);
+            sincosf(sn.y, &s2, &c2);
+            rec[0] = make_float4(obs[0], obs[1], obs[2], obs[3]);
+            rec[1] = make_float4(obs[4], obs[5], c1, s1);
+            rec[2] = make_float4(c2, s2, sn.z, sn.w);
+            rec[3] = tail;
+          }
+        }
+        ep_ret += r.reward;
+        if (done) {
+          n_episodes += 1;
+          ret_sum += (double)ep_ret;
+          ep_ret = 0.f;
+          ep = 0;
+          s = (ENV == TJ_ENV_CARTPOLE) ? sa_reset4(p.seed, (uint32_t)e, t, -0.05f, 0.1f) : sa_reset4(p.seed, (uint32_t)e, t, -0.1f, 0.2f);
+        } else {
+          s = sn;
+        }
+      }
+      if (!on_policy && tile == 0 && tid == 0)
+        p.block_ver[((p.cursor0 + (unsigned long long)step * p.N) % (unsigned long long)p.C) / p.N] = p.version;
+      // last step of a segment: bootstrap value of the state each env is now in
+      if (on_policy && (int)(t % (unsigned long long)p.T) == p.T - 1) {
+        float o2[6];
+        sa_observe<ENV>(s, o2);
+        __syncthreads();
+        if (tid < SA_TE) {
+#pragma unroll
+          for (int k = 0; k < 6; ++k)
+            if (k < D) sh.xs[k * SA_TE + tid] = owner ? o2[k] : 0.f;
+        }
+        __syncthreads();
+        ok = sa_forward(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        if (owner) {
+          const int slot = (int)((long long)(t / (unsigned long long)p.T) % p.G);
+          p.seg_val[((size_t)slot * (p.T + 1) + p.T) * p.N + e] = sh.out[p.A * SA_TE + tid];
+        }
+      }
+      __syncthreads();
+    }
+    if (owner) {
+      reinterpret_cast<float4*>(p.state)[e] = s;
+      p.ep_step[e] = ep;
+      p.ep_return[e] = ep_ret;
+    }
+  }
+  if (tid < SA_TE && n_episodes) {
+    atomicAdd(&p.stats->episodes, n_episodes);
+    atomicAdd(&p.stats->return_sum, ret_sum);
+  }
+  // the copies still in flight must land before the block gives its shared memory back
+  if (tid == 0) {
+    for (uint32_t g = used; g < copied; ++g)
+      if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
+    if (ctl->abort_flag) atomicExch(&p.stats->error, 4ull);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  }
+}
+
+// W2 [H][H] (row = neuron) -> scaled FP16 high and low parts, each as H / 32 chunks of H rows x 32 columns in the K-major
+// core-matrix layout: element (n, k) of chunk kc sits at ((n / 8) * 4 + (k % 32) / 8) * 64 + (n % 8) * 8 + k % 8.
+// scale_out[0] = the power of two the weights were multiplied by, scale_out[1] = 1 / (that x the activation scale).
+__global__ void split_scale_kernel(const float* __restrict__ blob, int D, int H, float* __restrict__ scale_out) {
+  __shared__ float wmax[32];
+  const float* W2 = blob + (size_t)H * D + H;
+  float m = 0.f;
+  for (int i = threadIdx.x; i < H * H; i += blockDim.x) m = fmaxf(m, fabsf(W2[i]));
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_down_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) m = fmaxf(m, wmax[w]);
+    // largest entry into [1024, 2048): far inside FP16's range, low parts of all but the tiniest entries normal
+    int e = 0;
+    if (m > 0.f && isfinite(m)) e = 10 - (int)floorf(log2f(m));
+    e = e < -24 ? -24 : (e > 24 ? 24 : e);
+    const float sc = exp2f((float)e);
+    scale_out[0] = sc;
+    scale_out[1] = 1.0f / (sc * SA_H_SCALE);
+  }
+}
+
+__global__ void split_pack_kernel(const float* __restrict__ blob, int D, int H, const float* __restrict__ scale, uint16_t* __restrict__ dst) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= H * H) return;
+  const float* W2 = blob + (size_t)H * D + H;
+  const int chunk = i / (H * SA_KC), within = i % (H * SA_KC);
+  const int core = within / 64, in_core = within % 64;
+  const int rg = core / (SA_KC / 8), kg = core % (SA_KC / 8);
+  const int n = rg * 8 + in_core / 8, k = chunk * SA_KC + kg * 8 + in_core % 8;
+  const float v = W2[(size_t)n * H + k] * scale[0];
+  const __half hi = __float2half_rn(v);
+  const __half lo = __float2half_rn(v - __half2float(hi));
+  dst[i] = __half_as_ushort(hi);
+  dst[(size_t)H * H + i] = __half_as_ushort(lo);
+}
+
+}  // namespace
+
+bool split_actor_supported(int env_kind, int D, int H, int Aout) {
+  return (env_kind == TJ_ENV_CARTPOLE || env_kind == TJ_ENV_ACROBOT) && D <= 8 && H >= 64 && H <= 256 && H % 64 == 0 && Aout <= 4;
+}
+
+size_t split_weight_halfs(int H) { return (size_t)2 * H * H; }
+
+cudaError_t launch_pack_split_weights(const float* blob, int D, int H, uint16_t* dst, float* scale, cudaStream_t s) {
+  split_scale_kernel<<<1, 1024, 0, s>>>(blob, D, H, scale);
+  split_pack_kernel<<<(H * H + 255) / 256, 256, 0, s>>>(blob, D, H, scale, dst);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_actor_split(int env_kind, const ActorParams& p, const uint16_t* w2parts, const float* w2scale, int sm_count,
+                               cudaStream_t s) {
+  if (p.N <= 0) return cudaSuccess;
+  if (!split_actor_supported(env_kind, p.D, p.H, p.Aout)) return cudaErrorInvalidConfiguration;
+  const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);
+  const size_t smem = (size_t)2 * SA_TE * p.H * 2 + (size_t)SA_SLOTS * p.H * SA_KC * 2 +
+                      (staged + (size_t)((p.D + 3) & ~3) * SA_TE + 3 * (size_t)p.Ap * SA_TE) * sizeof(float) + sizeof(SaCtl) + 64;
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  const int n_tiles = (p.N + SA_TE - 1) / SA_TE;
+  const int grid = n_tiles < sm_count ? n_tiles : sm_count;
+  cudaError_t e;
+  if (env_kind == TJ_ENV_CARTPOLE) {
+    if ((e = cudaFuncSetAttribute(actor_split_tc_kernel<TJ_ENV_CARTPOLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    actor_split_tc_kernel<TJ_ENV_CARTPOLE><<<grid, SA_NT, smem, s>>>(p, w2parts, w2scale);
+  } else {
+    if ((e = cudaFuncSetAttribute(actor_split_tc_kernel<TJ_ENV_ACROBOT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    actor_split_tc_kernel<TJ_ENV_ACROBOT><<<grid, SA_NT, smem, s>>>(p, w2parts, w2scale);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace tj

@@ -10,7 +10,7 @@ import numpy as np
 
 ENV_CARTPOLE, ENV_ACROBOT, ENV_LINGAUSS = 0, 1, 2
 POLICY_EPS_GREEDY, POLICY_CATEGORICAL = 0, 1
-W_FP32, W_BF16 = 0, 1
+W_FP32, W_BF16, W_FP32_TC = 0, 1, 2
 
 SEED = 0x25022019
 
