@@ -104,7 +104,10 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
   fence_async_smem();
   tc_fence_before();
   __syncthreads();   // A operand complete; every thread has finished reading the previous pass's accumulator
-  if (tid == 0) {
+  // The issuing lane's warp-mates wait at the warp barrier below, not in a polling loop: lanes of one warp that poll while
+  // another lane of it issues take turns with that lane, and every blocked poll then stalls the issue.
+  if (warp == 0) {
+   if (lane == 0) {
     // hidden x hidden layer: per chunk of 32 columns two K steps; the high parts of W2 meet both parts of h1, the low
     // parts only h1's high part.  After the MMAs of chunk g are issued, the slot of chunk g - 1 is refilled with chunk
     // g + 3 of the (cyclic) stream, so three copies are in flight while a chunk is multiplied.
@@ -138,8 +141,10 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
       }
     }
     umma_commit(&sh.ctl->acc_full);
+   }
+   __syncwarp();
   }
-  if (!tc_wait_warp(&sh.ctl->acc_full, pass & 1, abort_flag)) return false;
+  if (!tc_wait_elect(&sh.ctl->acc_full, pass & 1, abort_flag)) return false;
   tc_fence_after();
   // drain: two threads per row (the two column halves); h2 = relu(acc / scale + b2), head partial sums in column order
   {
@@ -153,22 +158,20 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const float h2 = fmaxf(fmaf(__uint_as_float(v[i]), inv_scale, mw.b2[c0 + i]), 0.f);
-        const float* w3 = mw.W3t + (size_t)(c0 + i) * p.Ap;
-        if (p.Ap == 4) {
-          const float4 w = *reinterpret_cast<const float4*>(w3);
-          pa[0] = fmaf(w.x, h2, pa[0]); pa[1] = fmaf(w.y, h2, pa[1]); pa[2] = fmaf(w.z, h2, pa[2]); pa[3] = fmaf(w.w, h2, pa[3]);
-        } else {
-          for (int a = 0; a < p.Aout && a < 4; ++a) pa[a] = fmaf(w3[a], h2, pa[a]);
-        }
+        const float* w3 = mw.W3t + (size_t)(c0 + i) * 4;
+        const float4 w = *reinterpret_cast<const float4*>(w3);      // Ap = 4: rows of W3t are one vector, zero beyond Aout
+        pa[0] = fmaf(w.x, h2, pa[0]); pa[1] = fmaf(w.y, h2, pa[1]); pa[2] = fmaf(w.z, h2, pa[2]); pa[3] = fmaf(w.w, h2, pa[3]);
       }
     }
-    for (int a = 0; a < p.Aout; ++a) sh.part[((size_t)half * p.Ap + a) * SA_TE + r] = pa[a];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+      if (a < p.Aout) sh.part[((size_t)half * 4 + a) * SA_TE + r] = pa[a];
   }
   tc_fence_before();
   __syncthreads();
   if (tid < SA_TE)
     for (int a = 0; a < p.Aout; ++a)
-      sh.out[a * SA_TE + tid] = (mw.b3[a] + sh.part[(size_t)a * SA_TE + tid]) + sh.part[((size_t)p.Ap + a) * SA_TE + tid];
+      sh.out[a * SA_TE + tid] = (mw.b3[a] + sh.part[(size_t)a * SA_TE + tid]) + sh.part[((size_t)4 + a) * SA_TE + tid];
   __syncthreads();
   return true;
 }
@@ -400,7 +403,7 @@ __global__ void split_pack_kernel(const float* __restrict__ blob, int D, int H, 
 }  // namespace
 
 bool split_actor_supported(int env_kind, int D, int H, int Aout) {
-  return (env_kind == TJ_ENV_CARTPOLE || env_kind == TJ_ENV_ACROBOT) && D <= 8 && H >= 64 && H <= 256 && H % 64 == 0 && Aout <= 4;
+  return (env_kind == TJ_ENV_CARTPOLE || env_kind == TJ_ENV_ACROBOT) && D <= 8 && H >= 64 && H <= 256 && H % 64 == 0 && Aout <= 4;   // so Ap = 4
 }
 
 size_t split_weight_halfs(int H) { return (size_t)2 * H * H; }
