@@ -6,10 +6,14 @@
 // of the 3 x TF32 form of the same idea).  Layer 1 (4 or 6 inputs) and the head (2-4 outputs) stay on the FP32 pipes.
 //
 // One thread block keeps a tile of 128 environments for all n_steps of the call (environments are independent): thread e
-// owns env e's state in registers, all 256 threads compute layer 1 and drain the accumulator.  Per step:
-//   observation -> shared memory;  layer 1 in the fixed FMA order of the FP32 path, ReLU, split -> FP16 A operand (128 rows x H);
-//   one lane streams W2's parts in 32-column chunks (bulk copies, four ring slots, the stream running on across steps) and
-//   issues the MMAs (M = 128, N = H);  accumulator -> + b2, ReLU, head partial sums by two threads per row -> outputs;
+// owns env e's state in registers.  Eight worker warps and one issuing warp; per step:
+//   observation -> shared memory;
+//   workers: layer 1 in the fixed FMA order of the FP32 path, ReLU, split -> FP16 A operand, 32 hidden units (one K chunk of
+//     the next layer) at a time, each chunk handed to the issuing lane through its own mbarrier;
+//   issuing lane: streams W2's parts in 32-column chunks (bulk copies, four ring slots, the stream running on across steps)
+//     and, per K chunk, issues W_hi x (h_hi, h_lo) and W_lo x h_hi (M = 128, N = H) as soon as that chunk of h1 exists, so
+//     the tensor pipe works underneath layer 1;
+//   workers: accumulator -> + b2, ReLU, head partial sums by two threads per row -> outputs;
 //   then exactly the FP32 kernel's selection, env step, record / segment write and reset.
 // Every wait is bounded; a timeout latches the context's error word and the block leaves after freeing its tensor memory.
 #include <cuda_fp16.h>
@@ -23,15 +27,18 @@ namespace tj {
 namespace {
 
 constexpr int SA_TE = 128;            // envs per tile = rows of the MMA
-constexpr int SA_NT = 256;
+constexpr int SA_WORKERS = 256;       // threads of the worker warps; one more warp issues
+constexpr int SA_NT = SA_WORKERS + 32;
 constexpr int SA_KC = 32;             // K columns per streamed chunk of W2
 constexpr int SA_SLOTS = 4;
+constexpr int SA_MAX_KC = 256 / SA_KC;
 constexpr float SA_H_SCALE = 16.0f;   // hidden activations are split after this scaling (|h1| < 4,094 stays inside FP16)
 
 struct SaCtl {
   uint64_t full[SA_SLOTS], empty[SA_SLOTS];
-  uint64_t wbar;          // small parameters staged
-  uint64_t acc_full;      // all MMAs of a forward pass complete
+  uint64_t a_ready[SA_MAX_KC];   // K chunk of the A operand written (one arrival per worker warp)
+  uint64_t wbar;                 // small parameters staged
+  uint64_t acc_full;             // all MMAs of a forward pass complete
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -58,99 +65,113 @@ struct SaShared {
   uint8_t *a_hi, *a_lo, *ring;
   float *xs, *out, *part;
   SaCtl* ctl;
-  int a_bytes, chunk_bytes, n_chunks;
 };
+
+// eight hidden units n0 .. n0+7 of layer 1 for one env, in the canonical order (bias, then inputs in index order), ReLU,
+// scaling, split; one 16-byte row segment of each part of the A operand
+template <int D>
+__device__ __forceinline__ void sa_layer1_block(const MlpWeights& mw, int Hp, const float* x, int n0, uint8_t* a_hi, uint8_t* a_lo, size_t off) {
+  float acc[8];
+  const float4 b0 = *reinterpret_cast<const float4*>(mw.b1 + n0), b1 = *reinterpret_cast<const float4*>(mw.b1 + n0 + 4);
+  acc[0] = b0.x; acc[1] = b0.y; acc[2] = b0.z; acc[3] = b0.w; acc[4] = b1.x; acc[5] = b1.y; acc[6] = b1.z; acc[7] = b1.w;
+#pragma unroll
+  for (int k = 0; k < D; ++k) {
+    const float4 w0 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * Hp + n0);
+    const float4 w1 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * Hp + n0 + 4);
+    acc[0] = fmaf(w0.x, x[k], acc[0]); acc[1] = fmaf(w0.y, x[k], acc[1]); acc[2] = fmaf(w0.z, x[k], acc[2]); acc[3] = fmaf(w0.w, x[k], acc[3]);
+    acc[4] = fmaf(w1.x, x[k], acc[4]); acc[5] = fmaf(w1.y, x[k], acc[5]); acc[6] = fmaf(w1.z, x[k], acc[6]); acc[7] = fmaf(w1.w, x[k], acc[7]);
+  }
+  uint32_t hi2[4], lo2[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float v0 = fmaxf(acc[2 * i], 0.f) * SA_H_SCALE, v1 = fmaxf(acc[2 * i + 1], 0.f) * SA_H_SCALE;
+    const float h0 = __uint_as_float(__float_as_uint(v0) & 0xFFFFE000u), h1 = __uint_as_float(__float_as_uint(v1) & 0xFFFFE000u);
+    hi2[i] = pack_f16x2(h0, h1);
+    lo2[i] = pack_f16x2(v0 - h0, v1 - h1);
+  }
+  *reinterpret_cast<uint4*>(a_hi + off) = make_uint4(hi2[0], hi2[1], hi2[2], hi2[3]);
+  *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(lo2[0], lo2[1], lo2[2], lo2[3]);
+}
 
 // Network outputs of the observations in xs -> out[i][e], i < Aout.  Called by every thread of the block; `pass` counts the
 // calls, `copied` / `used` are the issuing lane's positions in the chunk stream.  Returns false after a timeout.
+template <int D, int H>
 __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeights& mw, const SaShared& sh, const uint16_t* w2parts,
                                            float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied, uint32_t& used,
                                            volatile int* abort_flag) {
+  constexpr int NKC = H / SA_KC;                 // K chunks of the hidden x hidden layer
+  constexpr uint32_t NSTREAM = 2 * NKC;          // chunks of W2 per pass: (high, low) per K chunk
+  constexpr uint32_t CHUNK_BYTES = H * SA_KC * 2;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int H = p.H, D = p.D;
-  // layer 1 in the canonical order (bias, then inputs in index order), ReLU, scale, split, FP16 A operand rows
-  {
+  SaCtl* ctl = sh.ctl;
+  if (tid < SA_WORKERS) {
     const int e = tid & (SA_TE - 1), half = tid >> 7;
-    const int n_lo = half * (H / 2), n_hi = n_lo + H / 2;
-    float x[8];
+    float x[D];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) x[k] = k < D ? sh.xs[k * SA_TE + e] : 0.f;
-    for (int n0 = n_lo; n0 < n_hi; n0 += 8) {
-      float acc[8];
-      const float4 b0 = *reinterpret_cast<const float4*>(mw.b1 + n0), b1 = *reinterpret_cast<const float4*>(mw.b1 + n0 + 4);
-      acc[0] = b0.x; acc[1] = b0.y; acc[2] = b0.z; acc[3] = b0.w; acc[4] = b1.x; acc[5] = b1.y; acc[6] = b1.z; acc[7] = b1.w;
+    for (int k = 0; k < D; ++k) x[k] = sh.xs[k * SA_TE + e];
+    tc_fence_before();                            // this thread's accumulator reads of the previous pass are complete
+#pragma unroll 1
+    for (int kc = 0; kc < NKC; ++kc) {
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        if (k < D) {
-          const float4 w0 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * p.Hp + n0);
-          const float4 w1 = *reinterpret_cast<const float4*>(mw.W1t + (size_t)k * p.Hp + n0 + 4);
-          acc[0] = fmaf(w0.x, x[k], acc[0]); acc[1] = fmaf(w0.y, x[k], acc[1]); acc[2] = fmaf(w0.z, x[k], acc[2]); acc[3] = fmaf(w0.w, x[k], acc[3]);
-          acc[4] = fmaf(w1.x, x[k], acc[4]); acc[5] = fmaf(w1.y, x[k], acc[5]); acc[6] = fmaf(w1.z, x[k], acc[6]); acc[7] = fmaf(w1.w, x[k], acc[7]);
+      for (int b = 0; b < 2; ++b) {
+        const int n0 = kc * SA_KC + half * 16 + b * 8;
+        const size_t off = ((size_t)(e >> 3) * (H / 8) + (n0 >> 3)) * 128 + (e & 7) * 16;
+        sa_layer1_block<D>(mw, p.Hp, x, n0, sh.a_hi, sh.a_lo, off);
+      }
+      fence_async_smem();
+      mbar_arrive_warp(&ctl->a_ready[kc]);
+    }
+  } else {
+    // The issuing lane's warp-mates wait at the warp barrier, not in a polling loop: lanes of one warp that poll while
+    // another lane of it issues take turns with that lane, and every blocked poll then stalls the issue.
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_f16(H);
+      const uint32_t ahi_lo = desc_lo(smem_addr(sh.a_hi), 128u), alo_lo = desc_lo(smem_addr(sh.a_lo), 128u);
+      const uint32_t a_hiword = desc_hi((uint32_t)(H / 8) * 128u), b_hiword = desc_hi((uint32_t)(SA_KC / 8) * 128u);
+      const uint32_t ring_lo = desc_lo(smem_addr(sh.ring), 128u);
+      bool alive = true;
+#pragma unroll 1
+      for (int c = 0; c < (int)NSTREAM && alive; ++c, ++used) {
+        const int kc = c >> 1;
+        const bool low_part = c & 1;
+        if (!low_part) {
+          if (!tc_wait(&ctl->a_ready[kc], pass & 1, abort_flag)) break;
+          tc_fence_after();
+        }
+        const uint32_t s = used % SA_SLOTS;
+        if (!tc_wait(&ctl->full[s], (used / SA_SLOTS) & 1, abort_flag)) break;
+        const uint32_t b_lo = ring_lo + s * (CHUNK_BYTES / 16);
+#pragma unroll
+        for (int j = 0; j < SA_KC / 16; ++j) {
+          const uint32_t a_off = (uint32_t)(kc * (SA_KC / 8) + 2 * j) * 8u;        // in 16-byte units: 8 per core matrix
+          umma_ss(tmem, ahi_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, (c | j) != 0);
+          if (!low_part) umma_ss(tmem, alo_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, 1u);
+        }
+        umma_commit(&ctl->empty[s]);
+        if (used >= 1) {
+          // chunk `copied` goes into the slot chunk `used - 1` occupied (copied = used - 1 + SLOTS)
+          const uint32_t sp = copied % SA_SLOTS;
+          if (!tc_wait(&ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) { alive = false; continue; }
+          mbar_expect_tx(&ctl->full[sp], CHUNK_BYTES);
+          bulk_copy_g2s(sh.ring + (size_t)sp * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
+                        CHUNK_BYTES, &ctl->full[sp]);
+          ++copied;
         }
       }
-      uint32_t hi2[4], lo2[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float v0 = fmaxf(acc[2 * i], 0.f) * SA_H_SCALE, v1 = fmaxf(acc[2 * i + 1], 0.f) * SA_H_SCALE;
-        const float h0 = __uint_as_float(__float_as_uint(v0) & 0xFFFFE000u), h1 = __uint_as_float(__float_as_uint(v1) & 0xFFFFE000u);
-        hi2[i] = pack_f16x2(h0, h1);
-        lo2[i] = pack_f16x2(v0 - h0, v1 - h1);
-      }
-      const size_t off = ((size_t)(e >> 3) * (H / 8) + (n0 >> 3)) * 128 + (e & 7) * 16;
-      *reinterpret_cast<uint4*>(sh.a_hi + off) = make_uint4(hi2[0], hi2[1], hi2[2], hi2[3]);
-      *reinterpret_cast<uint4*>(sh.a_lo + off) = make_uint4(lo2[0], lo2[1], lo2[2], lo2[3]);
+      umma_commit(&ctl->acc_full);
     }
+    __syncwarp();
   }
-  fence_async_smem();
-  tc_fence_before();
-  __syncthreads();   // A operand complete; every thread has finished reading the previous pass's accumulator
-  // The issuing lane's warp-mates wait at the warp barrier below, not in a polling loop: lanes of one warp that poll while
-  // another lane of it issues take turns with that lane, and every blocked poll then stalls the issue.
-  if (warp == 0) {
-   if (lane == 0) {
-    // hidden x hidden layer: per chunk of 32 columns two K steps; the high parts of W2 meet both parts of h1, the low
-    // parts only h1's high part.  After the MMAs of chunk g are issued, the slot of chunk g - 1 is refilled with chunk
-    // g + 3 of the (cyclic) stream, so three copies are in flight while a chunk is multiplied.
-    const uint32_t idesc = make_idesc_f16(H);
-    const uint32_t ahi_lo = desc_lo(smem_addr(sh.a_hi), 128u), alo_lo = desc_lo(smem_addr(sh.a_lo), 128u);
-    const uint32_t a_hiword = desc_hi((uint32_t)(H / 8) * 128u), b_hiword = desc_hi((uint32_t)(SA_KC / 8) * 128u);
-    const uint32_t ring_lo = desc_lo(smem_addr(sh.ring), 128u);
-    tc_fence_after();
-    for (int c = 0; c < sh.n_chunks; ++c, ++used) {
-      const uint32_t s = used % SA_SLOTS;
-      if (!tc_wait(&sh.ctl->full[s], (used / SA_SLOTS) & 1, abort_flag)) break;
-      const bool low_part = c >= sh.n_chunks / 2;
-      const int kc = c % (sh.n_chunks / 2);
-      const uint32_t b_lo = ring_lo + s * (uint32_t)(sh.chunk_bytes / 16);
-#pragma unroll
-      for (int j = 0; j < SA_KC / 16; ++j) {
-        const uint32_t a_off = (uint32_t)(kc * (SA_KC / 8) + 2 * j) * 8u;        // in 16-byte units: 8 per core matrix
-        umma_ss(tmem, ahi_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, (c | j) != 0);
-        if (!low_part) umma_ss(tmem, alo_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, 1u);
-      }
-      umma_commit(&sh.ctl->empty[s]);
-      if (used >= 1) {
-        // chunk `copied` goes into the slot chunk `used - 1` occupied (copied = used - 1 + SLOTS)
-        const uint32_t sp = copied % SA_SLOTS;
-        if (!tc_wait(&sh.ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) break;
-        mbar_expect_tx(&sh.ctl->full[sp], (uint32_t)sh.chunk_bytes);
-        bulk_copy_g2s(sh.ring + (size_t)sp * sh.chunk_bytes,
-                      reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % (uint32_t)sh.n_chunks) * sh.chunk_bytes,
-                      (uint32_t)sh.chunk_bytes, &sh.ctl->full[sp]);
-        ++copied;
-      }
-    }
-    umma_commit(&sh.ctl->acc_full);
-   }
-   __syncwarp();
-  }
-  if (!tc_wait_elect(&sh.ctl->acc_full, pass & 1, abort_flag)) return false;
+  // after a timeout the abort flag is up: the pass runs to its end on meaningless numbers (every thread keeps to the same
+  // barriers) and the caller leaves
+  tc_wait_elect(&ctl->acc_full, pass & 1, abort_flag);
   tc_fence_after();
   // drain: two threads per row (the two column halves); h2 = relu(acc / scale + b2), head partial sums in column order
-  {
+  if (tid < SA_WORKERS) {
     const int q = warp & 3, half = warp >> 2, r = q * 32 + lane;
     float pa[4] = {0.f, 0.f, 0.f, 0.f};
     const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
+#pragma unroll 2
     for (int c0 = half * (H / 2); c0 < (half + 1) * (H / 2); c0 += 16) {
       uint32_t v[16];
       tmem_ld16(t_row + (uint32_t)c0, v);
@@ -158,8 +179,7 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
 #pragma unroll
       for (int i = 0; i < 16; ++i) {
         const float h2 = fmaxf(fmaf(__uint_as_float(v[i]), inv_scale, mw.b2[c0 + i]), 0.f);
-        const float* w3 = mw.W3t + (size_t)(c0 + i) * 4;
-        const float4 w = *reinterpret_cast<const float4*>(w3);      // Ap = 4: rows of W3t are one vector, zero beyond Aout
+        const float4 w = *reinterpret_cast<const float4*>(mw.W3t + (size_t)(c0 + i) * 4);   // a row of W3t (Ap = 4)
         pa[0] = fmaf(w.x, h2, pa[0]); pa[1] = fmaf(w.y, h2, pa[1]); pa[2] = fmaf(w.z, h2, pa[2]); pa[3] = fmaf(w.w, h2, pa[3]);
       }
     }
@@ -167,33 +187,32 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
     for (int a = 0; a < 4; ++a)
       if (a < p.Aout) sh.part[((size_t)half * 4 + a) * SA_TE + r] = pa[a];
   }
-  tc_fence_before();
   __syncthreads();
   if (tid < SA_TE)
     for (int a = 0; a < p.Aout; ++a)
       sh.out[a * SA_TE + tid] = (mw.b3[a] + sh.part[(size_t)a * SA_TE + tid]) + sh.part[((size_t)4 + a) * SA_TE + tid];
   __syncthreads();
-  return true;
+  return *abort_flag == 0;
 }
 
-template <int ENV>
+template <int ENV, int H>
 __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorParams p, const uint16_t* __restrict__ w2parts,
                                                                  const float* __restrict__ w2scale) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  const int H = p.H, D = p.D;
+  constexpr int D = ENV == TJ_ENV_CARTPOLE ? 4 : 6;
+  constexpr int A_BYTES = SA_TE * H * 2;                      // one FP16 part of the A operand
+  constexpr uint32_t CHUNK_BYTES = H * SA_KC * 2;             // one chunk of one part of W2
+  constexpr uint32_t NSTREAM = 2 * (H / SA_KC);
   SaShared sh;
-  sh.a_bytes = SA_TE * H * 2;                                 // one FP16 part of the A operand
-  sh.chunk_bytes = H * SA_KC * 2;                             // one chunk of one part of W2
-  sh.n_chunks = 2 * (H / SA_KC);                              // per forward pass: the high parts' chunks, then the low parts'
   sh.a_hi = smem_raw;
-  sh.a_lo = sh.a_hi + sh.a_bytes;
-  sh.ring = sh.a_lo + sh.a_bytes;
-  float* wsm = reinterpret_cast<float*>(sh.ring + SA_SLOTS * sh.chunk_bytes);
+  sh.a_lo = sh.a_hi + A_BYTES;
+  sh.ring = sh.a_lo + A_BYTES;
+  float* wsm = reinterpret_cast<float*>(sh.ring + SA_SLOTS * CHUNK_BYTES);
   const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);   // everything but the H x H matrix
-  sh.xs = wsm + staged;                                       // [D][TE]
-  sh.out = sh.xs + (size_t)((D + 3) & ~3) * SA_TE;            // [Ap][TE]
-  sh.part = sh.out + (size_t)p.Ap * SA_TE;                    // [2][Ap][TE]
-  sh.ctl = reinterpret_cast<SaCtl*>(sh.part + 2 * (size_t)p.Ap * SA_TE);
+  sh.xs = wsm + staged;                                       // [8][TE]
+  sh.out = sh.xs + (size_t)8 * SA_TE;                         // [4][TE]
+  sh.part = sh.out + (size_t)4 * SA_TE;                       // [2][4][TE]
+  sh.ctl = reinterpret_cast<SaCtl*>(sh.part + 2 * (size_t)4 * SA_TE);
   SaCtl* ctl = sh.ctl;
   const int tid = threadIdx.x, warp = tid >> 5;
   const int n_tiles = (p.N + SA_TE - 1) / SA_TE;
@@ -201,6 +220,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
 
   if (tid == 0) {
     for (int s = 0; s < SA_SLOTS; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    for (int k = 0; k < SA_MAX_KC; ++k) mbar_init(&ctl->a_ready[k], SA_WORKERS / 32);
     mbar_init(&ctl->wbar, 1);
     mbar_init(&ctl->acc_full, 1);
     ctl->abort_flag = 0;
@@ -216,17 +236,16 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort_flag;
-  bool ok = tc_wait_warp(&ctl->wbar, 0, abort_flag);
+  bool ok = tc_wait_elect(&ctl->wbar, 0, abort_flag);
   ok = __syncthreads_and(ok);
   const float inv_scale = w2scale[1];                         // 1 / (activation scale x weight scale)
 
   uint32_t copied = 0, used = 0, pass = 0;                     // chunk stream positions (issuing lane), forward passes
-  if (tid == 0 && ok) {
+  if (tid == SA_WORKERS && ok) {
     for (; copied < SA_SLOTS; ++copied) {
-      mbar_expect_tx(&ctl->full[copied], (uint32_t)sh.chunk_bytes);
-      bulk_copy_g2s(sh.ring + (size_t)copied * sh.chunk_bytes,
-                    reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % (uint32_t)sh.n_chunks) * sh.chunk_bytes,
-                    (uint32_t)sh.chunk_bytes, &ctl->full[copied]);
+      mbar_expect_tx(&ctl->full[copied], CHUNK_BYTES);
+      bulk_copy_g2s(sh.ring + (size_t)copied * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
+                    CHUNK_BYTES, &ctl->full[copied]);
     }
   }
 
@@ -249,11 +268,10 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
       sa_observe<ENV>(s, obs);
       if (tid < SA_TE) {
 #pragma unroll
-        for (int k = 0; k < 6; ++k)
-          if (k < D) sh.xs[k * SA_TE + tid] = owner ? obs[k] : 0.f;
+        for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? obs[k] : 0.f;
       }
       __syncthreads();
-      ok = sa_forward(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+      ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
       ok = __syncthreads_and(ok);
       if (!ok) break;
       if (owner) {
@@ -276,7 +294,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
           const int pos = (int)(t % (unsigned long long)p.T);
           const int slot = (int)(g % p.G);
           const size_t i = ((size_t)slot * p.T + pos) * p.N + e;
-          float* so = p.seg_obs + i * p.D;
+          float* so = p.seg_obs + i * D;
           if (ENV == TJ_ENV_CARTPOLE) *reinterpret_cast<float4*>(so) = s;
           else
             for (int k = 0; k < 6; ++k) so[k] = obs[k];
@@ -323,11 +341,10 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
         __syncthreads();
         if (tid < SA_TE) {
 #pragma unroll
-          for (int k = 0; k < 6; ++k)
-            if (k < D) sh.xs[k * SA_TE + tid] = owner ? o2[k] : 0.f;
+          for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? o2[k] : 0.f;
         }
         __syncthreads();
-        ok = sa_forward(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+        ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         if (owner) {
@@ -348,7 +365,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
     atomicAdd(&p.stats->return_sum, ret_sum);
   }
   // the copies still in flight must land before the block gives its shared memory back
-  if (tid == 0) {
+  if (tid == SA_WORKERS) {
     for (uint32_t g = used; g < copied; ++g)
       if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
     if (ctl->abort_flag) atomicExch(&p.stats->error, 4ull);
@@ -362,8 +379,9 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
   }
 }
 
-// W2 [H][H] (row = neuron) -> scaled FP16 high and low parts, each as H / 32 chunks of H rows x 32 columns in the K-major
-// core-matrix layout: element (n, k) of chunk kc sits at ((n / 8) * 4 + (k % 32) / 8) * 64 + (n % 8) * 8 + k % 8.
+// W2 [H][H] (row = neuron) -> scaled FP16 high and low parts as the stream the kernel consumes: for each K chunk kc of 32
+// columns first the high parts' chunk, then the low parts', each H rows x 32 columns in the K-major core-matrix layout:
+// element (n, k) sits at ((n / 8) * 4 + (k % 32) / 8) * 64 + (n % 8) * 8 + k % 8 inside its chunk.
 // scale_out[0] = the power of two the weights were multiplied by, scale_out[1] = 1 / (that x the activation scale).
 __global__ void split_scale_kernel(const float* __restrict__ blob, int D, int H, float* __restrict__ scale_out) {
   __shared__ float wmax[32];
@@ -389,21 +407,42 @@ __global__ void split_pack_kernel(const float* __restrict__ blob, int D, int H, 
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= H * H) return;
   const float* W2 = blob + (size_t)H * D + H;
-  const int chunk = i / (H * SA_KC), within = i % (H * SA_KC);
+  const int chunk_elems = H * SA_KC;
+  const int kc = i / chunk_elems, within = i % chunk_elems;
   const int core = within / 64, in_core = within % 64;
   const int rg = core / (SA_KC / 8), kg = core % (SA_KC / 8);
-  const int n = rg * 8 + in_core / 8, k = chunk * SA_KC + kg * 8 + in_core % 8;
+  const int n = rg * 8 + in_core / 8, k = kc * SA_KC + kg * 8 + in_core % 8;
   const float v = W2[(size_t)n * H + k] * scale[0];
   const __half hi = __float2half_rn(v);
   const __half lo = __float2half_rn(v - __half2float(hi));
-  dst[i] = __half_as_ushort(hi);
-  dst[(size_t)H * H + i] = __half_as_ushort(lo);
+  dst[(size_t)(2 * kc) * chunk_elems + within] = __half_as_ushort(hi);
+  dst[(size_t)(2 * kc + 1) * chunk_elems + within] = __half_as_ushort(lo);
+}
+
+template <int ENV, int H>
+cudaError_t launch_split(const ActorParams& p, const uint16_t* w2parts, const float* w2scale, int grid, size_t smem, cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(actor_split_tc_kernel<ENV, H>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  actor_split_tc_kernel<ENV, H><<<grid, SA_NT, smem, s>>>(p, w2parts, w2scale);
+  return cudaGetLastError();
+}
+
+template <int ENV>
+cudaError_t launch_split_env(const ActorParams& p, const uint16_t* w2parts, const float* w2scale, int grid, size_t smem, cudaStream_t s) {
+  switch (p.H) {
+    case 64: return launch_split<ENV, 64>(p, w2parts, w2scale, grid, smem, s);
+    case 128: return launch_split<ENV, 128>(p, w2parts, w2scale, grid, smem, s);
+    case 192: return launch_split<ENV, 192>(p, w2parts, w2scale, grid, smem, s);
+    case 256: return launch_split<ENV, 256>(p, w2parts, w2scale, grid, smem, s);
+    default: return cudaErrorInvalidConfiguration;
+  }
 }
 
 }  // namespace
 
 bool split_actor_supported(int env_kind, int D, int H, int Aout) {
-  return (env_kind == TJ_ENV_CARTPOLE || env_kind == TJ_ENV_ACROBOT) && D <= 8 && H >= 64 && H <= 256 && H % 64 == 0 && Aout <= 4;   // so Ap = 4
+  const bool env_ok = (env_kind == TJ_ENV_CARTPOLE && D == 4) || (env_kind == TJ_ENV_ACROBOT && D == 6);
+  return env_ok && H >= 64 && H <= 256 && H % 64 == 0 && Aout <= 4;   // Aout <= 4: rows of the head matrix are one float4
 }
 
 size_t split_weight_halfs(int H) { return (size_t)2 * H * H; }
@@ -420,19 +459,12 @@ cudaError_t launch_actor_split(int env_kind, const ActorParams& p, const uint16_
   if (!split_actor_supported(env_kind, p.D, p.H, p.Aout)) return cudaErrorInvalidConfiguration;
   const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);
   const size_t smem = (size_t)2 * SA_TE * p.H * 2 + (size_t)SA_SLOTS * p.H * SA_KC * 2 +
-                      (staged + (size_t)((p.D + 3) & ~3) * SA_TE + 3 * (size_t)p.Ap * SA_TE) * sizeof(float) + sizeof(SaCtl) + 64;
+                      (staged + (size_t)(8 + 4 + 8) * SA_TE) * sizeof(float) + sizeof(SaCtl) + 64;
   if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
   const int n_tiles = (p.N + SA_TE - 1) / SA_TE;
   const int grid = n_tiles < sm_count ? n_tiles : sm_count;
-  cudaError_t e;
-  if (env_kind == TJ_ENV_CARTPOLE) {
-    if ((e = cudaFuncSetAttribute(actor_split_tc_kernel<TJ_ENV_CARTPOLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    actor_split_tc_kernel<TJ_ENV_CARTPOLE><<<grid, SA_NT, smem, s>>>(p, w2parts, w2scale);
-  } else {
-    if ((e = cudaFuncSetAttribute(actor_split_tc_kernel<TJ_ENV_ACROBOT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    actor_split_tc_kernel<TJ_ENV_ACROBOT><<<grid, SA_NT, smem, s>>>(p, w2parts, w2scale);
-  }
-  return cudaGetLastError();
+  return env_kind == TJ_ENV_CARTPOLE ? launch_split_env<TJ_ENV_CARTPOLE>(p, w2parts, w2scale, grid, smem, s)
+                                     : launch_split_env<TJ_ENV_ACROBOT>(p, w2parts, w2scale, grid, smem, s);
 }
 
 }  // namespace tj
