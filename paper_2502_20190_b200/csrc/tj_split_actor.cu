@@ -6,12 +6,12 @@
 // of the 3 x TF32 form of the same idea).  Layer 1 (4 or 6 inputs) and the head (2-4 outputs) stay on the FP32 pipes.
 //
 // One thread block keeps a tile of 128 environments for all n_steps of the call (environments are independent): thread e
-// owns env e's state in registers.  Eight worker warps and one issuing warp; per step:
+// owns env e's state in registers.  Eight worker warps, one MMA-issuing warp, one copy warp; per step:
 //   observation -> shared memory;
 //   workers: layer 1 in the fixed FMA order of the FP32 path, ReLU, split -> FP16 A operand, 32 hidden units (one K chunk of
 //     the next layer) at a time, each chunk handed to the issuing lane through its own mbarrier;
-//   issuing lane: streams W2's parts in 32-column chunks (bulk copies, four ring slots, the stream running on across steps)
-//     and, per K chunk, issues W_hi x (h_hi, h_lo) and W_lo x h_hi (M = 128, N = H) as soon as that chunk of h1 exists, so
+//   copy lane: streams W2's parts in 32-column chunks (bulk copies, four ring slots, the stream running on across steps);
+//   issuing lane: per K chunk, issues W_hi x (h_hi, h_lo) and W_lo x h_hi (M = 128, N = H) as soon as that chunk of h1 exists, so
 //     the tensor pipe works underneath layer 1;
 //   workers: accumulator -> + b2, ReLU, head partial sums by two threads per row -> outputs;
 //   then exactly the FP32 kernel's selection, env step, record / segment write and reset.
@@ -28,7 +28,7 @@ namespace {
 
 constexpr int SA_TE = 128;            // envs per tile = rows of the MMA
 constexpr int SA_WORKERS = 256;       // threads of the worker warps; one more warp issues
-constexpr int SA_NT = SA_WORKERS + 32;
+constexpr int SA_NT = SA_WORKERS + 64;   // + the MMA-issuing warp and the copy warp
 constexpr int SA_KC = 32;             // K columns per streamed chunk of W2
 constexpr int SA_SLOTS = 4;
 constexpr int SA_MAX_KC = 256 / SA_KC;
@@ -94,10 +94,10 @@ __device__ __forceinline__ void sa_layer1_block(const MlpWeights& mw, int Hp, co
 }
 
 // Network outputs of the observations in xs -> out[i][e], i < Aout.  Called by every thread of the block; `pass` counts the
-// calls, `copied` / `used` are the issuing lane's positions in the chunk stream.  Returns false after a timeout.
+// calls, `copied` is the copy lane's position in the chunk stream.  Returns false after a timeout.
 template <int D, int H>
 __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeights& mw, const SaShared& sh, const uint16_t* w2parts,
-                                           float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied, uint32_t& used,
+                                           float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied,
                                            volatile int* abort_flag) {
   constexpr int NKC = H / SA_KC;                 // K chunks of the hidden x hidden layer
   constexpr uint32_t NSTREAM = 2 * NKC;          // chunks of W2 per pass: (high, low) per K chunk
@@ -121,44 +121,52 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
       fence_async_smem();
       mbar_arrive_warp(&ctl->a_ready[kc]);
     }
-  } else {
+  } else if (warp == SA_WORKERS / 32) {
     // The issuing lane's warp-mates wait at the warp barrier, not in a polling loop: lanes of one warp that poll while
     // another lane of it issues take turns with that lane, and every blocked poll then stalls the issue.
     if (lane == 0) {
+      // The stream position at the start of a pass is pass x NSTREAM, a multiple of the slot count: chunk c of any pass sits
+      // in slot c % SLOTS, and only the barrier parities depend on the pass.
       const uint32_t idesc = make_idesc_f16(H);
       const uint32_t ahi_lo = desc_lo(smem_addr(sh.a_hi), 128u), alo_lo = desc_lo(smem_addr(sh.a_lo), 128u);
       const uint32_t a_hiword = desc_hi((uint32_t)(H / 8) * 128u), b_hiword = desc_hi((uint32_t)(SA_KC / 8) * 128u);
       const uint32_t ring_lo = desc_lo(smem_addr(sh.ring), 128u);
+      const uint32_t round0 = pass * (NSTREAM / SA_SLOTS);           // trips around the ring before this pass
       bool alive = true;
-#pragma unroll 1
-      for (int c = 0; c < (int)NSTREAM && alive; ++c, ++used) {
-        const int kc = c >> 1;
-        const bool low_part = c & 1;
-        if (!low_part) {
-          if (!tc_wait(&ctl->a_ready[kc], pass & 1, abort_flag)) break;
-          tc_fence_after();
-        }
-        const uint32_t s = used % SA_SLOTS;
-        if (!tc_wait(&ctl->full[s], (used / SA_SLOTS) & 1, abort_flag)) break;
-        const uint32_t b_lo = ring_lo + s * (CHUNK_BYTES / 16);
 #pragma unroll
-        for (int j = 0; j < SA_KC / 16; ++j) {
-          const uint32_t a_off = (uint32_t)(kc * (SA_KC / 8) + 2 * j) * 8u;        // in 16-byte units: 8 per core matrix
-          umma_ss(tmem, ahi_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, (c | j) != 0);
-          if (!low_part) umma_ss(tmem, alo_lo + a_off, a_hiword, b_lo + j * 16u, b_hiword, idesc, 1u);
-        }
-        umma_commit(&ctl->empty[s]);
-        if (used >= 1) {
-          // chunk `copied` goes into the slot chunk `used - 1` occupied (copied = used - 1 + SLOTS)
-          const uint32_t sp = copied % SA_SLOTS;
-          if (!tc_wait(&ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) { alive = false; continue; }
-          mbar_expect_tx(&ctl->full[sp], CHUNK_BYTES);
-          bulk_copy_g2s(sh.ring + (size_t)sp * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
-                        CHUNK_BYTES, &ctl->full[sp]);
-          ++copied;
+      for (int kc = 0; kc < NKC; ++kc) {
+        if (!alive) break;
+        if (!tc_wait(&ctl->a_ready[kc], pass & 1, abort_flag)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t a_off = (uint32_t)kc * (SA_KC / 8) * 8u;     // in 16-byte units: 8 per core matrix, 4 core matrices per chunk
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+          const int c = 2 * kc + part, s = c % SA_SLOTS;
+          if (!tc_wait(&ctl->full[s], (round0 + c / SA_SLOTS) & 1, abort_flag)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t b_lo = ring_lo + (uint32_t)s * (CHUNK_BYTES / 16);
+#pragma unroll
+          for (int j = 0; j < SA_KC / 16; ++j) {
+            umma_ss(tmem, ahi_lo + a_off + 16u * j, a_hiword, b_lo + 16u * j, b_hiword, idesc, (c | j) != 0);
+            if (part == 0) umma_ss(tmem, alo_lo + a_off + 16u * j, a_hiword, b_lo + 16u * j, b_hiword, idesc, 1u);
+          }
+          umma_commit(&ctl->empty[s]);
         }
       }
       umma_commit(&ctl->acc_full);
+    }
+    __syncwarp();
+  } else {
+    // copy lane: keeps the ring full -- chunk g of the stream follows chunk g - SLOTS into its slot once that one is consumed
+    if (lane == 0) {
+#pragma unroll 1
+      for (uint32_t c = 0; c < NSTREAM; ++c, ++copied) {
+        const uint32_t sp = copied % SA_SLOTS;
+        if (!tc_wait(&ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(&ctl->full[sp], CHUNK_BYTES);
+        bulk_copy_g2s(sh.ring + (size_t)sp * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
+                      CHUNK_BYTES, &ctl->full[sp]);
+      }
     }
     __syncwarp();
   }
@@ -240,8 +248,8 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
   ok = __syncthreads_and(ok);
   const float inv_scale = w2scale[1];                         // 1 / (activation scale x weight scale)
 
-  uint32_t copied = 0, used = 0, pass = 0;                     // chunk stream positions (issuing lane), forward passes
-  if (tid == SA_WORKERS && ok) {
+  uint32_t copied = 0, pass = 0;                               // chunk stream position (copy lane), forward passes
+  if (tid == SA_WORKERS + 32 && ok) {
     for (; copied < SA_SLOTS; ++copied) {
       mbar_expect_tx(&ctl->full[copied], CHUNK_BYTES);
       bulk_copy_g2s(sh.ring + (size_t)copied * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
@@ -271,7 +279,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
         for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? obs[k] : 0.f;
       }
       __syncthreads();
-      ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+      ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
       ok = __syncthreads_and(ok);
       if (!ok) break;
       if (owner) {
@@ -344,7 +352,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
           for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? o2[k] : 0.f;
         }
         __syncthreads();
-        ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, used, abort_flag);
+        ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         if (owner) {
@@ -365,8 +373,8 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
     atomicAdd(&p.stats->return_sum, ret_sum);
   }
   // the copies still in flight must land before the block gives its shared memory back
-  if (tid == SA_WORKERS) {
-    for (uint32_t g = used; g < copied; ++g)
+  if (tid == SA_WORKERS + 32) {
+    for (uint32_t g = pass * NSTREAM; g < copied; ++g)
       if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
     if (ctl->abort_flag) atomicExch(&p.stats->error, 4ull);
   }
