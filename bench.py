@@ -140,9 +140,14 @@ def aggregate_throughput(units_per_replica, world, max_ms):
 class Runner:
     """Drives one context through the workload's call pattern."""
 
-    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False, two_stream=False):
+    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False, two_stream=False, tensor_fp32=False):
         self.torch, self.name = torch, name
         self.w = dict(synth.WORKLOADS[name])
+        if tensor_fp32:
+            # FP32 weights, the actor's hidden x hidden layer as split-operand tensor-core products (1e-5 of the FP32 path)
+            if self.w["weight_dtype"] != synth.W_FP32 or self.w["env_kind"] == synth.ENV_LINGAUSS or self.w["hidden"] % 64:
+                raise SystemExit("--tensor-fp32 applies to the FP32 CartPole / Acrobot workloads with hidden 64..256")
+            self.w["weight_dtype"] = synth.W_FP32_TC
         if n_envs:
             if self.w["replay_capacity"]:
                 self.w["replay_capacity"] = self.w["replay_capacity"] // self.w["n_envs"] * n_envs
@@ -298,7 +303,7 @@ def run_ours(args):
     binding.load_library()
     peaks = load_peaks()
     name = args.workload
-    r = Runner(name, torch, binding, local, args.envs, args.with_update, args.two_stream)
+    r = Runner(name, torch, binding, local, args.envs, args.with_update, args.two_stream, args.tensor_fp32)
     w = r.w
     N = w["n_envs"]
     R = args.patterns or PATTERNS_PER_STEP[name]
@@ -342,9 +347,10 @@ def run_ours(args):
     r.ctx.set_profiling(1)
     timed_loop(args.steps, False)
     prof = r.ctx.stats()
+    prof_learner_steps = r.learner_ok
     r.ctx.set_profiling(0)
     barrier()
-    fp32_peak = r.ctx.calibrate_fp32() if w["weight_dtype"] == synth.W_FP32 else None
+    fp32_peak = r.ctx.calibrate_fp32() if (w["weight_dtype"] == synth.W_FP32 or r.with_update) else None
 
     tot_ms, e2e_ms = max_over_ranks([tot_ms, e2e_ms], "cuda")
     learner_ok = int(min_over_ranks([learner_ok], "cuda")[0])
@@ -383,6 +389,18 @@ def run_ours(args):
                 "units_per_launch": N, "flop_per_unit": mlp_flops,
                 "hbm_view": {"bytes_per_unit": nbytes, "achieved_gbs": nbytes * N / (us * 1e-6) / 1e9,
                              "frac_of_measured": nbytes * N / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}}
+    elif dom == 0 and w["weight_dtype"] == synth.W_FP32_TC:
+        # split-operand tensor-core actor: one launch = actor_steps env steps; algorithmic MLP flops (the hidden x hidden
+        # layer costs three tensor-core products per algorithmic product, so the pipe does about 3x this work)
+        us = 1e3 * kms[0] / kcnt[0]
+        units = N * r.actor_steps
+        achieved = mlp_flops * units / (us * 1e-6) / 1e12
+        roof = {"kernel": "actor_split_tc_kernel (FP32 layer 1 + FP16-split tcgen05 hidden layer + head + selection + env step + insert)",
+                "bound": "tensor", "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
+                "peak_source": tensor_peak_name + ", of " + peaks["source"] + "; fp16 peak = bf16 peak", "us_per_launch": us,
+                "units_per_launch": units, "flop_per_unit": mlp_flops, "tensor_products_per_algorithmic_product": 3,
+                "hbm_view": {"bytes_per_unit": nbytes, "achieved_gbs": nbytes * units / (us * 1e-6) / 1e9,
+                             "frac_of_measured": nbytes * units / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}}
     elif dom == 0:
         # fused FP32 actor kernel: one launch = actor_steps env steps for all N envs
         us = 1e3 * kms[0] / kcnt[0]
@@ -401,6 +419,25 @@ def run_ours(args):
         roof = {"kernel": "mlp_bf16_tc_kernel (tcgen05 MLP forward)", "bound": "tensor", "achieved": achieved,
                 "peak": tensor_peak, "unit": "TFLOP/s", "peak_source": tensor_peak_name + ", of " + peaks["source"],
                 "us_per_launch": us, "units_per_launch": rows, "flop_per_unit": mlp_flops}
+    elif names[dom] == "sgd_update":
+        # the learner's gradient step dominates: forward + backward = 6 flops per weight and row, against the FP32 FMA rate
+        # (its weight-gradient products run as 3 x TF32 on the tensor cores, the rest on the FP32 pipes)
+        ms_per_update = kms[dom] / max(prof_learner_steps, 1)       # learner steps of the profiled loop
+        upd_flops = 6.0 * mlp_macs(w) * w["minibatch"]
+        roof = {"kernel": "sgd_update (tj_sgd_step: forward, backward, Adam)", "bound": "alu",
+                "achieved": upd_flops / (ms_per_update * 1e-3) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s",
+                "peak_source": "FP32 FMA loop on every SM, measured in this run (tj_calibrate_fp32)",
+                "us_per_launch": 1e3 * kms[dom] / kcnt[dom], "ms_per_update": ms_per_update, "units_per_launch": w["minibatch"],
+                "flop_per_unit": 6.0 * mlp_macs(w)}
+    elif names[dom] == "td" and w["weight_dtype"] != synth.W_BF16:
+        # FP32 TD kernel (online forward on obs, target forward on next_obs, then the elementwise error): two MLP passes per row
+        us = 1e3 * kms[dom] / (kcnt[dom] // 2 or 1)                 # the class counts the loss reduction launch as well
+        if fp32_peak is None:
+            fp32_peak = r.ctx.calibrate_fp32()
+        roof = {"kernel": "td_kernel (FP32 online + target forward, TD target, Huber) + loss reduction", "bound": "alu",
+                "achieved": 2 * mlp_flops * w["minibatch"] / (us * 1e-6) / 1e12, "peak": fp32_peak, "unit": "TFLOP/s",
+                "peak_source": "FP32 FMA loop on every SM, measured in this run (tj_calibrate_fp32)", "us_per_launch": us,
+                "units_per_launch": w["minibatch"], "flop_per_unit": 2 * mlp_flops}
     else:
         # a memory-bound class dominates (GAE on the on-policy workload, gather on tiny ones)
         nm = names[dom]
@@ -419,7 +456,7 @@ def run_ours(args):
     line = {
         "metric": "env-steps/s", "value": value, "unit": "env-steps/s", "n_gpus": world, "steps": K,
         "warmup": args.warmup, "ms_per_step": tot_ms / K, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if w["weight_dtype"] == synth.W_BF16 else "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16" if w["weight_dtype"] == synth.W_BF16 else ("f32 (hidden layer: 3 x fp16 split products)" if w["weight_dtype"] == synth.W_FP32_TC else "f32"), "data": "synthetic",
         "config": {"workload": name, "n_envs": N, "patterns_per_step": R, "actor_steps_per_pattern": r.actor_steps,
                    "minibatch": w.get("minibatch"), "mlp": "%d-%d-%d-%d" % (w["obs_dim"], w["hidden"], w["hidden"], w["n_actions"]),
                    "replicas": world, "learner_update": r.with_update, "two_stream": r.two_stream,
@@ -642,6 +679,7 @@ def main():
     ap.add_argument("--patterns", type=int, default=0, help="passes of the path per step (default: per workload, about 50 ms of GPU time)")
     ap.add_argument("--with-update", action="store_true", help="FP32 replay workloads: the learner step also runs tj_sgd_step and publishes the parameters it trains")
     ap.add_argument("--two-stream", action="store_true", help="replay workloads: learner calls on a second CUDA stream, passes software-pipelined (learner on the previous block beside the actor's next one)")
+    ap.add_argument("--tensor-fp32", action="store_true", help="FP32 CartPole / Acrobot workloads: weight mode TJ_W_FP32_TC (hidden x hidden layer on the tensor cores as split-operand products, 1e-5 of the FP32 path)")
     ap.add_argument("--sweep", action="store_true", help="also report consumed samples/s for each staleness bound the workload names")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=16.0)

@@ -401,7 +401,7 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
       return cuda_fail(x, e, "publish: host to device copy");
     src = x->blob_stage;
   }
-  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : (x->use_split ? 3 : 1)), true, true);
+  LaunchScope scope(x, TJ_K_PUBLISH, x->use_tc_pipelined ? 3 : (x->use_tc ? 2 : (x->use_split ? 2 : 1)), true, true);
   const int next = x->active ^ 1;
   float* dst = x->version == 0 ? x->wbuf[x->active] : x->wbuf[next];
   if ((e = launch_pack_weights(src, dst, x->wl, x->value_head, x->cfg.weight_dtype == TJ_W_BF16, x->lstream)) != cudaSuccess)
