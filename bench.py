@@ -34,7 +34,7 @@ from paper_2502_20190_b200 import synth  # noqa: E402
 # dram__bytes (read + write) per env-step of the fused tensor-core actor launch, from one ncu capture of the kernel as it
 # stands (a smaller number of envs, scaled: traffic grows with the number of envs).  None once the kernel has changed
 # since the counters were taken.
-NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": None}
+NCU_DRAM_BYTES_PER_ENV_STEP = {"cfg5": 1990.0}   # 226.3 MB per launch of 113,664 envs
 L2_FLUSH_BYTES = 256 << 20
 # passes of the path per bench step: about 50 ms of GPU time per step
 PATTERNS_PER_STEP = {"cfg1": 512, "cfg2": 256, "cfg3": 128, "cfg4": 8, "cfg5": 64}
