@@ -1,7 +1,7 @@
 /*
  * tj.h -- C ABI of the B200 (sm_100a) sample production/consumption library.
  *
- * The library runs, on ONE GPU and ONE CUDA stream, the data-parallel hot path of
+ * The library runs, on ONE GPU and one CUDA stream (or two: tj_set_learner_stream), the data-parallel hot path of
  * a TianJi-style actor/buffer/learner pipeline (arXiv 2502.20190):
  *
  *   actor   (Sec. 3.1, actor loop; Algorithm 1 tasks 1-2):
@@ -22,9 +22,10 @@
  * Conventions
  *   - Every function returns a tj_status (0 = OK, negative = error).  Nothing
  *     throws, aborts or prints.  tj_last_error() gives a readable message.
- *   - All device work is enqueued on the stream given to tj_create; calls are
- *     asynchronous with respect to the host unless stated otherwise, and take
- *     effect in host call order.
+ *   - All device work is enqueued on the stream given to tj_create (the learner-side
+ *     calls on the stream given to tj_set_learner_stream, if any, ordered against the
+ *     actor's by events); calls are asynchronous with respect to the host unless
+ *     stated otherwise, and take effect in host call order.
  *   - OWNERSHIP: the caller owns every byte of device memory.  tj_query_workspace
  *     reports how much the context needs, tj_create carves the caller's buffer.
  *     The library never calls cudaMalloc/cudaFree.  tj_ctx is a small host object.
