@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtj.so")
-SOURCES = ["tj_api.cu", "tj_actor.cu", "tj_learner.cu", "tj_tc.cu", "tj_tc_actor.cu", "tj_sgd.cu", "tj_calibrate.cu", "tj_consumer.cu", "tj_split_actor.cu"]
+SOURCES = ["tj_api.cu", "tj_actor.cu", "tj_learner.cu", "tj_tc.cu", "tj_tc_actor.cu", "tj_sgd.cu", "tj_calibrate.cu", "tj_consumer.cu", "tj_split_actor.cu", "tj_sgd_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "--expt-relaxed-constexpr", "-Wno-deprecated-gpu-targets"]
 

@@ -685,6 +685,13 @@ void lay_out_update_scratch(const tj_ctx* x, tj::SgdParams& p) {
   p.w2t = p.stat_partial + 5 * (rows / 16) + 8;
   p.w2t += (4 - ((reinterpret_cast<uintptr_t>(p.w2t) / sizeof(float)) & 3)) & 3;   // 16-byte rows for the vector loads
   p.grad_partial = p.w2t + (size_t)x->H * x->H;
+  {
+    // after the partial gradients: split weight copies for the tensor-core products, 128-byte aligned for the bulk copies
+    const size_t blob = (size_t)x->H * x->D + x->H + (size_t)x->H * x->H + x->H + 17 * (size_t)x->H + 17;
+    float* w = p.grad_partial + (size_t)tj::SG_SPLITS * blob;
+    w += (32 - ((reinterpret_cast<uintptr_t>(w) / sizeof(float)) & 31)) & 31;
+    p.wpack = w;
+  }
 }
 
 int learner_update(tj_ctx* x, const tj_batch* b, float lr, float* theta, const float* theta_target, const tj::AdamParams* adam,

@@ -108,7 +108,8 @@ struct SgdParams {
   float* g;                    // scratch [n][A]: dL/dq, non-zero at the selected action only
   float* partial;              // scratch: one Huber partial sum per 16 rows
   float* grad_partial;         // scratch: per row range one partial gradient laid out like the parameter blob
-  float* w2t;                  // scratch [H][H]: W2 transposed, the backward pass's operand on the tensor-core path
+  float* w2t;                  // scratch [H][H]: W2 transposed, the backward pass's operand on the older tensor-core path
+  float* wpack;                // scratch: split copies of W1, W2 (both networks) and W2^T for the tensor-core products
   int ldg;                     // row stride of g (A for the Q head, A + 1 with the value head's entry in column A)
   int value_head;              // 1: policy + value heads (PPO), theta carries Wv, bv after b3
   // PPO only
@@ -225,6 +226,24 @@ cudaError_t launch_eligible(const int* block_ver, int n_blocks, long long v_lear
 cudaError_t launch_sample_gather(const SampleParams& p, cudaStream_t s);
 cudaError_t launch_td(const TdParams& p, cudaStream_t s);
 int td_grid(int n);
+constexpr int SG_SPLITS = 32;     // at most this many row ranges per gradient product (partial sums go through scratch)
+// tensor-core products of the update (csrc/tj_sgd_tc.cu): C = epilogue(A B^T), B split and laid out once per update
+enum { GM_BIAS_RELU = 0, GM_BIAS = 1, GM_MASK = 2 };   // relu(acc + bias[n]) | acc + bias[n] | acc where mask[m][n] > 0, else 0
+struct TcGemm {
+  const float* A; int lda;      // M x K row-major, 16-byte rows
+  const float* Bpack;           // B (N x K) as launch_pack_tf32_operands wrote it
+  float* C; int ldc;            // M x N
+  int M, N, K;
+  const float* bias;            // GM_BIAS_RELU
+  const float* mask; int ldm;   // GM_MASK
+};
+struct TcGemmBatch { TcGemm g[2]; int n; };
+struct TcPackJob { const float* W; int ld; int transpose; int N, K; float* dst; };
+struct TcPackJobs { TcPackJob j[6]; int n; };
+bool tc_gemm2_ok(const float* A, int lda, int M, int N, int K);
+size_t tc_pack_floats(int N, int K);
+cudaError_t launch_pack_tf32_operands(const TcPackJobs& jobs, cudaStream_t s);
+cudaError_t launch_gemm_tc2(const TcGemmBatch& batch, int epi, unsigned long long* error, cudaStream_t s);
 size_t sgd_scratch_floats(int max_rows, int D, int H);   // activations, deltas and 32 partial gradients of the blob
 int sgd_partial_count(int n);
 bool sgd_supported(int D, int H, int A);

@@ -140,7 +140,6 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
 // 128 x 64 tile per block (32 x 64 for the heads, whose few outputs would leave most SMs idle with tall tiles), 16 k per
 // step, each thread 8 x 4 (2 x 4); k ascending, one accumulator per output: a fixed order.
 constexpr int GM_BM = 128, GM_BN = 64, GM_BK = 16, GM_THREADS = 256;
-enum { GM_BIAS_RELU = 0, GM_BIAS = 1, GM_MASK = 2 };   // relu(acc + bias[n]) | acc + bias[n] | acc where mask[m][n] > 0, else 0
 
 template <bool B_KN, int EPI, int BM>
 __global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
@@ -626,7 +625,6 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_backward_kernel(const SgdParam
   }
 }
 
-constexpr int SG_SPLITS = 32;     // at most this many row ranges per gradient product (partial sums go through scratch)
 
 // One gradient product of the update: C (M x N, at float offset `off` of the parameter blob) gets (Am rows)^T (Bm rows),
 // a bias (Bm == nullptr) a column of ones.  Tiles of all products are numbered in one list: tile_begin is this product's
@@ -773,7 +771,9 @@ size_t sgd_scratch_floats(int max_rows, int D, int H) {
   // h1, h2, dh1, dh2, g [rows][<= 16 actions + value], loss partials (1 + 5 per 16 rows), and per row range one partial
   // gradient of the whole parameter blob (at most 16 actions and a value head); W2 transposed
   const size_t blob = (size_t)H * D + H + (size_t)H * H + H + 17 * (size_t)H + 17;
-  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)H * H + (size_t)SG_SPLITS * blob;
+  // + split copies of W1 (x 2 networks), W2 (x 2) and W2^T for the tensor-core products
+  return 4 * rows * (size_t)H + rows * 17 + 6 * (rows / SG_ROWS) + 64 + (size_t)H * H + (size_t)SG_SPLITS * blob +
+         2 * tc_pack_floats(H, D) + 3 * tc_pack_floats(H, H) + 64;
 }
 
 int sgd_partial_count(int n) { return (n + SG_ROWS - 1) / SG_ROWS; }
@@ -786,6 +786,11 @@ bool sgd_supported(int D, int H, int A) {
 namespace {
 // the tiled path pays off once a layer is a real matrix product; below that the fused per-16-rows kernels launch less
 bool use_tiled(const SgdParams& p) { return !p.value_head && p.H >= 128 && p.n >= 512; }
+// wide layers with enough 128 x 256 tiles: the pre-split tensor-core products (both hidden layers must qualify)
+bool use_tc2(const SgdParams& p) {
+  return use_tiled(p) && p.wpack && tc_gemm2_ok(p.obs, p.D, p.n, p.H, p.D) && tc_gemm2_ok(p.next_obs, p.D, p.n, p.H, p.D) &&
+         tc_gemm2_ok(p.h1, p.H, p.n, p.H, p.H);
+}
 
 // the backward pass and every parameter update: C -= lr * (gradient rows)^T (input rows), a bias with a column of ones
 cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* adam, cudaStream_t s) {
@@ -798,7 +803,13 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     const float* W2m = p.theta + (size_t)H * D + H;
     const float* W3m = W2m + (size_t)H * H + H;
     sg_gemm<true, GM_MASK>(p.g, p.ldg, W3m, H, p.dh2, H, p.n, H, A, nullptr, p.h2, H, s);
-    if (tc_gemm_ok(p.dh2, H, p.w2t, H, p.n, H, H)) {
+    if (use_tc2(p)) {
+      // W2^T was split with the other weight matrices at the start of the step
+      TcGemmBatch b{};
+      b.g[0] = TcGemm{p.dh2, H, p.wpack + 2 * tc_pack_floats(H, D) + 2 * tc_pack_floats(H, H), p.dh1, H, p.n, H, H, nullptr, p.h1, H};
+      b.n = 1;
+      if ((e = launch_gemm_tc2(b, GM_MASK, p.error, s)) != cudaSuccess) return e;
+    } else if (tc_gemm_ok(p.dh2, H, p.w2t, H, p.n, H, H)) {
       // the tensor-core product wants both operands K-major: dh1 = dh2 (W2^T)^T with W2^T written out first
       sg_transpose_kernel<<<dim3((H + 31) / 32, (H + 31) / 32), 256, 0, s>>>(W2m, p.w2t, H);
       if ((e = sg_layer<GM_MASK>(p.dh2, H, p.w2t, H, p.dh1, H, p.n, H, H, nullptr, p.h1, H, p.error, s)) != cudaSuccess) return e;
@@ -862,10 +873,11 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
 // backward kernel, the grouped gradient products, the apply pass
 static int backward_launches(const SgdParams& p) {
   if (!use_tiled(p)) return 3;
+  if (use_tc2(p)) return 2 + 2;
   return (tc_gemm_ok(p.dh2, p.H, p.w2t, p.H, p.n, p.H, p.H) ? 3 : 2) + 2;
 }
 
-int sgd_step_launches(const SgdParams& p) { return (use_tiled(p) ? 7 : 1) + backward_launches(p); }
+int sgd_step_launches(const SgdParams& p) { return (use_tiled(p) ? (use_tc2(p) ? 6 : 7) : 1) + backward_launches(p); }
 
 int ppo_step_launches(const SgdParams& p, bool with_stats) { return 1 + (with_stats ? 1 : 0) + backward_launches(p); }
 
@@ -878,12 +890,40 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
     // online network: h1, h2 kept, Q values into g; target network: its activations borrow dh1 / dh2 (free until the
     // backward pass), its Q values then take dh1's place
     cudaError_t e;
-    if ((e = sg_layer<GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
-    if ((e = sg_layer<GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
-    sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
-    if ((e = sg_layer<GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
-    if ((e = sg_layer<GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
-    sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+    if (use_tc2(p)) {
+      // both networks' weight matrices (and W2^T for the backward pass) split once, then each layer of both networks in one launch
+      float* pk_W1 = p.wpack;
+      float* pk_T1 = pk_W1 + tc_pack_floats(H, D);
+      float* pk_W2 = pk_T1 + tc_pack_floats(H, D);
+      float* pk_T2 = pk_W2 + tc_pack_floats(H, H);
+      float* pk_W2t = pk_T2 + tc_pack_floats(H, H);
+      TcPackJobs jobs{};
+      jobs.j[jobs.n++] = TcPackJob{W1, D, 0, H, D, pk_W1};
+      jobs.j[jobs.n++] = TcPackJob{T1, D, 0, H, D, pk_T1};
+      jobs.j[jobs.n++] = TcPackJob{W2, H, 0, H, H, pk_W2};
+      jobs.j[jobs.n++] = TcPackJob{T2, H, 0, H, H, pk_T2};
+      jobs.j[jobs.n++] = TcPackJob{W2, H, 1, H, H, pk_W2t};
+      if ((e = launch_pack_tf32_operands(jobs, s)) != cudaSuccess) return e;
+      TcGemmBatch l1{};
+      l1.g[0] = TcGemm{p.obs, D, pk_W1, p.h1, H, n, H, D, b1, nullptr, 0};
+      l1.g[1] = TcGemm{p.next_obs, D, pk_T1, p.dh1, H, n, H, D, tb1, nullptr, 0};
+      l1.n = 2;
+      if ((e = launch_gemm_tc2(l1, GM_BIAS_RELU, p.error, s)) != cudaSuccess) return e;
+      TcGemmBatch l2{};
+      l2.g[0] = TcGemm{p.h1, H, pk_W2, p.h2, H, n, H, H, b2, nullptr, 0};
+      l2.g[1] = TcGemm{p.dh1, H, pk_T2, p.dh2, H, n, H, H, tb2, nullptr, 0};
+      l2.n = 2;
+      if ((e = launch_gemm_tc2(l2, GM_BIAS_RELU, p.error, s)) != cudaSuccess) return e;
+      sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
+      sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+    } else {
+      if ((e = sg_layer<GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+      if ((e = sg_layer<GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+      sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
+      if ((e = sg_layer<GM_BIAS_RELU>(p.next_obs, D, T1, D, p.dh1, H, n, H, D, tb1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+      if ((e = sg_layer<GM_BIAS_RELU>(p.dh1, H, T2, H, p.dh2, H, n, H, H, tb2, nullptr, 0, p.error, s)) != cudaSuccess) return e;
+      sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+    }
     sgd_loss_kernel<<<sgd_partial_count(n), 32, 0, s>>>(p, p.dh1);
     return backward_and_update(p, lr, adam, s);
   }

@@ -1,0 +1,250 @@
+// FP32-faithful matrix products of the learner update on the tensor cores (Algorithm 1, update line: the forward layers of
+// both networks and the backward pass's dh1 are dense contractions over 128-512 inputs for thousands of rows).
+//
+// C[M][N] = epilogue(A[M][K] B[N][K]^T): every operand is split into a TF32 high part (the top 19 bits) and the remainder,
+// and C accumulates A_hi B_hi + A_lo B_hi + A_hi B_lo in FP32 in tensor memory (the dropped A_lo B_lo term is 2^-22 of the
+// product, and the tensor core reads each remainder with 11 significant bits: another 2^-22 each).
+//
+// One 128 x 256 tile per thread block, ten warps:
+//   eight worker warps bring A from global memory sixteen columns at a time, split it and write the two parts into one of
+//     four shared-memory stages (K-major core matrices of 8 rows x 16 bytes), one mbarrier arrival per warp and stage;
+//   a copy lane streams B, which `launch_pack_tf32_operands` has split and laid out ONCE per update in exactly the order
+//     and layout the tile consumes (32 KB per 16 columns: high part, low part), into a four-slot ring with bulk copies;
+//   an issuing lane fires the six MMAs (two K = 8 steps x three products, N = 256) of a chunk as soon as its A stage and
+//     B slot are there, and commits free both; nobody else in its warp polls;
+//   the workers then drain the accumulator (bias + ReLU, or the backward pass's ReLU mask) to global memory.
+// Two problems (the online and the target network's layer) can share a launch: blockIdx.z picks the set.
+// Every wait is bounded; a timeout latches the error word, waits for the copies in flight and frees the tensor memory.
+#include "tj_internal.h"
+#include "tj_tc.cuh"
+
+namespace tj {
+
+namespace {
+
+constexpr int T2_M = 128, T2_N = 256, T2_K = 16;
+constexpr int T2_WORKERS = 256, T2_THREADS = T2_WORKERS + 64, T2_PF = 3;
+constexpr int T2_ASTAGES = 4, T2_BSLOTS = 4;
+constexpr int T2_A_PART = T2_M * T2_K * 4;                 // 8 KB: one part of an A stage
+constexpr int T2_A_STAGE = 2 * T2_A_PART;
+constexpr int T2_B_PART = T2_N * T2_K * 4;                 // 16 KB: one part of a B chunk
+constexpr int T2_B_SLOT = 2 * T2_B_PART;
+constexpr uint32_t T2_SBO = (T2_K / 4) * 128u;             // eight rows further: one row group of K/4 core matrices
+
+struct T2Ctl {
+  uint64_t a_ready[T2_ASTAGES], a_free[T2_ASTAGES], b_full[T2_BSLOTS], b_empty[T2_BSLOTS], acc_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr int T2_SMEM_BYTES = T2_ASTAGES * T2_A_STAGE + T2_BSLOTS * T2_B_SLOT + (int)sizeof(T2Ctl) + 1024;
+
+__global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemmBatch batch, int epi, unsigned long long* __restrict__ error) {
+  extern __shared__ uint8_t t2_raw[];
+  uint8_t* a_stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(t2_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* b_slots = a_stages + T2_ASTAGES * T2_A_STAGE;
+  T2Ctl* ctl = reinterpret_cast<T2Ctl*>(b_slots + T2_BSLOTS * T2_B_SLOT);
+  const TcGemm& g = batch.g[blockIdx.z];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m0 = blockIdx.y * T2_M, n0 = blockIdx.x * T2_N;
+  const int M = g.M, N = g.N, K = g.K, lda = g.lda;
+  const int nk = K / T2_K;
+  if (tid == 0) {
+    for (int i = 0; i < T2_ASTAGES; ++i) { mbar_init(&ctl->a_ready[i], T2_WORKERS / 32); mbar_init(&ctl->a_free[i], 1); }
+    for (int i = 0; i < T2_BSLOTS; ++i) { mbar_init(&ctl->b_full[i], 1); mbar_init(&ctl->b_empty[i], 1); }
+    mbar_init(&ctl->acc_full, 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&ctl->tmem_base)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (tid < T2_WORKERS) {
+    // loader mapping: a warp instruction covers eight rows x four 16-byte pieces (64 contiguous bytes per row); warp w
+    // owns rows 16 w .. 16 w + 15 of the tile, a thread two pieces
+    const float* __restrict__ A = g.A;
+    const int r8 = lane >> 2, kq = lane & 3;
+    float4 ra[T2_PF][2];
+    auto fetch = [&](int i, float4 (&fa)[2]) {
+      const int k = i * T2_K + kq * 4;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rr = warp * 16 + h * 8 + r8;
+        fa[h] = (m0 + rr < M) ? __ldg(reinterpret_cast<const float4*>(A + (size_t)(m0 + rr) * lda + k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    auto split_store = [](uint8_t* hi_dst, uint8_t* lo_dst, const float4 v) {
+      float4 hi, lo;
+      hi.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); lo.x = v.x - hi.x;
+      hi.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); lo.y = v.y - hi.y;
+      hi.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); lo.z = v.z - hi.z;
+      hi.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); lo.w = v.w - hi.w;
+      *reinterpret_cast<float4*>(hi_dst) = hi;
+      *reinterpret_cast<float4*>(lo_dst) = lo;
+    };
+    bool ok = true;
+    auto step = [&](int i, float4 (&fa)[2]) {
+      const int st = i % T2_ASTAGES;
+      uint8_t* base = a_stages + (size_t)st * T2_A_STAGE;
+      if (i >= T2_ASTAGES) ok = tc_wait_elect(&ctl->a_free[st], (uint32_t)(((i / T2_ASTAGES) - 1) & 1), abort_flag);
+      if (!ok) return;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rr = warp * 16 + h * 8 + r8;
+        const size_t off = (size_t)(rr >> 3) * T2_SBO + (size_t)(rr & 7) * 16 + (size_t)kq * 128;
+        split_store(base + off, base + T2_A_PART + off, fa[h]);
+      }
+      fence_async_smem();
+      mbar_arrive_warp(&ctl->a_ready[st]);
+      if (i + T2_PF < nk) fetch(i + T2_PF, fa);
+    };
+#pragma unroll
+    for (int pf = 0; pf < T2_PF; ++pf)
+      if (pf < nk) fetch(pf, ra[pf]);
+    for (int i = 0; i < nk && ok; i += T2_PF) {
+#pragma unroll
+      for (int pf = 0; pf < T2_PF; ++pf)
+        if (ok && i + pf < nk) step(i + pf, ra[pf]);
+    }
+  } else if (warp == T2_WORKERS / 32) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_tf32(T2_N);
+      const uint32_t a0 = smem_addr(a_stages), b0 = smem_addr(b_slots);
+      for (int i = 0; i < nk; ++i) {
+        const int st = i % T2_ASTAGES, sl = i % T2_BSLOTS;
+        if (!tc_wait(&ctl->a_ready[st], (uint32_t)((i / T2_ASTAGES) & 1), abort_flag)) break;
+        if (!tc_wait(&ctl->b_full[sl], (uint32_t)((i / T2_BSLOTS) & 1), abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_hi = a0 + (uint32_t)st * T2_A_STAGE, a_lo = a_hi + T2_A_PART;
+        const uint32_t b_hi = b0 + (uint32_t)sl * T2_B_SLOT, b_lo = b_hi + T2_B_PART;
+#pragma unroll
+        for (int j = 0; j < T2_K / 8; ++j) {
+          const uint32_t o = (uint32_t)j * 256u;     // eight columns further: two core matrices
+          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, (i | j) != 0);
+          umma_tf32(tmem, make_desc(a_lo + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, true);
+          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_lo + o, 128u, T2_SBO), idesc, true);
+        }
+        umma_commit(&ctl->a_free[st]);
+        umma_commit(&ctl->b_empty[sl]);
+      }
+      umma_commit(&ctl->acc_full);
+    }
+    __syncwarp();
+  } else {
+    if (lane == 0) {
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(g.Bpack) + (size_t)blockIdx.x * nk * T2_B_SLOT;
+      int issued = 0;
+      for (int i = 0; i < nk; ++i, ++issued) {
+        const int sl = i % T2_BSLOTS;
+        if (i >= T2_BSLOTS && !tc_wait(&ctl->b_empty[sl], (uint32_t)(((i / T2_BSLOTS) - 1) & 1), abort_flag)) break;
+        mbar_expect_tx(&ctl->b_full[sl], (uint32_t)T2_B_SLOT);
+        bulk_copy_g2s(b_slots + (size_t)sl * T2_B_SLOT, src + (size_t)i * T2_B_SLOT, (uint32_t)T2_B_SLOT, &ctl->b_full[sl]);
+      }
+      // after a timeout elsewhere the last copies may still be on their way: they must land before the block leaves
+      if (*abort_flag)
+        for (int i = issued > T2_BSLOTS ? issued - T2_BSLOTS : 0; i < issued; ++i)
+          if (!tc_wait(&ctl->b_full[i % T2_BSLOTS], (uint32_t)((i / T2_BSLOTS) & 1), abort_flag)) break;
+    }
+    __syncwarp();
+  }
+
+  // after a timeout the abort flag is up and the tile is not written
+  tc_wait_elect(&ctl->acc_full, 0u, abort_flag);
+  __syncthreads();
+  const bool good = *abort_flag == 0;
+  if (good && tid < T2_WORKERS) {
+    tc_fence_after();
+    const int q = warp & 3, half = warp >> 2;      // TMEM lane quarter of this warp, column half
+    const int m = m0 + q * 32 + lane;
+    const uint32_t t_acc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * (T2_N / 2));
+    float* __restrict__ C = g.C;
+    const float* __restrict__ bias = g.bias;
+    const float* __restrict__ mask = g.mask;
+#pragma unroll 1
+    for (int c0 = 0; c0 < T2_N / 2; c0 += 32) {
+      uint32_t v[32];
+      tmem_ld16(t_acc + (uint32_t)c0, v);
+      tmem_ld16(t_acc + (uint32_t)c0 + 16u, v + 16);
+      tmem_ld_wait();
+      if (m < M) {
+        const int n = n0 + half * (T2_N / 2) + c0;
+        float* dst = C + (size_t)m * g.ldc + n;
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          float4 o = make_float4(__uint_as_float(v[c4 * 4]), __uint_as_float(v[c4 * 4 + 1]), __uint_as_float(v[c4 * 4 + 2]),
+                                 __uint_as_float(v[c4 * 4 + 3]));
+          if (epi == GM_BIAS_RELU) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + n + c4 * 4));
+            o.x = fmaxf(o.x + b.x, 0.f); o.y = fmaxf(o.y + b.y, 0.f); o.z = fmaxf(o.z + b.z, 0.f); o.w = fmaxf(o.w + b.w, 0.f);
+          } else {
+            const float4 k = __ldg(reinterpret_cast<const float4*>(mask + (size_t)m * g.ldm + n + c4 * 4));
+            o.x = k.x > 0.f ? o.x : 0.f; o.y = k.y > 0.f ? o.y : 0.f; o.z = k.z > 0.f ? o.z : 0.f; o.w = k.w > 0.f ? o.w : 0.f;
+          }
+          *reinterpret_cast<float4*>(dst + c4 * 4) = o;
+        }
+      }
+    }
+  } else if (!good && tid == 0) {
+    atomicExch(error, 3ull);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  }
+}
+
+// W (N x K row-major, or K x N when `transpose`) -> TF32 high part and remainder in the order the product kernel streams
+// them: per tile of 256 rows and chunk of 16 columns one 32 KB block [high 256 x 16 | low 256 x 16], each part as K-major
+// core matrices (8 rows x 4 columns contiguous; element (n, k) at ((n / 8) * 4 + k / 4) * 32 + (n % 8) * 4 + k % 4).
+__global__ void __launch_bounds__(256) sg_pack_tf32_kernel(const TcPackJobs jobs) {
+  const TcPackJob& jb = jobs.j[blockIdx.y];
+  const int total = jb.N * jb.K, nk = jb.K / T2_K;
+  constexpr int PER = T2_N * T2_K;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int chunk = i / PER, within = i % PER;
+    const int tile = chunk / nk, c = chunk % nk;
+    const int core = within / 32, in_core = within % 32;
+    const int n = tile * T2_N + (core / 4) * 8 + in_core / 4, k = c * T2_K + (core % 4) * 4 + in_core % 4;
+    const float v = jb.transpose ? jb.W[(size_t)k * jb.ld + n] : jb.W[(size_t)n * jb.ld + k];
+    const float hi = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
+    float* d = jb.dst + (size_t)chunk * (2 * PER);
+    d[within] = hi;
+    d[PER + within] = v - hi;
+  }
+}
+
+}  // namespace
+
+bool tc_gemm2_ok(const float* A, int lda, int M, int N, int K) {
+  const long long tiles = (long long)((M + T2_M - 1) / T2_M) * (N / T2_N);
+  return N % T2_N == 0 && K % T2_K == 0 && K >= 2 * T2_K && (lda & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0 && tiles >= 48;
+}
+
+size_t tc_pack_floats(int N, int K) { return (size_t)2 * N * K; }
+
+cudaError_t launch_pack_tf32_operands(const TcPackJobs& jobs, cudaStream_t s) {
+  if (jobs.n <= 0) return cudaSuccess;
+  sg_pack_tf32_kernel<<<dim3(128, jobs.n), 256, 0, s>>>(jobs);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc2(const TcGemmBatch& batch, int epi, unsigned long long* error, cudaStream_t s) {
+  if (batch.n <= 0) return cudaSuccess;
+  const TcGemm& g0 = batch.g[0];
+  for (int i = 1; i < batch.n; ++i)
+    if (batch.g[i].M != g0.M || batch.g[i].N != g0.N) return cudaErrorInvalidValue;   // one grid for all problems of a launch
+  cudaError_t e = cudaFuncSetAttribute(sg_gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T2_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  sg_gemm_tc2_kernel<<<dim3(g0.N / T2_N, (g0.M + T2_M - 1) / T2_M, batch.n), T2_THREADS, T2_SMEM_BYTES, s>>>(batch, epi, error);
+  return cudaGetLastError();
+}
+
+}  // namespace tj
