@@ -240,6 +240,12 @@ struct TcGemm {
 struct TcGemmBatch { TcGemm g[2]; int n; };
 struct TcPackJob { const float* W; int ld; int transpose; int N, K; float* dst; };
 struct TcPackJobs { TcPackJob j[6]; int n; };
+struct TcWgrad { const float* Am; int lda; const float* Bm; int ldb; int M, N; int off; int tile_begin; };   // dW = Am^T Bm
+struct TcWgradBatch { TcWgrad g[2]; int n; int n_tiles; };
+bool tc_wgrad_ok(int M, int N, int rows);
+int tc_wgrad_tiles(int M, int N);
+cudaError_t launch_wgrad_tc(const TcWgradBatch& batch, float* P, int count, int n_rows, int rows_per_range, int n_ranges,
+                            unsigned long long* error, cudaStream_t s);
 bool tc_gemm2_ok(const float* A, int lda, int M, int N, int K);
 size_t tc_pack_floats(int N, int K);
 cudaError_t launch_pack_tf32_operands(const TcPackJobs& jobs, cudaStream_t s);

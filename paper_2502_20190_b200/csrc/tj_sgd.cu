@@ -848,9 +848,19 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     const int tm = M >= 128 ? 128 : 64;   // as the kernel picks it
     gp.n_tiles += ((M + tm - 1) / tm) * ((N + GP_TILE - 1) / GP_TILE);
   };
-  add(W1, H, D, p.dh1, H, p.obs, D);
+  // the two large products (W2, W1) on the tensor cores where the shapes allow; the rest on the FMA tiles
+  TcWgradBatch tb{};
+  auto add_tc = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
+    TcWgrad& d = tb.g[tb.n++];
+    d = TcWgrad{Am, lda, Bm, ldb, M, N, (int)(C - p.theta), tb.n_tiles};
+    tb.n_tiles += tc_wgrad_tiles(M, N);
+  };
+  const bool tc_grads = use_tc2(p);
+  if (tc_grads && tc_wgrad_ok(H, H, p.n)) add_tc(W2, H, H, p.dh2, H, p.h1, H);
+  else add(W2, H, H, p.dh2, H, p.h1, H);
+  if (tc_grads && tc_wgrad_ok(H, D, p.n)) add_tc(W1, H, D, p.dh1, H, p.obs, D);
+  else add(W1, H, D, p.dh1, H, p.obs, D);
   add(b1, H, 1, p.dh1, H, nullptr, 0);
-  add(W2, H, H, p.dh2, H, p.h1, H);
   add(b2, H, 1, p.dh2, H, nullptr, 0);
   add(W3, A, H, p.g, p.ldg, p.h2, H);
   add(b3, A, 1, p.g, p.ldg, nullptr, 0);
@@ -859,6 +869,7 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     add(bv, 1, 1, p.g + A, p.ldg, nullptr, 0);
   }
   const int count = (int)((p.value_head ? bv + 1 : b3 + A) - p.theta);
+  if (tb.n && (e = launch_wgrad_tc(tb, p.grad_partial, count, p.n, rows_per_range, n_ranges, p.error, s)) != cudaSuccess) return e;
   sgd_grad_partial_kernel<<<dim3(gp.n_tiles, n_ranges), 256, 0, s>>>(p.grad_partial, gp, count, p.n, rows_per_range);
   if (adam)
     sgd_apply_adam_kernel<<<(count + 255) / 256, 256, 0, s>>>(p.theta, adam->m, adam->v, p.grad_partial, count, n_ranges, lr, adam->beta1,
@@ -873,7 +884,7 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
 // backward kernel, the grouped gradient products, the apply pass
 static int backward_launches(const SgdParams& p) {
   if (!use_tiled(p)) return 3;
-  if (use_tc2(p)) return 2 + 2;
+  if (use_tc2(p)) return 2 + 2 + ((tc_wgrad_ok(p.H, p.H, p.n) || tc_wgrad_ok(p.H, p.D, p.n)) ? 1 : 0);
   return (tc_gemm_ok(p.dh2, p.H, p.w2t, p.H, p.n, p.H, p.H) ? 3 : 2) + 2;
 }
 

@@ -48,6 +48,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
   const int m0 = blockIdx.y * T2_M, n0 = blockIdx.x * T2_N;
   const int M = g.M, N = g.N, K = g.K, lda = g.lda;
   const int nk = K / T2_K;
+  // Blocks that share a tile of B walk the K chunks in rotated order, so that they do not all ask L2 for the same 32 KB at
+  // the same moment; step i of this block is chunk (i + rot) mod nk.  The order of a block's sums depends on its row tile only.
+  const int rot = (int)((blockIdx.y * 5u + blockIdx.z * 3u) % (unsigned)nk);
   if (tid == 0) {
     for (int i = 0; i < T2_ASTAGES; ++i) { mbar_init(&ctl->a_ready[i], T2_WORKERS / 32); mbar_init(&ctl->a_free[i], 1); }
     for (int i = 0; i < T2_BSLOTS; ++i) { mbar_init(&ctl->b_full[i], 1); mbar_init(&ctl->b_empty[i], 1); }
@@ -72,7 +75,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
     const int r8 = lane >> 2, kq = lane & 3;
     float4 ra[T2_PF][2];
     auto fetch = [&](int i, float4 (&fa)[2]) {
-      const int k = i * T2_K + kq * 4;
+      const int c = i + rot < nk ? i + rot : i + rot - nk;
+      const int k = c * T2_K + kq * 4;
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int rr = warp * 16 + h * 8 + r8;
@@ -144,7 +148,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
         const int sl = i % T2_BSLOTS;
         if (i >= T2_BSLOTS && !tc_wait(&ctl->b_empty[sl], (uint32_t)(((i / T2_BSLOTS) - 1) & 1), abort_flag)) break;
         mbar_expect_tx(&ctl->b_full[sl], (uint32_t)T2_B_SLOT);
-        bulk_copy_g2s(b_slots + (size_t)sl * T2_B_SLOT, src + (size_t)i * T2_B_SLOT, (uint32_t)T2_B_SLOT, &ctl->b_full[sl]);
+        const int c = i + rot < nk ? i + rot : i + rot - nk;
+        bulk_copy_g2s(b_slots + (size_t)sl * T2_B_SLOT, src + (size_t)c * T2_B_SLOT, (uint32_t)T2_B_SLOT, &ctl->b_full[sl]);
       }
       // after a timeout elsewhere the last copies may still be on their way: they must land before the block leaves
       if (*abort_flag)
@@ -187,6 +192,188 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
             o.x = k.x > 0.f ? o.x : 0.f; o.y = k.y > 0.f ? o.y : 0.f; o.z = k.z > 0.f ? o.z : 0.f; o.w = k.w > 0.f ? o.w : 0.f;
           }
           *reinterpret_cast<float4*>(dst + c4 * 4) = o;
+        }
+      }
+    }
+  } else if (!good && tid == 0) {
+    atomicExch(error, 3ull);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  }
+}
+
+// Weight-gradient products on the same tensor-core path: dW[m][n] = sum over minibatch rows r of G[r][m] X[r][n] (G the
+// gradient rows of a layer, X its input rows).  The contraction runs over the rows, so both operands are K-major only after a
+// transposition, which the workers do on the way from global memory to shared memory: a thread reads one feature of four
+// consecutive rows (a warp 32 consecutive features of a row per load: coalesced), which is exactly one 16-byte word of the
+// K-major core-matrix layout, splits it and stores both parts.  One thread block = one 128 x 256 (or 128 x 128) tile of one
+// product over one range of rows; it writes its sums to P[range][off + m * N + n], a partial gradient laid out like the
+// parameter blob, and the apply kernel adds the ranges in order (no atomics, one fixed order).
+constexpr int WG_STAGES = 4;
+constexpr int WG_A_PART = T2_M * T2_K * 4, WG_B_PART = T2_N * T2_K * 4;          // 8 KB, 16 KB
+constexpr int WG_STAGE = 2 * WG_A_PART + 2 * WG_B_PART;                          // A_hi | A_lo | B_hi | B_lo: 48 KB
+struct WgCtl {
+  uint64_t ready[WG_STAGES], free_[WG_STAGES], acc_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE + (int)sizeof(WgCtl) + 1024;
+
+__global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgradBatch batch, float* __restrict__ P, int count, int n_rows,
+                                                                    int rows_per_range, unsigned long long* __restrict__ error) {
+  extern __shared__ uint8_t wg_raw[];
+  uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(wg_raw) + 1023) & ~(uintptr_t)1023);
+  WgCtl* ctl = reinterpret_cast<WgCtl*>(stages + WG_STAGES * WG_STAGE);
+  int q = 0;
+  while (q + 1 < batch.n && (int)blockIdx.x >= batch.g[q + 1].tile_begin) ++q;
+  const TcWgrad& g = batch.g[q];
+  const int BN = g.N % T2_N == 0 ? T2_N : 128;                 // columns of this product's tiles
+  const int t = blockIdx.x - g.tile_begin, tiles_n = g.N / BN;
+  const int m0 = (t / tiles_n) * T2_M, n0 = (t % tiles_n) * BN;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int j_begin = blockIdx.y * rows_per_range;
+  const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
+  const int nk = j_end > j_begin ? (j_end - j_begin + T2_K - 1) / T2_K : 0;
+  if (tid == 0) {
+    for (int i = 0; i < WG_STAGES; ++i) { mbar_init(&ctl->ready[i], T2_WORKERS / 32); mbar_init(&ctl->free_[i], 1); }
+    mbar_init(&ctl->acc_full, 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&ctl->tmem_base)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (tid < T2_WORKERS) {
+    // task u of a thread: feature (tid + 256 u) mod F of row group (tid + 256 u) / F, F = 128 (A) or BN (B)
+    const float* __restrict__ Am = g.Am;
+    const float* __restrict__ Bm = g.Bm;
+    const int lda = g.lda, ldb = g.ldb;
+    const int nb_tasks = BN / 64;                               // 4 or 2 per thread
+    float4 ra[2][2], rb[2][4];
+    auto load4 = [&](const float* base, int ld, int j, int col) -> float4 {
+      float4 v;
+      v.x = j < j_end ? __ldg(base + (size_t)j * ld + col) : 0.f;
+      v.y = j + 1 < j_end ? __ldg(base + (size_t)(j + 1) * ld + col) : 0.f;
+      v.z = j + 2 < j_end ? __ldg(base + (size_t)(j + 2) * ld + col) : 0.f;
+      v.w = j + 3 < j_end ? __ldg(base + (size_t)(j + 3) * ld + col) : 0.f;
+      return v;
+    };
+    auto fetch = [&](int i, float4 (&fa)[2], float4 (&fb)[4]) {
+      const int j0 = j_begin + i * T2_K;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int task = tid + 256 * u;
+        fa[u] = load4(Am, lda, j0 + (task >> 7) * 4, m0 + (task & 127));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (u < nb_tasks) {
+          const int task = tid + 256 * u;
+          fb[u] = BN == T2_N ? load4(Bm, ldb, j0 + (task >> 8) * 4, n0 + (task & 255)) : load4(Bm, ldb, j0 + (task >> 7) * 4, n0 + (task & 127));
+        }
+      }
+    };
+    auto split_store = [](uint8_t* hi_dst, uint8_t* lo_dst, const float4 v) {
+      float4 hi, lo;
+      hi.x = __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u); lo.x = v.x - hi.x;
+      hi.y = __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u); lo.y = v.y - hi.y;
+      hi.z = __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u); lo.z = v.z - hi.z;
+      hi.w = __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u); lo.w = v.w - hi.w;
+      *reinterpret_cast<float4*>(hi_dst) = hi;
+      *reinterpret_cast<float4*>(lo_dst) = lo;
+    };
+    bool ok = true;
+    auto step = [&](int i, float4 (&fa)[2], float4 (&fb)[4]) {
+      const int st = i % WG_STAGES;
+      uint8_t* base = stages + (size_t)st * WG_STAGE;
+      if (i >= WG_STAGES) ok = tc_wait_elect(&ctl->free_[st], (uint32_t)(((i / WG_STAGES) - 1) & 1), abort_flag);
+      if (!ok) return;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int task = tid + 256 * u, f = task & 127, kg = task >> 7;
+        const size_t off = (size_t)((f >> 3) * 4 + kg) * 128 + (size_t)(f & 7) * 16;
+        split_store(base + off, base + WG_A_PART + off, fa[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (u < nb_tasks) {
+          const int task = tid + 256 * u;
+          const int f = BN == T2_N ? (task & 255) : (task & 127), kg = BN == T2_N ? (task >> 8) : (task >> 7);
+          const size_t off = (size_t)((f >> 3) * 4 + kg) * 128 + (size_t)(f & 7) * 16;
+          split_store(base + 2 * WG_A_PART + off, base + 2 * WG_A_PART + WG_B_PART + off, fb[u]);
+        }
+      }
+      fence_async_smem();
+      mbar_arrive_warp(&ctl->ready[st]);
+      if (i + 2 < nk) fetch(i + 2, fa, fb);
+    };
+    if (0 < nk) fetch(0, ra[0], rb[0]);
+    if (1 < nk) fetch(1, ra[1], rb[1]);
+    for (int i = 0; i < nk && ok; i += 2) {
+      step(i, ra[0], rb[0]);
+      if (ok && i + 1 < nk) step(i + 1, ra[1], rb[1]);
+    }
+  } else if (warp == T2_WORKERS / 32) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_tf32(BN);
+      const uint32_t s0 = smem_addr(stages);
+      for (int i = 0; i < nk; ++i) {
+        const int st = i % WG_STAGES;
+        if (!tc_wait(&ctl->ready[st], (uint32_t)((i / WG_STAGES) & 1), abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_hi = s0 + (uint32_t)st * WG_STAGE, a_lo = a_hi + WG_A_PART, b_hi = a_hi + 2 * WG_A_PART, b_lo = b_hi + WG_B_PART;
+#pragma unroll
+        for (int j = 0; j < T2_K / 8; ++j) {
+          const uint32_t o = (uint32_t)j * 256u;     // eight rows of the minibatch further: two core matrices
+          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, (i | j) != 0);
+          umma_tf32(tmem, make_desc(a_lo + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, true);
+          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_lo + o, 128u, T2_SBO), idesc, true);
+        }
+        umma_commit(&ctl->free_[st]);
+      }
+      umma_commit(&ctl->acc_full);
+    }
+    __syncwarp();
+  }
+
+  tc_wait_elect(&ctl->acc_full, 0u, abort_flag);
+  __syncthreads();
+  const bool good = *abort_flag == 0;
+  if (good && tid < T2_WORKERS) {
+    tc_fence_after();
+    const int q4 = warp & 3, half = warp >> 2;      // TMEM lane quarter of this warp, column half
+    const int m = m0 + q4 * 32 + lane;
+    const int cols = BN / 2;
+    const uint32_t t_acc = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * cols);
+    float* dst_row = P + (size_t)blockIdx.y * count + g.off + (size_t)m * g.N + n0 + half * cols;
+#pragma unroll 1
+    for (int c0 = 0; c0 < cols; c0 += 32) {
+      uint32_t v[32];
+      if (nk > 0) {
+        tmem_ld16(t_acc + (uint32_t)c0, v);
+        tmem_ld16(t_acc + (uint32_t)c0 + 16u, v + 16);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = 0u;       // an empty range of rows contributes nothing
+      }
+      if (m < g.M) {
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          float* d = dst_row + c0 + c4 * 4;           // the blob's matrices start at any multiple of four bytes: scalar stores
+          d[0] = __uint_as_float(v[c4 * 4]); d[1] = __uint_as_float(v[c4 * 4 + 1]);
+          d[2] = __uint_as_float(v[c4 * 4 + 2]); d[3] = __uint_as_float(v[c4 * 4 + 3]);
         }
       }
     }
@@ -244,6 +431,19 @@ cudaError_t launch_gemm_tc2(const TcGemmBatch& batch, int epi, unsigned long lon
   cudaError_t e = cudaFuncSetAttribute(sg_gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, T2_SMEM_BYTES);
   if (e != cudaSuccess) return e;
   sg_gemm_tc2_kernel<<<dim3(g0.N / T2_N, (g0.M + T2_M - 1) / T2_M, batch.n), T2_THREADS, T2_SMEM_BYTES, s>>>(batch, epi, error);
+  return cudaGetLastError();
+}
+
+bool tc_wgrad_ok(int M, int N, int rows) { return M % T2_M == 0 && N % 128 == 0 && rows >= 1024; }
+
+int tc_wgrad_tiles(int M, int N) { return (M / T2_M) * (N / (N % T2_N == 0 ? T2_N : 128)); }
+
+cudaError_t launch_wgrad_tc(const TcWgradBatch& batch, float* P, int count, int n_rows, int rows_per_range, int n_ranges,
+                            unsigned long long* error, cudaStream_t s) {
+  if (batch.n <= 0 || batch.n_tiles <= 0) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(sg_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, WG_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  sg_wgrad_tc_kernel<<<dim3(batch.n_tiles, n_ranges), T2_THREADS, WG_SMEM_BYTES, s>>>(batch, P, count, n_rows, rows_per_range, error);
   return cudaGetLastError();
 }
 

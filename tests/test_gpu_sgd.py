@@ -62,11 +62,14 @@ def test_sgd_step_on_the_tensor_core_path_matches_oracle(env):
     _check_sgd_step(env, 2, 16, 5, 500, 512, 3100, 0, rtol=RTOL_TF32X3)
 
 
-def test_sgd_step_on_the_presplit_tensor_core_path_matches_oracle(env):
-    """Hidden 512 (two 256-column tiles) and 3,100 rows (25 row tiles, the last one ragged): both hidden layers of both
-    networks and dh1 run as 128 x 256 tensor-core tiles whose weight operand was split once per update.  Same three
-    products per tile as the path above, same tolerance."""
-    _check_sgd_step(env, 2, 32, 5, 512, 512, 3100, 0, rtol=RTOL_TF32X3)
+@pytest.mark.parametrize("D", [32, 128])
+def test_sgd_step_on_the_presplit_tensor_core_path_matches_oracle(env, D):
+    """Hidden 512 (two 256-column tiles) and 3,100 rows (25 row tiles, the last one ragged; row ranges of the weight
+    gradients that end inside a chunk): both hidden layers of both networks and dh1 run as 128 x 256 tensor-core tiles
+    whose weight operand was split once per update, and the weight gradients of W2 (256-column tiles) and, with 128
+    inputs, of W1 (128-column tiles) as tensor-core products over the minibatch rows.  Same three products per tile as
+    the path above, same tolerance."""
+    _check_sgd_step(env, 2, D, 5, 512, 512, 3100, 0, rtol=RTOL_TF32X3)
 
 
 def _relu_gate_allowance(theta, D, H, A, obs, act, lr, kappa, margin=2e-6):
