@@ -691,6 +691,7 @@ void lay_out_update_scratch(const tj_ctx* x, tj::SgdParams& p) {
     float* w = p.grad_partial + (size_t)tj::SG_SPLITS * blob;
     w += (32 - ((reinterpret_cast<uintptr_t>(w) / sizeof(float)) & 31)) & 31;
     p.wpack = w;
+    p.sm_count = x->sm_count;
   }
 }
 

@@ -109,6 +109,7 @@ struct SgdParams {
   float* partial;              // scratch: one Huber partial sum per 16 rows
   float* grad_partial;         // scratch: per row range one partial gradient laid out like the parameter blob
   float* w2t;                  // scratch [H][H]: W2 transposed, the backward pass's operand on the older tensor-core path
+  int sm_count;                // SMs of the device (sizes the row ranges of the tensor-core gradient products)
   float* wpack;                // scratch: split copies of W1, W2 (both networks) and W2^T for the tensor-core products
   int ldg;                     // row stride of g (A for the Q head, A + 1 with the value head's entry in column A)
   int value_head;              // 1: policy + value heads (PPO), theta carries Wv, bv after b3
@@ -240,9 +241,10 @@ struct TcGemm {
 struct TcGemmBatch { TcGemm g[2]; int n; };
 struct TcPackJob { const float* W; int ld; int transpose; int N, K; float* dst; };
 struct TcPackJobs { TcPackJob j[6]; int n; };
-struct TcWgrad { const float* Am; int lda; const float* Bm; int ldb; int M, N; int off; int tile_begin; };   // dW = Am^T Bm
-struct TcWgradBatch { TcWgrad g[2]; int n; int n_tiles; };
-bool tc_wgrad_ok(int M, int N, int rows);
+// dW = Am^T Bm for Am [rows][M], Bm [rows][N]; bias_off >= 0: the column sums of Am (the bias gradient) go to that offset
+struct TcWgrad { const float* Am; int lda; const float* Bm; int ldb; int M, N; int off; int bias_off; int tile_begin; };
+struct TcWgradBatch { TcWgrad g[4]; int n; int n_tiles; };
+bool tc_wgrad_ok(int N, int rows);
 int tc_wgrad_tiles(int M, int N);
 cudaError_t launch_wgrad_tc(const TcWgradBatch& batch, float* P, int count, int n_rows, int rows_per_range, int n_ranges,
                             unsigned long long* error, cudaStream_t s);

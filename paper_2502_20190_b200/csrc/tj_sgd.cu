@@ -142,9 +142,9 @@ __global__ void __launch_bounds__(SG_THREADS) sgd_forward_kernel(const SgdParams
 constexpr int GM_BM = 128, GM_BN = 64, GM_BK = 16, GM_THREADS = 256;
 
 template <bool B_KN, int EPI, int BM>
-__global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
-                                                             float* __restrict__ C, int ldc, int M, int N, int K,
-                                                             const float* __restrict__ bias, const float* __restrict__ mask, int ldm) {
+__device__ __forceinline__ void sg_gemm_body(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+                                             float* __restrict__ C, int ldc, int M, int N, int K,
+                                             const float* __restrict__ bias, const float* __restrict__ mask, int ldm) {
   __shared__ __align__(16) float As[GM_BK][BM + 4];
   __shared__ __align__(16) float Bs[GM_BK][GM_BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -252,6 +252,21 @@ __global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __rest
       C[(size_t)m * ldc + n] = v;
     }
   }
+}
+
+template <bool B_KN, int EPI, int BM>
+__global__ void __launch_bounds__(GM_THREADS) sg_gemm_kernel(const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+                                                             float* __restrict__ C, int ldc, int M, int N, int K,
+                                                             const float* __restrict__ bias, const float* __restrict__ mask, int ldm) {
+  sg_gemm_body<B_KN, EPI, BM>(A, lda, B, ldb, C, ldc, M, N, K, bias, mask, ldm);
+}
+
+// the same product for two operand sets of one shape in one launch (the two networks' heads): blockIdx.z picks the set
+struct GemmPair { const float* A[2]; const float* B[2]; float* C[2]; const float* bias[2]; };
+template <bool B_KN, int EPI, int BM>
+__global__ void __launch_bounds__(GM_THREADS) sg_gemm_pair_kernel(const GemmPair pr, int lda, int ldb, int ldc, int M, int N, int K) {
+  const int z = blockIdx.z;
+  sg_gemm_body<B_KN, EPI, BM>(pr.A[z], lda, pr.B[z], ldb, pr.C[z], ldc, M, N, K, pr.bias[z], nullptr, 0);
 }
 
 template <bool B_KN, int EPI, int BM = GM_BM>
@@ -828,12 +843,9 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
   float* b3 = W3 + (size_t)A * H;
   float* Wv = b3 + A;
   float* bv = Wv + H;
-  int n_ranges = (p.n + 127) / 128;
-  if (n_ranges > SG_SPLITS) n_ranges = SG_SPLITS;
-  const int rows_per_range = ((p.n + n_ranges - 1) / n_ranges + 31) / 32 * 32;
-  n_ranges = (p.n + rows_per_range - 1) / rows_per_range;
-  // the backward pass has read W2 and the heads; now the parameters may change: all products in one launch, then one
-  // pass over the whole blob
+  // the backward pass has read W2 and the heads; now the parameters may change: all products in one or two launches, then
+  // one pass over the whole blob.  Products whose input width is a multiple of 128 go to the tensor cores (with their bias
+  // gradient), the others to the FMA tiles.
   GradProducts gp{};
   auto add = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
     GradProduct& d = gp.g[gp.n++];
@@ -848,29 +860,38 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
     const int tm = M >= 128 ? 128 : 64;   // as the kernel picks it
     gp.n_tiles += ((M + tm - 1) / tm) * ((N + GP_TILE - 1) / GP_TILE);
   };
-  // the two large products (W2, W1) on the tensor cores where the shapes allow; the rest on the FMA tiles
   TcWgradBatch tb{};
-  auto add_tc = [&](float* C, int M, int N, const float* Am, int lda, const float* Bm, int ldb) {
-    TcWgrad& d = tb.g[tb.n++];
-    d = TcWgrad{Am, lda, Bm, ldb, M, N, (int)(C - p.theta), tb.n_tiles};
-    tb.n_tiles += tc_wgrad_tiles(M, N);
-  };
   const bool tc_grads = use_tc2(p);
-  if (tc_grads && tc_wgrad_ok(H, H, p.n)) add_tc(W2, H, H, p.dh2, H, p.h1, H);
-  else add(W2, H, H, p.dh2, H, p.h1, H);
-  if (tc_grads && tc_wgrad_ok(H, D, p.n)) add_tc(W1, H, D, p.dh1, H, p.obs, D);
-  else add(W1, H, D, p.dh1, H, p.obs, D);
-  add(b1, H, 1, p.dh1, H, nullptr, 0);
-  add(b2, H, 1, p.dh2, H, nullptr, 0);
-  add(W3, A, H, p.g, p.ldg, p.h2, H);
-  add(b3, A, 1, p.g, p.ldg, nullptr, 0);
-  if (p.value_head) {
-    add(Wv, 1, H, p.g + A, p.ldg, p.h2, H);
-    add(bv, 1, 1, p.g + A, p.ldg, nullptr, 0);
+  // one product and its bias: C [M][N] = G^T X, bias [M] = column sums of G
+  auto product = [&](float* C, float* bias, int M, int N, const float* G, int ldg, const float* X, int ldx) {
+    if (tc_grads && tc_wgrad_ok(N, p.n)) {
+      TcWgrad& d = tb.g[tb.n++];
+      d = TcWgrad{G, ldg, X, ldx, M, N, (int)(C - p.theta), (int)(bias - p.theta), tb.n_tiles};
+      tb.n_tiles += tc_wgrad_tiles(M, N);
+    } else {
+      add(C, M, N, G, ldg, X, ldx);
+      add(bias, M, 1, G, ldg, nullptr, 0);
+    }
+  };
+  product(W1, b1, H, D, p.dh1, H, p.obs, D);
+  product(W2, b2, H, H, p.dh2, H, p.h1, H);
+  product(W3, b3, A, H, p.g, p.ldg, p.h2, H);
+  if (p.value_head) product(Wv, bv, 1, H, p.g + A, p.ldg, p.h2, H);
+  // row ranges: with tensor-core tiles about one thread block per SM in all (a block costs a fixed ~10 us beside its rows);
+  // otherwise 128 rows or more per range
+  int n_ranges;
+  if (tb.n_tiles > 0) {
+    n_ranges = (p.sm_count > 0 ? p.sm_count : 148) / tb.n_tiles;
+    if (n_ranges < 1) n_ranges = 1;
+  } else {
+    n_ranges = (p.n + 127) / 128;
   }
+  if (n_ranges > SG_SPLITS) n_ranges = SG_SPLITS;
+  const int rows_per_range = ((p.n + n_ranges - 1) / n_ranges + 31) / 32 * 32;
+  n_ranges = (p.n + rows_per_range - 1) / rows_per_range;
   const int count = (int)((p.value_head ? bv + 1 : b3 + A) - p.theta);
   if (tb.n && (e = launch_wgrad_tc(tb, p.grad_partial, count, p.n, rows_per_range, n_ranges, p.error, s)) != cudaSuccess) return e;
-  sgd_grad_partial_kernel<<<dim3(gp.n_tiles, n_ranges), 256, 0, s>>>(p.grad_partial, gp, count, p.n, rows_per_range);
+  if (gp.n_tiles > 0) sgd_grad_partial_kernel<<<dim3(gp.n_tiles, n_ranges), 256, 0, s>>>(p.grad_partial, gp, count, p.n, rows_per_range);
   if (adam)
     sgd_apply_adam_kernel<<<(count + 255) / 256, 256, 0, s>>>(p.theta, adam->m, adam->v, p.grad_partial, count, n_ranges, lr, adam->beta1,
                                                               adam->beta2, adam->eps, adam->c1, adam->c2);
@@ -884,11 +905,11 @@ cudaError_t backward_and_update(const SgdParams& p, float lr, const AdamParams* 
 // backward kernel, the grouped gradient products, the apply pass
 static int backward_launches(const SgdParams& p) {
   if (!use_tiled(p)) return 3;
-  if (use_tc2(p)) return 2 + 2 + ((tc_wgrad_ok(p.H, p.H, p.n) || tc_wgrad_ok(p.H, p.D, p.n)) ? 1 : 0);
+  if (use_tc2(p)) return 2 + 2 + (tc_wgrad_ok(p.D, p.n) ? 0 : 1);   // hidden-width products always qualify; W1's by obs_dim
   return (tc_gemm_ok(p.dh2, p.H, p.w2t, p.H, p.n, p.H, p.H) ? 3 : 2) + 2;
 }
 
-int sgd_step_launches(const SgdParams& p) { return (use_tiled(p) ? (use_tc2(p) ? 6 : 7) : 1) + backward_launches(p); }
+int sgd_step_launches(const SgdParams& p) { return (use_tiled(p) ? (use_tc2(p) ? 5 : 7) : 1) + backward_launches(p); }
 
 int ppo_step_launches(const SgdParams& p, bool with_stats) { return 1 + (with_stats ? 1 : 0) + backward_launches(p); }
 
@@ -925,8 +946,9 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
       l2.g[1] = TcGemm{p.dh1, H, pk_T2, p.dh2, H, n, H, H, tb2, nullptr, 0};
       l2.n = 2;
       if ((e = launch_gemm_tc2(l2, GM_BIAS_RELU, p.error, s)) != cudaSuccess) return e;
-      sg_gemm<false, GM_BIAS, 32>(p.h2, H, W3, H, p.g, A, n, A, H, b3, nullptr, 0, s);
-      sg_gemm<false, GM_BIAS, 32>(p.dh2, H, T3, H, p.dh1, A, n, A, H, tb3, nullptr, 0, s);
+      // both heads in one launch: Q of the online network into g, of the target network into dh1's place
+      GemmPair heads{{p.h2, p.dh2}, {W3, T3}, {p.g, p.dh1}, {b3, tb3}};
+      sg_gemm_pair_kernel<false, GM_BIAS, 32><<<dim3((A + GM_BN - 1) / GM_BN, (n + 31) / 32, 2), GM_THREADS, 0, s>>>(heads, H, H, A, n, A, H);
     } else {
       if ((e = sg_layer<GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
       if ((e = sg_layer<GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, p.error, s)) != cudaSuccess) return e;

@@ -212,7 +212,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
 // consecutive rows (a warp 32 consecutive features of a row per load: coalesced), which is exactly one 16-byte word of the
 // K-major core-matrix layout, splits it and stores both parts.  One thread block = one 128 x 256 (or 128 x 128) tile of one
 // product over one range of rows; it writes its sums to P[range][off + m * N + n], a partial gradient laid out like the
-// parameter blob, and the apply kernel adds the ranges in order (no atomics, one fixed order).
+// parameter blob, and the apply kernel adds the ranges in order (no atomics, one fixed order).  A product with fewer than 128
+// gradient columns (the head: one column per action) reads zeros beyond them.  The first column tile of a product also
+// writes the bias gradient, the column sums of G over the range: its loaders hold those values anyway.
 constexpr int WG_STAGES = 4;
 constexpr int WG_A_PART = T2_M * T2_K * 4, WG_B_PART = T2_N * T2_K * 4;          // 8 KB, 16 KB
 constexpr int WG_STAGE = 2 * WG_A_PART + 2 * WG_B_PART;                          // A_hi | A_lo | B_hi | B_lo: 48 KB
@@ -220,6 +222,7 @@ struct WgCtl {
   uint64_t ready[WG_STAGES], free_[WG_STAGES], acc_full;
   uint32_t tmem_base;
   int abort_flag;
+  float bias_part[T2_WORKERS];     // per loader thread: its feature's sum over the row groups it read
 };
 constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE + (int)sizeof(WgCtl) + 1024;
 
@@ -235,6 +238,8 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
   const int t = blockIdx.x - g.tile_begin, tiles_n = g.N / BN;
   const int m0 = (t / tiles_n) * T2_M, n0 = (t % tiles_n) * BN;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool with_bias = g.bias_off >= 0 && n0 == 0;
+  float bsum = 0.f;
   const int j_begin = blockIdx.y * rows_per_range;
   const int j_end = j_begin + rows_per_range < n_rows ? j_begin + rows_per_range : n_rows;
   const int nk = j_end > j_begin ? (j_end - j_begin + T2_K - 1) / T2_K : 0;
@@ -274,7 +279,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         const int task = tid + 256 * u;
-        fa[u] = load4(Am, lda, j0 + (task >> 7) * 4, m0 + (task & 127));
+        fa[u] = m0 + (task & 127) < g.M ? load4(Am, lda, j0 + (task >> 7) * 4, m0 + (task & 127)) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -304,6 +309,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
         const int task = tid + 256 * u, f = task & 127, kg = task >> 7;
         const size_t off = (size_t)((f >> 3) * 4 + kg) * 128 + (size_t)(f & 7) * 16;
         split_store(base + off, base + WG_A_PART + off, fa[u]);
+        bsum += (fa[u].x + fa[u].y) + (fa[u].z + fa[u].w);     // rows beyond the range were read as zeros
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -324,6 +330,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
       step(i, ra[0], rb[0]);
       if (ok && i + 1 < nk) step(i + 1, ra[1], rb[1]);
     }
+    ctl->bias_part[tid] = bsum;
   } else if (warp == T2_WORKERS / 32) {
     if (lane == 0) {
       const uint32_t idesc = make_idesc_tf32(BN);
@@ -377,6 +384,9 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
         }
       }
     }
+    // bias gradient: feature f was read by threads f (row groups 0 and 2 of every chunk) and f + 128 (groups 1 and 3)
+    if (with_bias && tid < T2_M && m0 + tid < g.M)
+      P[(size_t)blockIdx.y * count + g.bias_off + m0 + tid] = ctl->bias_part[tid] + ctl->bias_part[tid + T2_M];
   } else if (!good && tid == 0) {
     atomicExch(error, 3ull);
   }
@@ -434,9 +444,9 @@ cudaError_t launch_gemm_tc2(const TcGemmBatch& batch, int epi, unsigned long lon
   return cudaGetLastError();
 }
 
-bool tc_wgrad_ok(int M, int N, int rows) { return M % T2_M == 0 && N % 128 == 0 && rows >= 1024; }
+bool tc_wgrad_ok(int N, int rows) { return N % 128 == 0 && rows >= 1024; }
 
-int tc_wgrad_tiles(int M, int N) { return (M / T2_M) * (N / (N % T2_N == 0 ? T2_N : 128)); }
+int tc_wgrad_tiles(int M, int N) { return ((M + T2_M - 1) / T2_M) * (N / (N % T2_N == 0 ? T2_N : 128)); }
 
 cudaError_t launch_wgrad_tc(const TcWgradBatch& batch, float* P, int count, int n_rows, int rows_per_range, int n_ranges,
                             unsigned long long* error, cudaStream_t s) {
