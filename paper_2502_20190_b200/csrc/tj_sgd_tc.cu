@@ -118,21 +118,22 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
     }
   } else if (warp == T2_WORKERS / 32) {
     if (lane == 0) {
-      const uint32_t idesc = make_idesc_tf32(T2_N);
-      const uint32_t a0 = smem_addr(a_stages), b0 = smem_addr(b_slots);
+      // descriptors as 32-bit halves: the high word is a constant of the layout, the low word the address in 16-byte units
+      const uint32_t idesc = make_idesc_tf32(T2_N), hiword = desc_hi(T2_SBO);
+      const uint32_t a0 = desc_lo(smem_addr(a_stages), 128u), b0 = desc_lo(smem_addr(b_slots), 128u);
       for (int i = 0; i < nk; ++i) {
         const int st = i % T2_ASTAGES, sl = i % T2_BSLOTS;
         if (!tc_wait(&ctl->a_ready[st], (uint32_t)((i / T2_ASTAGES) & 1), abort_flag)) break;
         if (!tc_wait(&ctl->b_full[sl], (uint32_t)((i / T2_BSLOTS) & 1), abort_flag)) break;
         tc_fence_after();
-        const uint32_t a_hi = a0 + (uint32_t)st * T2_A_STAGE, a_lo = a_hi + T2_A_PART;
-        const uint32_t b_hi = b0 + (uint32_t)sl * T2_B_SLOT, b_lo = b_hi + T2_B_PART;
+        const uint32_t a_hi = a0 + (uint32_t)st * (T2_A_STAGE / 16), a_lo = a_hi + T2_A_PART / 16;
+        const uint32_t b_hi = b0 + (uint32_t)sl * (T2_B_SLOT / 16), b_lo = b_hi + T2_B_PART / 16;
 #pragma unroll
         for (int j = 0; j < T2_K / 8; ++j) {
-          const uint32_t o = (uint32_t)j * 256u;     // eight columns further: two core matrices
-          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, (i | j) != 0);
-          umma_tf32(tmem, make_desc(a_lo + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, true);
-          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_lo + o, 128u, T2_SBO), idesc, true);
+          const uint32_t o = (uint32_t)j * 16u;      // eight columns further: two core matrices = 256 bytes
+          umma_ss_tf32(tmem, a_hi + o, hiword, b_hi + o, hiword, idesc, (i | j) != 0);
+          umma_ss_tf32(tmem, a_lo + o, hiword, b_hi + o, hiword, idesc, 1u);
+          umma_ss_tf32(tmem, a_hi + o, hiword, b_lo + o, hiword, idesc, 1u);
         }
         umma_commit(&ctl->a_free[st]);
         umma_commit(&ctl->b_empty[sl]);
@@ -333,19 +334,20 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
     ctl->bias_part[tid] = bsum;
   } else if (warp == T2_WORKERS / 32) {
     if (lane == 0) {
-      const uint32_t idesc = make_idesc_tf32(BN);
-      const uint32_t s0 = smem_addr(stages);
+      const uint32_t idesc = make_idesc_tf32(BN), hiword = desc_hi(T2_SBO);
+      const uint32_t s0 = desc_lo(smem_addr(stages), 128u);
       for (int i = 0; i < nk; ++i) {
         const int st = i % WG_STAGES;
         if (!tc_wait(&ctl->ready[st], (uint32_t)((i / WG_STAGES) & 1), abort_flag)) break;
         tc_fence_after();
-        const uint32_t a_hi = s0 + (uint32_t)st * WG_STAGE, a_lo = a_hi + WG_A_PART, b_hi = a_hi + 2 * WG_A_PART, b_lo = b_hi + WG_B_PART;
+        const uint32_t a_hi = s0 + (uint32_t)st * (WG_STAGE / 16), a_lo = a_hi + WG_A_PART / 16, b_hi = a_hi + 2 * (WG_A_PART / 16),
+                       b_lo = b_hi + WG_B_PART / 16;
 #pragma unroll
         for (int j = 0; j < T2_K / 8; ++j) {
-          const uint32_t o = (uint32_t)j * 256u;     // eight rows of the minibatch further: two core matrices
-          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, (i | j) != 0);
-          umma_tf32(tmem, make_desc(a_lo + o, 128u, T2_SBO), make_desc(b_hi + o, 128u, T2_SBO), idesc, true);
-          umma_tf32(tmem, make_desc(a_hi + o, 128u, T2_SBO), make_desc(b_lo + o, 128u, T2_SBO), idesc, true);
+          const uint32_t o = (uint32_t)j * 16u;      // eight rows of the minibatch further: two core matrices = 256 bytes
+          umma_ss_tf32(tmem, a_hi + o, hiword, b_hi + o, hiword, idesc, (i | j) != 0);
+          umma_ss_tf32(tmem, a_lo + o, hiword, b_hi + o, hiword, idesc, 1u);
+          umma_ss_tf32(tmem, a_hi + o, hiword, b_lo + o, hiword, idesc, 1u);
         }
         umma_commit(&ctl->free_[st]);
       }
