@@ -140,9 +140,14 @@ def aggregate_throughput(units_per_replica, world, max_ms):
 class Runner:
     """Drives one context through the workload's call pattern."""
 
-    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False, two_stream=False, tensor_fp32=False):
+    def __init__(self, name, torch, binding, device_index, n_envs=0, with_update=False, two_stream=False, tensor_fp32=None):
         self.torch, self.name = torch, name
         self.w = dict(synth.WORKLOADS[name])
+        if tensor_fp32 is None:
+            # default: the FP32 workloads whose hidden x hidden layer is a dense contraction (hidden >= 256: cfg3, cfg4) run it
+            # on the tensor cores at FP32 accuracy; --fp32-fma selects the bit-reproducible FMA kernel instead
+            tensor_fp32 = (self.w["weight_dtype"] == synth.W_FP32 and self.w["env_kind"] != synth.ENV_LINGAUSS
+                           and self.w["hidden"] in (256,))
         if tensor_fp32:
             # FP32 weights, the actor's hidden x hidden layer as split-operand tensor-core products (1e-5 of the FP32 path)
             if self.w["weight_dtype"] != synth.W_FP32 or self.w["env_kind"] == synth.ENV_LINGAUSS or self.w["hidden"] % 64:
@@ -303,7 +308,10 @@ def run_ours(args):
     binding.load_library()
     peaks = load_peaks()
     name = args.workload
-    r = Runner(name, torch, binding, local, args.envs, args.with_update, args.two_stream, args.tensor_fp32)
+    if args.tensor_fp32 and args.fp32_fma:
+        raise SystemExit("--tensor-fp32 and --fp32-fma exclude each other")
+    r = Runner(name, torch, binding, local, args.envs, args.with_update, args.two_stream,
+               True if args.tensor_fp32 else (False if args.fp32_fma else None))
     w = r.w
     N = w["n_envs"]
     R = args.patterns or PATTERNS_PER_STEP[name]
@@ -459,7 +467,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": "bf16" if w["weight_dtype"] == synth.W_BF16 else ("f32 (hidden layer: 3 x fp16 split products)" if w["weight_dtype"] == synth.W_FP32_TC else "f32"), "data": "synthetic",
         "config": {"workload": name, "n_envs": N, "patterns_per_step": R, "actor_steps_per_pattern": r.actor_steps,
                    "minibatch": w.get("minibatch"), "mlp": "%d-%d-%d-%d" % (w["obs_dim"], w["hidden"], w["hidden"], w["n_actions"]),
-                   "replicas": world, "learner_update": r.with_update, "two_stream": r.two_stream,
+                   "replicas": world, "learner_update": r.with_update, "two_stream": r.two_stream, "weight_mode": {0: "fp32 fma", 1: "bf16 tensor", 2: "fp32 weights, split-operand tensor"}[w["weight_dtype"]],
                    "l2": "flushed between steps (256 MiB write outside the per-step event pairs)" if need_flush
                    else "ring larger than L2"},
         "consumed_samples_per_s": consumed / (tot_ms * 1e-3),
@@ -680,6 +688,7 @@ def main():
     ap.add_argument("--with-update", action="store_true", help="FP32 replay workloads: the learner step also runs tj_sgd_step and publishes the parameters it trains")
     ap.add_argument("--two-stream", action="store_true", help="replay workloads: learner calls on a second CUDA stream, passes software-pipelined (learner on the previous block beside the actor's next one)")
     ap.add_argument("--tensor-fp32", action="store_true", help="FP32 CartPole / Acrobot workloads: weight mode TJ_W_FP32_TC (hidden x hidden layer on the tensor cores as split-operand products, 1e-5 of the FP32 path)")
+    ap.add_argument("--fp32-fma", action="store_true", help="FP32 workloads: weight mode TJ_W_FP32 (FMA kernel, one fixed rounding order) also where the tensor-core mode is the default (hidden 256)")
     ap.add_argument("--sweep", action="store_true", help="also report consumed samples/s for each staleness bound the workload names")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=16.0)

@@ -391,11 +391,12 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
 // columns first the high parts' chunk, then the low parts', each H rows x 32 columns in the K-major core-matrix layout:
 // element (n, k) sits at ((n / 8) * 4 + (k % 32) / 8) * 64 + (n % 8) * 8 + k % 8 inside its chunk.
 // scale_out[0] = the power of two the weights were multiplied by, scale_out[1] = 1 / (that x the activation scale).
-// One launch: every block finds the largest |entry| of the matrix itself (64 K floats from L2 at most), so no block waits
-// for another; block 0 records the scale.
-__global__ void __launch_bounds__(256) split_pack_kernel(const float* __restrict__ blob, int D, int H, float* __restrict__ scale_out,
-                                                         uint16_t* __restrict__ dst) {
-  __shared__ float wmax[8];
+// One launch of a few large blocks: every block finds the largest |entry| of the matrix itself (64 K floats from L2 at most,
+// 64 per thread), so no block waits for another; block 0 records the scale; then each block packs its share.
+constexpr int SPLIT_PACK_BLOCKS = 32, SPLIT_PACK_THREADS = 1024;
+__global__ void __launch_bounds__(SPLIT_PACK_THREADS) split_pack_kernel(const float* __restrict__ blob, int D, int H, float* __restrict__ scale_out,
+                                                                        uint16_t* __restrict__ dst) {
+  __shared__ float wmax[32];
   const float* W2 = blob + (size_t)H * D + H;
   float m = 0.f;
   for (int i = threadIdx.x; i < H * H; i += blockDim.x) m = fmaxf(m, fabsf(W2[i]));   // the caller's pointer may be only 4-byte aligned
@@ -412,18 +413,18 @@ __global__ void __launch_bounds__(256) split_pack_kernel(const float* __restrict
     scale_out[0] = sc;
     scale_out[1] = 1.0f / (sc * SA_H_SCALE);
   }
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= H * H) return;
   const int chunk_elems = H * SA_KC;
-  const int kc = i / chunk_elems, within = i % chunk_elems;
-  const int core = within / 64, in_core = within % 64;
-  const int rg = core / (SA_KC / 8), kg = core % (SA_KC / 8);
-  const int n = rg * 8 + in_core / 8, k = kc * SA_KC + kg * 8 + in_core % 8;
-  const float v = W2[(size_t)n * H + k] * sc;
-  const __half hi = __float2half_rn(v);
-  const __half lo = __float2half_rn(v - __half2float(hi));
-  dst[(size_t)(2 * kc) * chunk_elems + within] = __half_as_ushort(hi);
-  dst[(size_t)(2 * kc + 1) * chunk_elems + within] = __half_as_ushort(lo);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < H * H; i += gridDim.x * blockDim.x) {
+    const int kc = i / chunk_elems, within = i % chunk_elems;
+    const int core = within / 64, in_core = within % 64;
+    const int rg = core / (SA_KC / 8), kg = core % (SA_KC / 8);
+    const int n = rg * 8 + in_core / 8, k = kc * SA_KC + kg * 8 + in_core % 8;
+    const float v = W2[(size_t)n * H + k] * sc;
+    const __half hi = __float2half_rn(v);
+    const __half lo = __float2half_rn(v - __half2float(hi));
+    dst[(size_t)(2 * kc) * chunk_elems + within] = __half_as_ushort(hi);
+    dst[(size_t)(2 * kc + 1) * chunk_elems + within] = __half_as_ushort(lo);
+  }
 }
 
 template <int ENV, int H>
@@ -455,7 +456,7 @@ bool split_actor_supported(int env_kind, int D, int H, int Aout) {
 size_t split_weight_halfs(int H) { return (size_t)2 * H * H; }
 
 cudaError_t launch_pack_split_weights(const float* blob, int D, int H, uint16_t* dst, float* scale, cudaStream_t s) {
-  split_pack_kernel<<<(H * H + 255) / 256, 256, 0, s>>>(blob, D, H, scale, dst);
+  split_pack_kernel<<<SPLIT_PACK_BLOCKS, SPLIT_PACK_THREADS, 0, s>>>(blob, D, H, scale, dst);
   return cudaGetLastError();
 }
 

@@ -36,9 +36,10 @@ def test_config_struct_matches_and_workspace_sizes(lib):
         if C_:
             assert nbytes >= C_ * (2 * D + 4) * 4
             # beside the ring and the env state: the learner update's scratch (four activation / delta arrays of
-            # minibatch x hidden, 32 partial gradients of the parameter blob, W2 transposed) and 64 MiB for the rest
+            # minibatch x hidden, 32 partial gradients of the parameter blob, W2 transposed, the split copies of W1 (two
+            # networks), W2 (two) and W2^T for the tensor-core products) and 64 MiB for the rest
             B, H = w["minibatch"], w["hidden"]
-            update = (4 * B * H + 32 * (H * (D + H + 19) + 17) + H * H + 24 * B) * 4
+            update = (4 * B * H + 32 * (H * (D + H + 19) + 17) + H * H + 24 * B + 2 * (2 * H * D + 3 * H * H)) * 4
             assert nbytes < C_ * (2 * D + 4) * 4 + N * max(D, 4) * 4 + update + 64 * 2**20
     # the largest workload's ring is 16M records of 1040 bytes
     assert nbytes > 17.4e9
