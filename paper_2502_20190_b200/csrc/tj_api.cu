@@ -136,6 +136,8 @@ size_t carve(tj_ctx* x, void* base) {
       x->wsplit[i] = cv.take<uint16_t>(split_weight_halfs(c.hidden));
       x->wsplit_scale[i] = cv.take<float>(2);
     }
+    x->wsplit_target = cv.take<uint16_t>(split_weight_halfs(c.hidden));
+    x->wsplit_scale_target = cv.take<float>(2);
   }
   x->use_tc = c.weight_dtype == TJ_W_BF16 && tc_mlp_supported(D, c.hidden, c.n_actions + vh);
   if (x->use_tc) {
@@ -426,6 +428,14 @@ int tj_publish_weights(tj_ctx* x, const void* blob, size_t nbytes, int32_t on_de
   if (!x->has_target || (x->cfg.target_sync_interval > 0 && x->k - x->k_last_sync >= x->cfg.target_sync_interval)) {
     if ((e = cudaMemcpyAsync(x->wtarget, dst, x->wl.total * sizeof(float), cudaMemcpyDeviceToDevice, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: target refresh");
+    if (x->use_split) {
+      const int slot = x->active;
+      if ((e = cudaMemcpyAsync(x->wsplit_target, x->wsplit[slot], split_weight_halfs(x->H) * sizeof(uint16_t), cudaMemcpyDeviceToDevice,
+                               x->lstream)) != cudaSuccess ||
+          (e = cudaMemcpyAsync(x->wsplit_scale_target, x->wsplit_scale[slot], 2 * sizeof(float), cudaMemcpyDeviceToDevice, x->lstream)) !=
+              cudaSuccess)
+        return cuda_fail(x, e, "publish: target refresh (split matrix)");
+    }
     if (x->use_tc && (e = cudaMemcpyAsync(x->wtc_target, dst_tc, tc_weight_elems(x->D, x->H) * sizeof(uint16_t),
                                           cudaMemcpyDeviceToDevice, x->lstream)) != cudaSuccess)
       return cuda_fail(x, e, "publish: target refresh (tensor-core weights)");
@@ -644,6 +654,15 @@ int tj_td_error(tj_ctx* x, const tj_batch* b, float* td_out, float* huber_out, f
       if ((e = launch_td_finish(x->td_partial, td_grid(b->n), b->n, loss_mean_out, x->lstream)) != cudaSuccess)
         return cuda_fail(x, e, "TD error (loss reduction)");
     }
+    learner_launched(x);
+    return TJ_OK;
+  }
+  if (x->use_split && x->cfg.replay_capacity > 0 && x->A <= 4) {
+    // weight mode TJ_W_FP32_TC: both forwards with the hidden x hidden layer on the tensor cores, like the actor's
+    LaunchScope scope(x, TJ_K_TD, loss_mean_out ? 2 : 1, true, true);
+    e = launch_td_split(p, x->wsplit[x->active], x->wsplit_scale[x->active], x->wsplit_target, x->wsplit_scale_target, x->lstream);
+    if (e == cudaSuccess && loss_mean_out) e = launch_td_finish(x->td_partial, td_split_grid(b->n), b->n, loss_mean_out, x->lstream);
+    if (e != cudaSuccess) return cuda_fail(x, e, "TD error (split-operand tensor-core forward)");
     learner_launched(x);
     return TJ_OK;
   }

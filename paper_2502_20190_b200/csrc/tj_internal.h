@@ -274,6 +274,9 @@ size_t split_weight_halfs(int H);
 cudaError_t launch_pack_split_weights(const float* blob, int D, int H, uint16_t* dst, float* scale, cudaStream_t s);
 cudaError_t launch_actor_split(int env_kind, const ActorParams& p, const uint16_t* w2parts, const float* w2scale, int sm_count,
                                cudaStream_t s);
+int td_split_grid(int n);   // loss partials (one per 128 rows) of launch_td_split
+cudaError_t launch_td_split(const TdParams& p, const uint16_t* parts_online, const float* scale_online, const uint16_t* parts_target,
+                            const float* scale_target, cudaStream_t s);
 size_t fma_rate_sink_floats(int sm_count);
 double launch_fma_rate(float* sink, int sm_count, int outer, cudaStream_t s, cudaError_t* err);
 cudaError_t launch_transpose_pad(const float* src, float* dst, int rows, int cols, int ld_dst, cudaStream_t s);
@@ -322,6 +325,8 @@ struct tj_ctx {
   bool use_split;
   uint16_t* wsplit[2];
   float* wsplit_scale[2];
+  uint16_t* wsplit_target;     // the target network's split matrix (refreshed with the target parameters)
+  float* wsplit_scale_target;
   // tensor-core path (BF16 weights, supported shapes only)
   bool use_tc;
   int sm_count;

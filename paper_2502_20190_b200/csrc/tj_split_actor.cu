@@ -94,10 +94,11 @@ __device__ __forceinline__ void sa_layer1_block(const MlpWeights& mw, int Hp, co
 }
 
 // Network outputs of the observations in xs -> out[i][e], i < Aout.  Called by every thread of the block; `pass` counts the
-// calls, `copied` is the copy lane's position in the chunk stream.  Returns false after a timeout.
+// calls, `copied` is the copy lane's position in the chunk stream: pass q reads the split matrix parts[q & 1] (the actor
+// passes the same matrix twice, the TD kernel the online and the target network's).  Returns false after a timeout.
 template <int D, int H>
-__device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeights& mw, const SaShared& sh, const uint16_t* w2parts,
-                                           float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied,
+__device__ __forceinline__ bool sa_forward(int Hp, int Aout, const MlpWeights& mw, const SaShared& sh, const uint16_t* parts0,
+                                           const uint16_t* parts1, float inv_scale, uint32_t tmem, uint32_t pass, uint32_t& copied,
                                            volatile int* abort_flag) {
   constexpr int NKC = H / SA_KC;                 // K chunks of the hidden x hidden layer
   constexpr uint32_t NSTREAM = 2 * NKC;          // chunks of W2 per pass: (high, low) per K chunk
@@ -116,7 +117,7 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
       for (int b = 0; b < 2; ++b) {
         const int n0 = kc * SA_KC + half * 16 + b * 8;
         const size_t off = ((size_t)(e >> 3) * (H / 8) + (n0 >> 3)) * 128 + (e & 7) * 16;
-        sa_layer1_block<D>(mw, p.Hp, x, n0, sh.a_hi, sh.a_lo, off);
+        sa_layer1_block<D>(mw, Hp, x, n0, sh.a_hi, sh.a_lo, off);
       }
       fence_async_smem();
       mbar_arrive_warp(&ctl->a_ready[kc]);
@@ -164,7 +165,8 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
         const uint32_t sp = copied % SA_SLOTS;
         if (!tc_wait(&ctl->empty[sp], ((copied / SA_SLOTS) - 1) & 1, abort_flag)) break;
         mbar_expect_tx(&ctl->full[sp], CHUNK_BYTES);
-        bulk_copy_g2s(sh.ring + (size_t)sp * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(w2parts) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
+        const uint16_t* src = ((copied / NSTREAM) & 1u) ? parts1 : parts0;
+        bulk_copy_g2s(sh.ring + (size_t)sp * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(src) + (size_t)(copied % NSTREAM) * CHUNK_BYTES,
                       CHUNK_BYTES, &ctl->full[sp]);
       }
     }
@@ -193,11 +195,11 @@ __device__ __forceinline__ bool sa_forward(const ActorParams& p, const MlpWeight
     }
 #pragma unroll
     for (int a = 0; a < 4; ++a)
-      if (a < p.Aout) sh.part[((size_t)half * 4 + a) * SA_TE + r] = pa[a];
+      if (a < Aout) sh.part[((size_t)half * 4 + a) * SA_TE + r] = pa[a];
   }
   __syncthreads();
   if (tid < SA_TE)
-    for (int a = 0; a < p.Aout; ++a)
+    for (int a = 0; a < Aout; ++a)
       sh.out[a * SA_TE + tid] = (mw.b3[a] + sh.part[(size_t)a * SA_TE + tid]) + sh.part[((size_t)4 + a) * SA_TE + tid];
   __syncthreads();
   return *abort_flag == 0;
@@ -279,7 +281,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
         for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? obs[k] : 0.f;
       }
       __syncthreads();
-      ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
+      ok = sa_forward<D, H>(p.Hp, p.Aout, mw, sh, w2parts, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
       ok = __syncthreads_and(ok);
       if (!ok) break;
       if (owner) {
@@ -352,7 +354,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
           for (int k = 0; k < D; ++k) sh.xs[k * SA_TE + tid] = owner ? o2[k] : 0.f;
         }
         __syncthreads();
-        ok = sa_forward<D, H>(p, mw, sh, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
+        ok = sa_forward<D, H>(p.Hp, p.Aout, mw, sh, w2parts, w2parts, inv_scale, tmem, pass++, copied, abort_flag);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         if (owner) {
@@ -377,6 +379,133 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
     for (uint32_t g = pass * NSTREAM; g < copied; ++g)
       if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
     if (ctl->abort_flag) atomicExch(&p.stats->error, 4ull);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  }
+}
+
+// TD error (Algorithm 1, TD-error line; Huber loss on it) for a context in this weight mode: a tile of 128 sampled rows per
+// block, the online network on obs (pass 0), the target network on next_obs (pass 1), both with the split-operand hidden
+// layer above; the small parameters are staged twice, the chunk stream alternates between the two split matrices.
+// Outputs and the per-block loss partial as in the FP32 TD kernel (one partial per 128 rows, summed in row order).
+template <int D, int H>
+__global__ void __launch_bounds__(SA_NT, 1) td_split_tc_kernel(const TdParams p, const uint16_t* __restrict__ parts_online,
+                                                              const float* __restrict__ scale_online,
+                                                              const uint16_t* __restrict__ parts_target,
+                                                              const float* __restrict__ scale_target) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  constexpr int A_BYTES = SA_TE * H * 2;
+  constexpr uint32_t CHUNK_BYTES = H * SA_KC * 2;
+  constexpr uint32_t NSTREAM = 2 * (H / SA_KC);
+  SaShared sh;
+  sh.a_hi = smem_raw;
+  sh.a_lo = sh.a_hi + A_BYTES;
+  sh.ring = sh.a_lo + A_BYTES;
+  float* wsm = reinterpret_cast<float*>(sh.ring + SA_SLOTS * CHUNK_BYTES);
+  const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);
+  sh.xs = wsm + staged;
+  sh.out = sh.xs + (size_t)8 * SA_TE;
+  sh.part = sh.out + (size_t)4 * SA_TE;
+  sh.ctl = reinterpret_cast<SaCtl*>(sh.part + 2 * (size_t)4 * SA_TE);
+  SaCtl* ctl = sh.ctl;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int j0 = blockIdx.x * SA_TE, n_here = min(SA_TE, p.n - j0);
+  if (tid == 0) {
+    for (int s = 0; s < SA_SLOTS; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+    for (int k = 0; k < SA_MAX_KC; ++k) mbar_init(&ctl->a_ready[k], SA_WORKERS / 32);
+    mbar_init(&ctl->wbar, 1);
+    mbar_init(&ctl->acc_full, 1);
+    ctl->abort_flag = 0;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&ctl->tmem_base)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  MlpWeights mw = stage_mlp_weights<1>(p, p.Wonline, wsm, &ctl->wbar, tid == 0);
+  for (int i = tid; i < SA_TE * D; i += SA_NT) {
+    const int el = i / D, k = i % D;
+    sh.xs[k * SA_TE + el] = el < n_here ? p.obs[(size_t)(j0 + el) * D + k] : 0.f;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort_flag;
+  bool ok = tc_wait_elect(&ctl->wbar, 0, abort_flag);
+  ok = __syncthreads_and(ok);
+  uint32_t copied = 0;
+  if (tid == SA_WORKERS + 32 && ok) {
+    for (; copied < SA_SLOTS; ++copied) {
+      mbar_expect_tx(&ctl->full[copied], CHUNK_BYTES);
+      bulk_copy_g2s(sh.ring + (size_t)copied * CHUNK_BYTES, reinterpret_cast<const uint8_t*>(parts_online) + (size_t)copied * CHUNK_BYTES,
+                    CHUNK_BYTES, &ctl->full[copied]);
+    }
+  }
+  uint32_t passes = 0;
+  float qsel = 0.f;
+  if (ok) {
+    ok = sa_forward<D, H>(p.Hp, p.A, mw, sh, parts_online, parts_target, scale_online[1], tmem, 0u, copied, abort_flag);
+    passes = 1;
+    ok = __syncthreads_and(ok);
+  }
+  if (ok) {
+    if (tid < n_here) {
+      int a = p.act[j0 + tid];
+      a = a < 0 ? 0 : (a >= p.A ? p.A - 1 : a);
+      qsel = sh.out[a * SA_TE + tid];
+    }
+    __syncthreads();   // every thread is done with the online parameters and outputs: the staging buffer may be refilled
+    mw = stage_mlp_weights<1>(p, p.Wtarget, wsm, &ctl->wbar, tid == 0);
+    for (int i = tid; i < SA_TE * D; i += SA_NT) {
+      const int el = i / D, k = i % D;
+      sh.xs[k * SA_TE + el] = el < n_here ? p.next_obs[(size_t)(j0 + el) * D + k] : 0.f;
+    }
+    ok = tc_wait_elect(&ctl->wbar, 1, abort_flag);
+    ok = __syncthreads_and(ok);
+  }
+  if (ok) {
+    ok = sa_forward<D, H>(p.Hp, p.A, mw, sh, parts_online, parts_target, scale_target[1], tmem, 1u, copied, abort_flag);
+    passes = 2;
+    ok = __syncthreads_and(ok);
+  }
+  const float nan = __int_as_float(0x7FC00000);
+  float* hub = sh.part;                       // free again after the pass
+  if (tid < SA_TE) {
+    float h = 0.f;
+    if (tid < n_here) {
+      const int j = j0 + tid;
+      float delta = nan;
+      h = nan;
+      if (ok) {
+        float qmax = sh.out[tid];
+        for (int i = 1; i < p.A; ++i) qmax = fmaxf(qmax, sh.out[i * SA_TE + tid]);
+        const float y = p.rew[j] + p.gamma * (p.done[j] ? 0.f : 1.f) * qmax;
+        delta = y - qsel;
+        const float ad = fabsf(delta);
+        h = ad <= p.kappa ? 0.5f * delta * delta : p.kappa * (ad - 0.5f * p.kappa);
+      }
+      if (p.td_out) p.td_out[j] = delta;        // after a timeout: defined outputs (NaN), never what an earlier call left
+      if (p.huber_out) p.huber_out[j] = h;
+    }
+    hub[tid] = h;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float sum = 0.f;
+    for (int i = 0; i < n_here; ++i) sum += hub[i];
+    p.partial[blockIdx.x] = sum;
+    if (ctl->abort_flag && p.error) atomicExch(p.error, 4ull);
+  }
+  // the copies still in flight must land before the block gives its shared memory back
+  if (tid == SA_WORKERS + 32) {
+    for (uint32_t g = passes * NSTREAM; g < copied; ++g)
+      if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
   }
   tc_fence_before();
   __syncthreads();
@@ -472,6 +601,41 @@ cudaError_t launch_actor_split(int env_kind, const ActorParams& p, const uint16_
   const int grid = n_tiles < sm_count ? n_tiles : sm_count;
   return env_kind == TJ_ENV_CARTPOLE ? launch_split_env<TJ_ENV_CARTPOLE>(p, w2parts, w2scale, grid, smem, s)
                                      : launch_split_env<TJ_ENV_ACROBOT>(p, w2parts, w2scale, grid, smem, s);
+}
+
+template <int D>
+static cudaError_t launch_td_split_d(const TdParams& p, const uint16_t* po, const float* so, const uint16_t* pt, const float* st, int grid,
+                                     size_t smem, cudaStream_t s) {
+#define TJ_TD_SPLIT_CASE(HH)                                                                                                      \
+  case HH: {                                                                                                                      \
+    cudaError_t e = cudaFuncSetAttribute(td_split_tc_kernel<D, HH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
+    if (e != cudaSuccess) return e;                                                                                               \
+    td_split_tc_kernel<D, HH><<<grid, SA_NT, smem, s>>>(p, po, so, pt, st);                                                        \
+    return cudaGetLastError();                                                                                                    \
+  }
+  switch (p.H) {
+    TJ_TD_SPLIT_CASE(64)
+    TJ_TD_SPLIT_CASE(128)
+    TJ_TD_SPLIT_CASE(192)
+    TJ_TD_SPLIT_CASE(256)
+    default: return cudaErrorInvalidConfiguration;
+  }
+#undef TJ_TD_SPLIT_CASE
+}
+
+int td_split_grid(int n) { return (n + SA_TE - 1) / SA_TE; }
+
+cudaError_t launch_td_split(const TdParams& p, const uint16_t* parts_online, const float* scale_online, const uint16_t* parts_target,
+                            const float* scale_target, cudaStream_t s) {
+  if (p.n <= 0) return cudaSuccess;
+  if (!(p.D == 4 || p.D == 6) || p.A > 4 || p.Ap != 4) return cudaErrorInvalidConfiguration;
+  const size_t staged = p.w_total - (p.off_b2 - p.off_W2t);
+  const size_t smem = (size_t)2 * SA_TE * p.H * 2 + (size_t)SA_SLOTS * p.H * SA_KC * 2 +
+                      (staged + (size_t)(8 + 4 + 8) * SA_TE) * sizeof(float) + sizeof(SaCtl) + 64;
+  if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;
+  const int grid = td_split_grid(p.n);
+  return p.D == 4 ? launch_td_split_d<4>(p, parts_online, scale_online, parts_target, scale_target, grid, smem, s)
+                  : launch_td_split_d<6>(p, parts_online, scale_online, parts_target, scale_target, grid, smem, s);
 }
 
 }  // namespace tj

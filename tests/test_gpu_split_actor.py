@@ -160,3 +160,49 @@ def test_unsupported_shapes_are_refused(env):
         with pytest.raises(Exception) as ei:
             binding.Context(**dict(f, weight_dtype=W_FP32_TC))
         assert "TJ_W_FP32_TC" in str(ei.value)
+
+
+@pytest.mark.parametrize("kind,D,A,H,B", [(0, 4, 2, 64, 256), (1, 6, 3, 256, 77), (1, 6, 3, 128, 300), (0, 4, 2, 256, 1)])
+def test_td_error_in_this_weight_mode_follows_the_lagging_target(env, kind, D, A, H, B):
+    """tj_td_error of a context in this weight mode runs both forwards with the split-operand hidden layer; the oracle's FP32
+    TD error is the reference at the FP32 tolerance (relative to the terms the error is a difference of).  The target network
+    lags one version at versions 2 and 4: there the GPU's errors must follow the lagging target, not the newest parameters."""
+    torch, orc, binding = env
+    f = _ring_fields(kind, D, A, H, 32, replay_capacity=32 * 16, minibatch=B, warmup=32, staleness_bound=50,
+                     target_sync_interval=2, max_episode_steps=11)
+    ctx, o = _pair(orc, binding, **f)
+    fresh = orc.Oracle(**dict(f, target_sync_interval=1, weight_dtype=W_FP32))
+    tally = Tally()
+    for v in range(1, 6):
+        blob = blob_for(f, v)
+        ctx.publish_weights(blob)
+        o.publish(blob)
+        fresh.publish(blob)
+        for _ in range(4):
+            lockstep_step(ctx, o, torch, rtol=RTOL_FP32, env_kind=kind, tally=tally, logits_exact=False)
+        _, batch = ctx.replay_sample()
+        o.sample()
+        fresh.set_counters(0, 0, v)
+        out = ctx.td_error(batch)
+        rec = np.zeros((B, 2 * D + 4), np.float32)
+        rec[:, :D] = batch["obs"].cpu().numpy()
+        rec[:, D:2 * D] = batch["next_obs"].cpu().numpy()
+        rec.view(np.int32)[:, 2 * D] = batch["act"].cpu().numpy()
+        rec[:, 2 * D + 1] = batch["rew"].cpu().numpy()
+        rec.view(np.int32)[:, 2 * D + 2] = batch["done"].cpu().numpy()
+        st, td, hub, loss, qs, qn = o.td(rec)
+        assert st == 0
+        rms = float(np.sqrt(np.mean(qs ** 2) + np.mean(qn ** 2)))
+        terms = np.abs(qs) + np.abs(qn) + np.abs(rec[:, 2 * D + 1]) + rms
+        g_td = out["td"].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(g_td - td) <= RTOL_FP32 * (np.abs(td) + terms)), float(np.max(np.abs(g_td - td) / (np.abs(td) + terms)))
+        g_h = out["huber"].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(g_h - hub) <= 2 * RTOL_FP32 * (hub + terms * np.maximum(1.0, np.abs(td))))
+        assert abs(float(out["loss"].item()) - loss) <= 2 * RTOL_FP32 * (abs(loss) + float(terms.mean()))
+        if v in (2, 4) and B > 1:
+            _, td_fresh, _, _, _, _ = fresh.td(rec)
+            moved = np.abs(td_fresh - td) > 100 * RTOL_FP32 * (np.abs(td) + terms)
+            live = rec.view(np.int32)[:, 2 * D + 2] == 0
+            assert moved[live].mean() > 0.9
+            assert np.all(np.abs(g_td - td_fresh)[moved] > RTOL_FP32 * (np.abs(td) + terms)[moved])
+    assert ctx.stats()["device_error"] == 0
