@@ -24,7 +24,9 @@ namespace {
 
 constexpr int T2_M = 128, T2_N = 256, T2_K = 16;
 constexpr int T2_WORKERS = 256, T2_THREADS = T2_WORKERS + 64, T2_PF = 3;
-constexpr int T2_ASTAGES = 4, T2_BSLOTS = 4;
+constexpr int T2_ASTAGES = 4, T2_BSLOTS = 3;
+constexpr int T2_STG_LD = 36;                              // floats per row of a warp's 32 x 32 staging block (144 bytes)
+constexpr int T2_STG_BYTES = (T2_WORKERS / 32) * 32 * T2_STG_LD * 4;   // 36 KB: one block per worker warp
 constexpr int T2_A_PART = T2_M * T2_K * 4;                 // 8 KB: one part of an A stage
 constexpr int T2_A_STAGE = 2 * T2_A_PART;
 constexpr int T2_B_PART = T2_N * T2_K * 4;                 // 16 KB: one part of a B chunk
@@ -36,13 +38,29 @@ struct T2Ctl {
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr int T2_SMEM_BYTES = T2_ASTAGES * T2_A_STAGE + T2_BSLOTS * T2_B_SLOT + (int)sizeof(T2Ctl) + 1024;
+constexpr int T2_SMEM_BYTES = T2_ASTAGES * T2_A_STAGE + T2_BSLOTS * T2_B_SLOT + T2_STG_BYTES + (int)sizeof(T2Ctl) + 1024;
+
+// A thread owns a row of the accumulator, and a row written straight to global memory costs one 16-byte sector per lane and
+// store instruction (8,192 separate sectors per 128 x 256 tile: about 24 K cycles).  So every warp passes its 32 rows x 32
+// columns through a staging block of its own: lane r writes row r, then lane l reads the 16-byte piece l % 8 of rows
+// l / 8 + 4 i, so that one store instruction writes four rows of 128 contiguous bytes.  Only warp-level synchronisation.
+__device__ __forceinline__ void stage_rows(float* stg, int lane, const uint32_t (&v)[32]) {
+  __syncwarp();                                   // the block's previous readers are done
+  float* row = stg + lane * T2_STG_LD;
+#pragma unroll
+  for (int c4 = 0; c4 < 8; ++c4) *reinterpret_cast<uint4*>(row + c4 * 4) = make_uint4(v[c4 * 4], v[c4 * 4 + 1], v[c4 * 4 + 2], v[c4 * 4 + 3]);
+  __syncwarp();
+}
+__device__ __forceinline__ float4 staged_piece(const float* stg, int lane, int i) {
+  return *reinterpret_cast<const float4*>(stg + ((lane >> 3) + 4 * i) * T2_STG_LD + (lane & 7) * 4);
+}
 
 __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemmBatch batch, int epi, unsigned long long* __restrict__ error) {
   extern __shared__ uint8_t t2_raw[];
   uint8_t* a_stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(t2_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* b_slots = a_stages + T2_ASTAGES * T2_A_STAGE;
-  T2Ctl* ctl = reinterpret_cast<T2Ctl*>(b_slots + T2_BSLOTS * T2_B_SLOT);
+  float* stg_all = reinterpret_cast<float*>(b_slots + T2_BSLOTS * T2_B_SLOT);
+  T2Ctl* ctl = reinterpret_cast<T2Ctl*>(b_slots + T2_BSLOTS * T2_B_SLOT + T2_STG_BYTES);
   const TcGemm& g = batch.g[blockIdx.z];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m0 = blockIdx.y * T2_M, n0 = blockIdx.x * T2_N;
@@ -167,32 +185,33 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
   if (good && tid < T2_WORKERS) {
     tc_fence_after();
     const int q = warp & 3, half = warp >> 2;      // TMEM lane quarter of this warp, column half
-    const int m = m0 + q * 32 + lane;
     const uint32_t t_acc = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * (T2_N / 2));
     float* __restrict__ C = g.C;
     const float* __restrict__ bias = g.bias;
     const float* __restrict__ mask = g.mask;
+    float* stg = stg_all + warp * (32 * T2_STG_LD);
 #pragma unroll 1
     for (int c0 = 0; c0 < T2_N / 2; c0 += 32) {
       uint32_t v[32];
       tmem_ld16(t_acc + (uint32_t)c0, v);
       tmem_ld16(t_acc + (uint32_t)c0 + 16u, v + 16);
       tmem_ld_wait();
-      if (m < M) {
-        const int n = n0 + half * (T2_N / 2) + c0;
-        float* dst = C + (size_t)m * g.ldc + n;
+      stage_rows(stg, lane, v);
+      const int n = n0 + half * (T2_N / 2) + c0 + (lane & 7) * 4;
+      float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (epi == GM_BIAS_RELU) bv = __ldg(reinterpret_cast<const float4*>(bias + n));
 #pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
-          float4 o = make_float4(__uint_as_float(v[c4 * 4]), __uint_as_float(v[c4 * 4 + 1]), __uint_as_float(v[c4 * 4 + 2]),
-                                 __uint_as_float(v[c4 * 4 + 3]));
+      for (int i = 0; i < 8; ++i) {
+        const int m = m0 + q * 32 + (lane >> 3) + 4 * i;
+        float4 o = staged_piece(stg, lane, i);
+        if (m < M) {
           if (epi == GM_BIAS_RELU) {
-            const float4 b = __ldg(reinterpret_cast<const float4*>(bias + n + c4 * 4));
-            o.x = fmaxf(o.x + b.x, 0.f); o.y = fmaxf(o.y + b.y, 0.f); o.z = fmaxf(o.z + b.z, 0.f); o.w = fmaxf(o.w + b.w, 0.f);
+            o.x = fmaxf(o.x + bv.x, 0.f); o.y = fmaxf(o.y + bv.y, 0.f); o.z = fmaxf(o.z + bv.z, 0.f); o.w = fmaxf(o.w + bv.w, 0.f);
           } else {
-            const float4 k = __ldg(reinterpret_cast<const float4*>(mask + (size_t)m * g.ldm + n + c4 * 4));
+            const float4 k = __ldg(reinterpret_cast<const float4*>(mask + (size_t)m * g.ldm + n));
             o.x = k.x > 0.f ? o.x : 0.f; o.y = k.y > 0.f ? o.y : 0.f; o.z = k.z > 0.f ? o.z : 0.f; o.w = k.w > 0.f ? o.w : 0.f;
           }
-          *reinterpret_cast<float4*>(dst + c4 * 4) = o;
+          *reinterpret_cast<float4*>(C + (size_t)m * g.ldc + n) = o;
         }
       }
     }
@@ -216,7 +235,7 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_gemm_tc2_kernel(const TcGemm
 // parameter blob, and the apply kernel adds the ranges in order (no atomics, one fixed order).  A product with fewer than 128
 // gradient columns (the head: one column per action) reads zeros beyond them.  The first column tile of a product also
 // writes the bias gradient, the column sums of G over the range: its loaders hold those values anyway.
-constexpr int WG_STAGES = 4;
+constexpr int WG_STAGES = 3;
 constexpr int WG_A_PART = T2_M * T2_K * 4, WG_B_PART = T2_N * T2_K * 4;          // 8 KB, 16 KB
 constexpr int WG_STAGE = 2 * WG_A_PART + 2 * WG_B_PART;                          // A_hi | A_lo | B_hi | B_lo: 48 KB
 struct WgCtl {
@@ -225,13 +244,14 @@ struct WgCtl {
   int abort_flag;
   float bias_part[T2_WORKERS];     // per loader thread: its feature's sum over the row groups it read
 };
-constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE + (int)sizeof(WgCtl) + 1024;
+constexpr int WG_SMEM_BYTES = WG_STAGES * WG_STAGE + T2_STG_BYTES + (int)sizeof(WgCtl) + 1024;
 
 __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgradBatch batch, float* __restrict__ P, int count, int n_rows,
                                                                     int rows_per_range, unsigned long long* __restrict__ error) {
   extern __shared__ uint8_t wg_raw[];
   uint8_t* stages = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(wg_raw) + 1023) & ~(uintptr_t)1023);
-  WgCtl* ctl = reinterpret_cast<WgCtl*>(stages + WG_STAGES * WG_STAGE);
+  float* stg_all = reinterpret_cast<float*>(stages + WG_STAGES * WG_STAGE);
+  WgCtl* ctl = reinterpret_cast<WgCtl*>(stages + WG_STAGES * WG_STAGE + T2_STG_BYTES);
   int q = 0;
   while (q + 1 < batch.n && (int)blockIdx.x >= batch.g[q + 1].tile_begin) ++q;
   const TcWgrad& g = batch.g[q];
@@ -362,10 +382,10 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
   if (good && tid < T2_WORKERS) {
     tc_fence_after();
     const int q4 = warp & 3, half = warp >> 2;      // TMEM lane quarter of this warp, column half
-    const int m = m0 + q4 * 32 + lane;
     const int cols = BN / 2;
     const uint32_t t_acc = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(half * cols);
-    float* dst_row = P + (size_t)blockIdx.y * count + g.off + (size_t)m * g.N + n0 + half * cols;
+    float* stg = stg_all + warp * (32 * T2_STG_LD);
+    float* dst = P + (size_t)blockIdx.y * count + g.off;
 #pragma unroll 1
     for (int c0 = 0; c0 < cols; c0 += 32) {
       uint32_t v[32];
@@ -377,12 +397,19 @@ __global__ void __launch_bounds__(T2_THREADS, 1) sg_wgrad_tc_kernel(const TcWgra
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = 0u;       // an empty range of rows contributes nothing
       }
-      if (m < g.M) {
+      stage_rows(stg, lane, v);
+      const int n = n0 + half * cols + c0 + (lane & 7) * 4;
 #pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4) {
-          float* d = dst_row + c0 + c4 * 4;           // the blob's matrices start at any multiple of four bytes: scalar stores
-          d[0] = __uint_as_float(v[c4 * 4]); d[1] = __uint_as_float(v[c4 * 4 + 1]);
-          d[2] = __uint_as_float(v[c4 * 4 + 2]); d[3] = __uint_as_float(v[c4 * 4 + 3]);
+      for (int i = 0; i < 8; ++i) {
+        const int m = m0 + q4 * 32 + (lane >> 3) + 4 * i;
+        const float4 o = staged_piece(stg, lane, i);
+        if (m < g.M) {
+          float* d = dst + (size_t)m * g.N + n;          // the blob's matrices start at any multiple of four bytes
+          if ((reinterpret_cast<uintptr_t>(d) & 15) == 0) {
+            *reinterpret_cast<float4*>(d) = o;
+          } else {
+            d[0] = o.x; d[1] = o.y; d[2] = o.z; d[3] = o.w;
+          }
         }
       }
     }
