@@ -269,6 +269,70 @@ __global__ void __launch_bounds__(GM_THREADS) sg_gemm_pair_kernel(const GemmPair
   sg_gemm_body<B_KN, EPI, BM>(pr.A[z], lda, pr.B[z], ldb, pr.C[z], ldc, M, N, K, pr.bias[z], nullptr, 0);
 }
 
+// The heads of both networks for wide hidden layers: out[row][a] = bias[a] + sum_k h[row][k] W[a][k], a < A <= 16, H a
+// multiple of 128.  A 32-row FMA tile pads the few outputs to 64 columns and pays a block barrier per 16 k; here a warp takes
+// a row at a time: lane l reads the 16-byte pieces l, l + 32, ... of the row (coalesced), multiplies them with the head's
+// weights (in shared memory, laid out so that consecutive lanes read consecutive 16-byte words) into 16 partial outputs, and
+// the 16 x 32 partials are summed by a fixed halving exchange (16 shuffles).  blockIdx.y picks the network.
+constexpr int HD_ROWS = 64;   // rows per block: eight per warp
+__global__ void __launch_bounds__(256) sg_heads_kernel(const GemmPair pr, int n_rows, int H, int A, int ldc) {
+  extern __shared__ __align__(16) float4 hd_w[];       // [(j * 4 + kk) * 4 + aq][lane]: W[aq * 4 .. + 3][4 (32 j + lane) + kk]
+  const int z = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* __restrict__ W = pr.B[z];
+  const float* __restrict__ hrows = pr.A[z];
+  const float* __restrict__ bias = pr.bias[z];
+  float* __restrict__ out = pr.C[z];
+  const int nj = H / 128;
+  for (int i = tid; i < nj * 16 * 32; i += blockDim.x) {
+    const int l = i & 31, aq = (i >> 5) & 3, kk = (i >> 7) & 3, j = i >> 9;
+    const int k = 4 * (32 * j + l) + kk, a = aq * 4;
+    float4 w;
+    w.x = a < A ? W[(size_t)a * H + k] : 0.f;
+    w.y = a + 1 < A ? W[(size_t)(a + 1) * H + k] : 0.f;
+    w.z = a + 2 < A ? W[(size_t)(a + 2) * H + k] : 0.f;
+    w.w = a + 3 < A ? W[(size_t)(a + 3) * H + k] : 0.f;
+    hd_w[i] = w;
+  }
+  __syncthreads();
+  const int a_mine = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+  const float b_mine = a_mine < A ? bias[a_mine] : 0.f;
+  for (int r = warp; r < HD_ROWS; r += 8) {
+    const int row = blockIdx.x * HD_ROWS + r;
+    if (row >= n_rows) break;
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+    for (int j = 0; j < nj; ++j) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(hrows + (size_t)row * H) + 32 * j + lane);
+      const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+        for (int aq = 0; aq < 4; ++aq) {
+          const float4 w = hd_w[((j * 4 + kk) * 4 + aq) * 32 + lane];
+          v[aq * 4] = fmaf(xs[kk], w.x, v[aq * 4]); v[aq * 4 + 1] = fmaf(xs[kk], w.y, v[aq * 4 + 1]);
+          v[aq * 4 + 2] = fmaf(xs[kk], w.z, v[aq * 4 + 2]); v[aq * 4 + 3] = fmaf(xs[kk], w.w, v[aq * 4 + 3]);
+        }
+    }
+    // halving exchange: after the step with distance d a lane keeps the half of its values that its bit d selects
+#define TJ_HD_STEP(D, CNT)                                                                     \
+    {                                                                                             \
+      const bool upper = (lane & (D)) != 0;                                                       \
+      _Pragma("unroll") for (int i = 0; i < (CNT); ++i) {                                         \
+        const float keep = upper ? v[i + (CNT)] : v[i], send = upper ? v[i] : v[i + (CNT)];      \
+        v[i] = keep + __shfl_xor_sync(0xffffffffu, send, (D));                                   \
+      }                                                                                           \
+    }
+    TJ_HD_STEP(16, 8)
+    TJ_HD_STEP(8, 4)
+    TJ_HD_STEP(4, 2)
+    TJ_HD_STEP(2, 1)
+#undef TJ_HD_STEP
+    const float total = v[0] + __shfl_xor_sync(0xffffffffu, v[0], 1);
+    if ((lane & 1) == 0 && a_mine < A) out[(size_t)row * ldc + a_mine] = total + b_mine;
+  }
+}
+
 template <bool B_KN, int EPI, int BM = GM_BM>
 void sg_gemm(const float* A, int lda, const float* B, int ldb, float* C, int ldc, int M, int N, int K, const float* bias,
              const float* mask, int ldm, cudaStream_t s) {
@@ -948,7 +1012,13 @@ cudaError_t launch_sgd_step(const SgdParams& p, float lr, const AdamParams* adam
       if ((e = launch_gemm_tc2(l2, GM_BIAS_RELU, p.error, s)) != cudaSuccess) return e;
       // both heads in one launch: Q of the online network into g, of the target network into dh1's place
       GemmPair heads{{p.h2, p.dh2}, {W3, T3}, {p.g, p.dh1}, {b3, tb3}};
-      sg_gemm_pair_kernel<false, GM_BIAS, 32><<<dim3((A + GM_BN - 1) / GM_BN, (n + 31) / 32, 2), GM_THREADS, 0, s>>>(heads, H, H, A, n, A, H);
+      const size_t hd_smem = (size_t)H * 16 * sizeof(float);
+      if (H % 128 == 0 && A <= 16 && hd_smem <= 96 * 1024) {
+        if ((e = cudaFuncSetAttribute(sg_heads_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hd_smem)) != cudaSuccess) return e;
+        sg_heads_kernel<<<dim3((n + HD_ROWS - 1) / HD_ROWS, 2), 256, hd_smem, s>>>(heads, n, H, A, A);
+      } else {
+        sg_gemm_pair_kernel<false, GM_BIAS, 32><<<dim3((A + GM_BN - 1) / GM_BN, (n + 31) / 32, 2), GM_THREADS, 0, s>>>(heads, H, H, A, n, A, H);
+      }
     } else {
       if ((e = sg_layer<GM_BIAS_RELU>(p.obs, D, W1, D, p.h1, H, n, H, D, b1, nullptr, 0, p.error, s)) != cudaSuccess) return e;
       if ((e = sg_layer<GM_BIAS_RELU>(p.h1, H, W2, H, p.h2, H, n, H, H, b2, nullptr, 0, p.error, s)) != cudaSuccess) return e;

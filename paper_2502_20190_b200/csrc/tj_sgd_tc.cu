@@ -24,7 +24,7 @@ namespace {
 
 constexpr int T2_M = 128, T2_N = 256, T2_K = 16;
 constexpr int T2_WORKERS = 256, T2_THREADS = T2_WORKERS + 64, T2_PF = 3;
-constexpr int T2_ASTAGES = 4, T2_BSLOTS = 3;
+constexpr int T2_ASTAGES = 3, T2_BSLOTS = 4;
 constexpr int T2_STG_LD = 36;                              // floats per row of a warp's 32 x 32 staging block (144 bytes)
 constexpr int T2_STG_BYTES = (T2_WORKERS / 32) * 32 * T2_STG_LD * 4;   // 36 KB: one block per worker warp
 constexpr int T2_A_PART = T2_M * T2_K * 4;                 // 8 KB: one part of an A stage
