@@ -67,7 +67,9 @@ enum { TJ_W_FP32 = 0,      /* FP32 FMA in one fixed rounding order: outputs (and
        TJ_W_FP32_TC = 2 }; /* FP32 weights; the actor's hidden x hidden layer on the tensor cores as three products of split
                               operands (the role a 3 x TF32 product plays, here with FP16 parts at twice that rate; about
                               2^-22 per term): outputs within 1e-5 of TJ_W_FP32's, actions equal wherever the top-2 gap
-                              exceeds that.  CartPole / Acrobot, hidden 64 / 128 / 192 / 256.  tj_td_error runs its two
+                              exceeds that.  CartPole / Acrobot, hidden 64 / 128 / 192 / 256.  First-layer activations must
+                              stay below 4,094 (16 x that is FP16's range); a pass that sees a larger one latches
+                              device_error 5 and its outputs are meaningless.  tj_td_error runs its two
                               forwards the same way (same tolerance); tj_td_error_static and the parameter updates
                               use the FP32 kernels. */
 /* kernel classes reported by tj_stats (Sec. 3.3: performance analysis measures the production and the

@@ -41,6 +41,7 @@ struct SaCtl {
   uint64_t acc_full;             // all MMAs of a forward pass complete
   uint32_t tmem_base;
   int abort_flag;
+  int range_flag;               // a scaled hidden activation left FP16's range: the outputs of that pass are meaningless
 };
 
 __device__ __forceinline__ float4 sa_reset4(uint2 seed, uint32_t e, unsigned long long step, float lo, float width) {
@@ -70,7 +71,7 @@ struct SaShared {
 // eight hidden units n0 .. n0+7 of layer 1 for one env, in the canonical order (bias, then inputs in index order), ReLU,
 // scaling, split; one 16-byte row segment of each part of the A operand
 template <int D>
-__device__ __forceinline__ void sa_layer1_block(const MlpWeights& mw, int Hp, const float* x, int n0, uint8_t* a_hi, uint8_t* a_lo, size_t off) {
+__device__ __forceinline__ float sa_layer1_block(const MlpWeights& mw, int Hp, const float* x, int n0, uint8_t* a_hi, uint8_t* a_lo, size_t off) {
   float acc[8];
   const float4 b0 = *reinterpret_cast<const float4*>(mw.b1 + n0), b1 = *reinterpret_cast<const float4*>(mw.b1 + n0 + 4);
   acc[0] = b0.x; acc[1] = b0.y; acc[2] = b0.z; acc[3] = b0.w; acc[4] = b1.x; acc[5] = b1.y; acc[6] = b1.z; acc[7] = b1.w;
@@ -82,15 +83,18 @@ __device__ __forceinline__ void sa_layer1_block(const MlpWeights& mw, int Hp, co
     acc[4] = fmaf(w1.x, x[k], acc[4]); acc[5] = fmaf(w1.y, x[k], acc[5]); acc[6] = fmaf(w1.z, x[k], acc[6]); acc[7] = fmaf(w1.w, x[k], acc[7]);
   }
   uint32_t hi2[4], lo2[4];
+  float vmax = 0.f;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float v0 = fmaxf(acc[2 * i], 0.f) * SA_H_SCALE, v1 = fmaxf(acc[2 * i + 1], 0.f) * SA_H_SCALE;
+    vmax = fmaxf(vmax, fmaxf(v0, v1));
     const float h0 = __uint_as_float(__float_as_uint(v0) & 0xFFFFE000u), h1 = __uint_as_float(__float_as_uint(v1) & 0xFFFFE000u);
     hi2[i] = pack_f16x2(h0, h1);
     lo2[i] = pack_f16x2(v0 - h0, v1 - h1);
   }
   *reinterpret_cast<uint4*>(a_hi + off) = make_uint4(hi2[0], hi2[1], hi2[2], hi2[3]);
   *reinterpret_cast<uint4*>(a_lo + off) = make_uint4(lo2[0], lo2[1], lo2[2], lo2[3]);
+  return vmax;
 }
 
 // Network outputs of the observations in xs -> out[i][e], i < Aout.  Called by every thread of the block; `pass` counts the
@@ -111,17 +115,20 @@ __device__ __forceinline__ bool sa_forward(int Hp, int Aout, const MlpWeights& m
 #pragma unroll
     for (int k = 0; k < D; ++k) x[k] = sh.xs[k * SA_TE + e];
     tc_fence_before();                            // this thread's accumulator reads of the previous pass are complete
+    float vmax = 0.f;
 #pragma unroll 1
     for (int kc = 0; kc < NKC; ++kc) {
 #pragma unroll
       for (int b = 0; b < 2; ++b) {
         const int n0 = kc * SA_KC + half * 16 + b * 8;
         const size_t off = ((size_t)(e >> 3) * (H / 8) + (n0 >> 3)) * 128 + (e & 7) * 16;
-        sa_layer1_block<D>(mw, Hp, x, n0, sh.a_hi, sh.a_lo, off);
+        vmax = fmaxf(vmax, sa_layer1_block<D>(mw, Hp, x, n0, sh.a_hi, sh.a_lo, off));
       }
       fence_async_smem();
       mbar_arrive_warp(&ctl->a_ready[kc]);
     }
+    // 65,504 is FP16's largest finite value (a NaN activation also lands here: the comparison is written to catch it)
+    if (!(vmax <= 65504.f)) ctl->range_flag = 1;
   } else if (warp == SA_WORKERS / 32) {
     // The issuing lane's warp-mates wait at the warp barrier, not in a polling loop: lanes of one warp that poll while
     // another lane of it issues take turns with that lane, and every blocked poll then stalls the issue.
@@ -234,6 +241,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
     mbar_init(&ctl->wbar, 1);
     mbar_init(&ctl->acc_full, 1);
     ctl->abort_flag = 0;
+    ctl->range_flag = 0;
   }
   __syncthreads();
   if (warp == 0) {
@@ -379,6 +387,7 @@ __global__ void __launch_bounds__(SA_NT, 1) actor_split_tc_kernel(const ActorPar
     for (uint32_t g = pass * NSTREAM; g < copied; ++g)
       if (!tc_wait(&ctl->full[g % SA_SLOTS], (g / SA_SLOTS) & 1, abort_flag)) break;
     if (ctl->abort_flag) atomicExch(&p.stats->error, 4ull);
+    else if (ctl->range_flag) atomicExch(&p.stats->error, 5ull);
   }
   tc_fence_before();
   __syncthreads();
@@ -421,6 +430,7 @@ __global__ void __launch_bounds__(SA_NT, 1) td_split_tc_kernel(const TdParams p,
     mbar_init(&ctl->wbar, 1);
     mbar_init(&ctl->acc_full, 1);
     ctl->abort_flag = 0;
+    ctl->range_flag = 0;
   }
   __syncthreads();
   if (warp == 0) {
@@ -501,6 +511,7 @@ __global__ void __launch_bounds__(SA_NT, 1) td_split_tc_kernel(const TdParams p,
     for (int i = 0; i < n_here; ++i) sum += hub[i];
     p.partial[blockIdx.x] = sum;
     if (ctl->abort_flag && p.error) atomicExch(p.error, 4ull);
+    else if (ctl->range_flag && p.error) atomicExch(p.error, 5ull);
   }
   // the copies still in flight must land before the block gives its shared memory back
   if (tid == SA_WORKERS + 32) {

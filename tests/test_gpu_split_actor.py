@@ -206,3 +206,20 @@ def test_td_error_in_this_weight_mode_follows_the_lagging_target(env, kind, D, A
             assert moved[live].mean() > 0.9
             assert np.all(np.abs(g_td - td_fresh)[moved] > RTOL_FP32 * (np.abs(td) + terms)[moved])
     assert ctx.stats()["device_error"] == 0
+
+
+def test_activation_beyond_the_split_range_is_reported(env):
+    """The hidden activations are split after a scaling by 16, so they must stay below 4,094; parameters that push them
+    beyond that must not pass silently: the kernel latches device_error 5 (no fault, the context stays usable)."""
+    torch, orc, binding = env
+    f = _ring_fields(0, 4, 2, 64, 64)
+    ctx = binding.Context(**dict(f, weight_dtype=W_FP32_TC))
+    blob = blob_for(f, 1)
+    ctx.publish_weights(blob)
+    ctx.actor_step(2)
+    assert ctx.stats()["device_error"] == 0
+    big = blob.copy()
+    big[:64 * 4] *= 1e6                      # first-layer weights: activations of the order of 1e4 and more
+    ctx.publish_weights(big)
+    ctx.actor_step(1)
+    assert ctx.stats()["device_error"] == 5
